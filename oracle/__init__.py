@@ -1,0 +1,159 @@
+"""ctypes front end of the CPU oracle (test infrastructure, not product code).
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg import this
+package.  It compiles ``dte_oracle.cpp`` with g++ on first use and exposes the
+oracle's functions on numpy arrays.  Nothing here touches the CUDA library.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "dte_oracle.cpp")
+_LIB = os.path.join(_HERE, "libdte_oracle.so")
+_CXXFLAGS = ["-O2", "-std=c++17", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle into ``libdte_oracle.so`` next to its source."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.run(["g++", *_CXXFLAGS, "-o", tmp, _SRC], check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    with _lock:
+        if _lib is None:
+            L = ctypes.CDLL(build())
+            c = ctypes
+            L.oracle_derive_constants.argtypes = [c.c_int64, c.c_double, c.c_double, c.c_double,
+                                                  c.c_double, c.c_double, c.c_void_p]
+            L.oracle_derive_constants.restype = None
+            L.oracle_invert.argtypes = [c.c_void_p] * 3 + [c.c_uint64, c.c_void_p, c.c_void_p]
+            L.oracle_invert.restype = None
+            L.oracle_bf16_rne.argtypes = [c.c_void_p, c.c_uint64, c.c_void_p]
+            L.oracle_bf16_rne.restype = None
+            L.oracle_changed_mask.argtypes = [c.c_void_p] * 3 + [c.c_uint64] + [c.c_void_p] * 3
+            L.oracle_changed_mask.restype = c.c_uint64
+            L.oracle_extract.argtypes = [c.c_uint64, c.c_void_p, c.c_uint64, c.c_void_p, c.c_uint64,
+                                         c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+            L.oracle_extract.restype = c.c_void_p
+            L.oracle_result_error.argtypes = [c.c_void_p]
+            L.oracle_result_error.restype = c.c_char_p
+            L.oracle_result_total.argtypes = [c.c_void_p]
+            L.oracle_result_total.restype = c.c_uint64
+            L.oracle_result_copy.argtypes = [c.c_void_p] * 4
+            L.oracle_result_copy.restype = None
+            L.oracle_result_free.argtypes = [c.c_void_p]
+            L.oracle_result_free.restype = None
+            L.oracle_apply.argtypes = [c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
+                                       c.c_void_p]
+            L.oracle_apply.restype = c.c_int
+            _lib = L
+    return _lib
+
+
+def _f32(a) -> np.ndarray:
+    return np.ascontiguousarray(a, dtype=np.float32).reshape(-1)
+
+
+def derive_constants(step, lr, beta1, beta2, eps, wd) -> np.ndarray:
+    """{bc1, bc2, decay, lr, eps} as fp32 (Eq. 2's call-uniform scalars)."""
+    out = np.zeros(5, np.float32)
+    lib().oracle_derive_constants(int(step), float(lr), float(beta1), float(beta2), float(eps),
+                                  float(wd), out.ctypes.data)
+    return out
+
+
+def invert(theta, m, v, consts) -> np.ndarray:
+    """Reconstructed theta_{t-1} (Eq. 2), element-wise fp32."""
+    theta, m, v = _f32(theta), _f32(m), _f32(v)
+    c = _f32(consts)
+    prev = np.empty_like(theta)
+    lib().oracle_invert(theta.ctypes.data, m.ctypes.data, v.ctypes.data, theta.size,
+                        c.ctypes.data, prev.ctypes.data)
+    return prev
+
+
+def bf16_rne(x) -> np.ndarray:
+    """BF16 bit patterns (uint16) of fp32 inputs, round-to-nearest-even."""
+    x = _f32(x)
+    out = np.empty(x.size, np.uint16)
+    lib().oracle_bf16_rne(x.ctypes.data, x.size, out.ctypes.data)
+    return out
+
+
+def changed_mask(theta, m, v, consts):
+    """Eq. 4 on one tensor: (mask uint8[n], BF16(theta_t) uint16[n])."""
+    theta, m, v = _f32(theta), _f32(m), _f32(v)
+    c = _f32(consts)
+    mask = np.empty(theta.size, np.uint8)
+    val = np.empty(theta.size, np.uint16)
+    lib().oracle_changed_mask(theta.ctypes.data, m.ctypes.data, v.ctypes.data, theta.size,
+                              c.ctypes.data, mask.ctypes.data, val.ctypes.data)
+    return mask, val
+
+
+def _ptr_array(arrs):
+    return (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
+
+
+def extract(tensor_shapes, shard_numels, ops, theta, m, v, consts):
+    """Full extract (Eq. 2, 4, 5, 6) over a transfer plan.
+
+    tensor_shapes: [(n0, n1)] per source tensor; shard_numels: [numel] per
+    receiver-local tensor; ops: rows of 10 integers {src_tensor, dst_shard,
+    a_s0, a_s1, e0, e1, dst_base, dst_ld, a_r0, a_r1}; theta/m/v: lists of
+    fp32 arrays.  Returns (list_ptr uint64[n_shards+1], offsets uint32[M],
+    values uint16[M]).
+    """
+    L = lib()
+    shp = np.ascontiguousarray(tensor_shapes, dtype=np.int64).reshape(-1, 2)
+    num = np.ascontiguousarray(shard_numels, dtype=np.int64).reshape(-1)
+    op = np.ascontiguousarray(ops, dtype=np.int64).reshape(-1, 10)
+    th = [_f32(a) for a in theta]
+    mm = [_f32(a) for a in m]
+    vv = [_f32(a) for a in v]
+    for p in range(shp.shape[0]):
+        n = int(shp[p, 0] * shp[p, 1])
+        assert th[p].size == n and mm[p].size == n and vv[p].size == n, "tensor size mismatch"
+    c = _f32(consts)
+    h = L.oracle_extract(shp.shape[0], shp.ctypes.data, num.size, num.ctypes.data, op.shape[0],
+                         op.ctypes.data, _ptr_array(th), _ptr_array(mm), _ptr_array(vv),
+                         c.ctypes.data)
+    try:
+        err = L.oracle_result_error(h)
+        if err:
+            raise ValueError(err.decode())
+        total = L.oracle_result_total(h)
+        list_ptr = np.zeros(num.size + 1, np.uint64)
+        offsets = np.zeros(total, np.uint32)
+        values = np.zeros(total, np.uint16)
+        L.oracle_result_copy(h, list_ptr.ctypes.data, offsets.ctypes.data, values.ctypes.data)
+    finally:
+        L.oracle_result_free(h)
+    return list_ptr, offsets, values
+
+
+def apply(shard_numels, list_ptr, offsets, values, shards) -> None:
+    """Eq. 7 in place on ``shards`` (list of contiguous uint16 arrays)."""
+    num = np.ascontiguousarray(shard_numels, dtype=np.int64).reshape(-1)
+    lp = np.ascontiguousarray(list_ptr, dtype=np.uint64)
+    off = np.ascontiguousarray(offsets, dtype=np.uint32)
+    val = np.ascontiguousarray(values, dtype=np.uint16)
+    for k, s in enumerate(shards):
+        assert s.dtype == np.uint16 and s.flags.c_contiguous and s.size == num[k]
+    rc = lib().oracle_apply(num.size, num.ctypes.data, lp.ctypes.data, off.ctypes.data,
+                            val.ctypes.data, _ptr_array(shards))
+    if rc != 0:
+        raise ValueError("receiver index outside its shard")
