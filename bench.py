@@ -1,0 +1,454 @@
+#!/usr/bin/env python
+"""Benchmark of the delta-transfer hot path on synthetic Qwen3-8B-shaped optimizer state.
+
+One step = one pass of the whole path over the resident state: the fused extract kernel
+(AdamW inversion, BF16 compare, ordered compaction, receiver remap) followed by the apply
+kernel on the receiver shard buffers.  Prints one JSON line (rank 0).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload full|layers:L|config1|config4]
+    python bench.py --impl reference ...      # the CPU oracle, timed on the host cores
+
+With N > 1 (torchrun) every rank runs the same per-GPU workload on its own device: the
+path partitions by tensor with no data-path collective, so this is weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from synth import configs, plans  # noqa: E402
+
+METRIC = "delta_extract_scanned_GBps"
+UNIT = "GB/s"
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per scanned element of the extract kernel, from the ncu capture summarised in
+# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over a 2.3 GB case, per element).
+NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT = None
+
+
+def log(*a):
+    print(*a, file=sys.stderr, flush=True)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.rows = []
+        self.proc = None
+        self.index = index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), line.strip()))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        sm, mx, reasons = [], [], set()
+        rows = [r for t, r in self.rows if t0 <= t <= t1] or [r for _, r in self.rows[-3:]]
+        for r in rows:
+            f = [x.strip() for x in r.split(",")]
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except Exception:
+                continue
+            for name, val in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def build_workload(name: str, device):
+    if name == "full":
+        return configs.config3(device)
+    if name.startswith("layers:"):
+        return configs.config3(device, n_layers=int(name.split(":")[1]), with_embeddings=False)
+    if name == "config1":
+        return configs.config1()
+    if name == "config2":
+        return configs.config2()
+    if name == "config4":
+        return configs.config4(device)
+    raise SystemExit(f"unknown workload {name}")
+
+
+def materialize_resident(wl, device, dte):
+    """theta/m/v resident on the device; shards initialised to remapped BF16(true theta_{t-1})."""
+    plan = wl.plan
+    shards = [torch.zeros(n, dtype=torch.int16, device=device) for n in plan.shard_numels]
+    ops_by_tensor = {}
+    for o in plan.ops:
+        ops_by_tensor.setdefault(o[0], []).append(o)
+    st = configs.State([None] * plan.n_tensors, [None] * plan.n_tensors, [None] * plan.n_tensors,
+                       [None] * plan.n_tensors)
+    for p in range(plan.n_tensors):
+        one = wl.materialize(device, [p])
+        st.theta[p], st.m[p], st.v[p] = one.theta[p], one.m[p], one.v[p]
+        prev = one.prev_bf16[p].view(torch.int16).reshape(plan.tensor_shapes[p])
+        for (_, dst, a0, a1, e0, e1, base, ld, r0, r1) in ops_by_tensor.get(p, []):
+            shards[dst].as_strided((e0, e1), (ld, 1), base + r0 * ld + r1).copy_(prev[a0:a0 + e0, a1:a1 + e1])
+        del one, prev
+    return st, shards
+
+
+def reconstruction_vs_truth(plan, st, shards_after, init_vals, delta_host):
+    """FN = truly changed but not emitted (receiver left stale); FP = emitted but not truly changed."""
+    lp, off, val = delta_host
+    fp = 0
+    for k in range(plan.n_shards):
+        a, b = int(lp[k]), int(lp[k + 1])
+        if b > a:
+            fp += int((init_vals[a:b] == val[a:b]).sum().item())
+    ops_by_shard = {}
+    for o in plan.ops:
+        ops_by_shard.setdefault(o[1], []).append(o)
+    fn = 0
+    for k in range(plan.n_shards):
+        exp = torch.zeros_like(shards_after[k])
+        for (src, _, a0, a1, e0, e1, base, ld, r0, r1) in ops_by_shard.get(k, []):
+            s2 = st.theta[src].reshape(plan.tensor_shapes[src])[a0:a0 + e0, a1:a1 + e1]
+            exp.as_strided((e0, e1), (ld, 1), base + r0 * ld + r1).copy_(s2.to(torch.bfloat16).view(torch.int16))
+        fn += int((exp != shards_after[k]).sum().item())
+        del exp
+    return fn, fp
+
+
+def oracle_sample(wl, st, max_elements):
+    """Source tensors (in order) up to max_elements, copied to the host for the oracle."""
+    plan = wl.plan
+    chosen, n = [], 0
+    for p in range(plan.n_tensors):
+        if n + plan.numel(p) > max_elements and chosen:
+            break
+        chosen.append(p)
+        n += plan.numel(p)
+    return chosen, n
+
+
+def oracle_inputs(plan, st, chosen):
+    """Host arrays and the sub-plan (operations of the chosen tensors) in the oracle's format."""
+    ops = plan.ops_array()
+    ops = ops[np.isin(ops[:, 0], np.asarray(chosen))]
+    zero = np.zeros(0, np.float32)
+    cs = set(chosen)
+    shapes = [s if p in cs else (0, 1) for p, s in enumerate(plan.tensor_shapes)]
+    host = [[l[p].cpu().numpy() if p in cs else zero for p in range(plan.n_tensors)]
+            for l in (st.theta, st.m, st.v)]
+    return shapes, ops, host
+
+
+def time_oracle(wl, st, chosen):
+    import oracle
+    shapes, ops, host = oracle_inputs(wl.plan, st, chosen)
+    c = oracle.derive_constants(*wl.hp.as_args())
+    t0 = time.perf_counter()
+    res = oracle.extract(shapes, wl.plan.shard_numels, ops, *host, c)
+    return time.perf_counter() - t0, res
+
+
+def run_reference(args, rank):
+    """The CPU oracle, as it stands, on a bounded sample of the same workload."""
+    if rank != 0:
+        return
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    wl = build_workload(args.workload, dev)
+    plan = wl.plan
+    budget = int(args.ref_elements)
+    chosen, n = [], 0
+    for p in range(plan.n_tensors):
+        if n + plan.numel(p) > budget and chosen:
+            break
+        chosen.append(p); n += plan.numel(p)
+    st = wl.materialize(dev, chosen)
+    import oracle
+    shapes, ops, host = oracle_inputs(plan, st, chosen)
+    scanned = int((ops[:, 4] * ops[:, 5]).sum())
+    c = oracle.derive_constants(*wl.hp.as_args())
+    times, M = [], 0
+    for i in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        lp, off, val = oracle.extract(shapes, plan.shard_numels, ops, *host, c)
+        # apply is part of the step: scatter into receiver-sized host buffers
+        bufs = [np.zeros(nn if lp[k + 1] > lp[k] else 0, np.uint16) for k, nn in enumerate(plan.shard_numels)]
+        numels = [b.size for b in bufs]
+        oracle.apply(numels, lp, off, val, bufs)
+        dt = time.perf_counter() - t0
+        M = int(lp[-1])
+        if i >= args.warmup:
+            times.append(dt)
+    t = sum(times) / len(times)
+    value = (12.0 * scanned + 6.0 * M) / t / 1e9
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+           "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+           "config": {"workload": wl.name, "sample": f"first {len(chosen)} source tensors, {scanned} elements per step"},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                            "sample": f"first {len(chosen)} source tensors ({scanned} elements) of {wl.name}"},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "elements_per_s": scanned / t, "changed": M}
+    print(json.dumps(out), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="dte", choices=["dte", "reference"])
+    ap.add_argument("--workload", default="full")
+    ap.add_argument("--capacity-frac", type=float, default=0.03)
+    ap.add_argument("--e2e-gb", type=float, default=10.0, help="host-resident state for the e2e leg (GB)")
+    ap.add_argument("--cpu-elements", type=float, default=1.2e9, help="oracle sample size (elements)")
+    ap.add_argument("--ref-elements", type=float, default=4e8, help="--impl reference: elements per step")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU path); use --impl reference for the oracle")
+    import paper_2608_00455_b200 as dte
+
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    t_gen = time.time()
+    wl = build_workload(args.workload, device)
+    plan = wl.plan
+    st, shards = materialize_resident(wl, device, dte)
+    torch.cuda.synchronize()
+    log(f"[bench] generated {wl.name}: {plan.total_source_elements()} source elements in {time.time() - t_gen:.1f}s, "
+        f"{torch.cuda.memory_allocated() / 1e9:.1f} GB allocated")
+
+    lay = dte.Layout.from_plan(plan, local_rank)
+    N = lay.num_elements
+    delta = lay.new_delta(int(N * args.capacity_frac) + 1024)
+    tabs = lay.source_tables(st.theta, st.m, st.v)
+    shard_tab = lay.shard_table(shards)
+    hp = wl.hp.as_args()
+    stream = torch.cuda.current_stream()
+
+    # ---- untimed first pass: reconstruction-based change set vs the true one ----------------
+    dte.dte_extract_delta(lay, tabs, *hp, delta)
+    torch.cuda.synchronize()
+    bits = delta.status_bits()
+    if bits:
+        raise SystemExit(f"extract reported device status bits {bits} (capacity {delta.capacity}, total {delta.total()})")
+    M = delta.total()
+    lp_d = delta.list_ptr.cpu()
+    init_vals = torch.empty(M, dtype=torch.int16, device=device)
+    for k in range(plan.n_shards):
+        a, b = int(lp_d[k]), int(lp_d[k + 1])
+        if b > a:
+            init_vals[a:b] = shards[k][delta.offsets[a:b].to(torch.int64) & 0xFFFFFFFF]
+    dte.dte_apply(lay, delta, shard_tab)
+    torch.cuda.synchronize()
+    fn = fp = None
+    if rank == 0:
+        fn, fp = reconstruction_vs_truth(plan, st, shards, init_vals, (lp_d, delta.offsets, delta.values))
+    del init_vals
+    log(f"[bench] N={N} changed={M} ({100.0 * M / N:.3f} %), FN={fn} FP={fp}")
+
+    # ---- timed region -------------------------------------------------------------------------
+    def step(ev=None):
+        if ev: ev[0].record(stream)
+        dte.dte_extract_delta(lay, tabs, *hp, delta)
+        if ev: ev[1].record(stream)
+        dte.dte_apply(lay, delta, shard_tab)
+        if ev: ev[2].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    if dist: dist.barrier()
+    torch.cuda.synchronize()
+    w0 = time.time()
+    for i in range(args.steps):
+        step(evs[i])
+    torch.cuda.synchronize()
+    if dist: dist.barrier()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1) if rank == 0 else None
+    total_ms = evs[0][0].elapsed_time(evs[-1][2])
+    ext_ms = [e[0].elapsed_time(e[1]) for e in evs]
+    app_ms = [e[1].elapsed_time(e[2]) for e in evs]
+    launches = lay.last_launch()["kernels"] * args.steps + args.steps
+    if dist:
+        t = torch.tensor([total_ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    bytes_per_step = 12.0 * N + 6.0 * M
+    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    ext_avg = sum(ext_ms) / len(ext_ms)
+    app_avg = sum(app_ms) / len(app_ms)
+    peak, peak_kind = measured_peak()
+    achieved = bytes_per_step / (ext_avg * 1e-3) / 1e9
+    traffic = None
+    if NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT is not None:
+        traffic = NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT * N
+
+    # ---- end to end through the host-buffer entry point -----------------------------------------
+    e2e = None
+    if not args.no_e2e:
+        e2e = run_e2e(args, wl, st, device, dte, world, dist)
+
+    # ---- CPU baseline: the oracle on a bounded sample ---------------------------------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        chosen, n_el = oracle_sample(wl, st, int(args.cpu_elements))
+        dt, res = time_oracle(wl, st, chosen)
+        ops = plan.ops_array()
+        ops = ops[np.isin(ops[:, 0], chosen)]
+        scanned = int((ops[:, 4] * ops[:, 5]).sum())
+        m_cpu = int(res[0][-1])
+        # the sampled lists must equal the GPU's
+        lp_g, off_g, val_g = delta.to_host()
+        ok = True
+        for k in sorted(set(int(x) for x in ops[:, 1])):
+            full = all(int(o[0]) in chosen for o in plan.ops if o[1] == k)
+            if not full:
+                continue
+            a, b, c, d = int(lp_g[k]), int(lp_g[k + 1]), int(res[0][k]), int(res[0][k + 1])
+            ok &= (b - a == d - c) and np.array_equal(off_g[a:b], res[1][c:d]) and np.array_equal(val_g[a:b], res[2][c:d])
+        cpu = {"value": (12.0 * scanned + 6.0 * m_cpu) / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"first {len(chosen)} source tensors ({scanned} scanned elements) of {wl.name}, extract only, "
+                         f"{dt:.1f} s", "elements_per_s": scanned / dt, "lists_equal_gpu": bool(ok)}
+
+    if rank == 0:
+        out = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": wl.name, "elements_scanned": N, "changed": M, "changed_frac": M / N,
+                       "lists": lay.num_lists, "l2": "inputs larger than L2 (no flush needed)" if 12 * N > 1e9 else "inputs smaller than 1 GB",
+                       "hyper": {"step": wl.hp.step, "lr": wl.hp.lr, "wd": wl.hp.wd}, **wl.notes},
+            "extract": {"ms": ext_avg, "ms_min": min(ext_ms), "GBps": achieved, "elements_per_s": N / (ext_avg * 1e-3),
+                        "frac_of_8TBps": achieved / 8000.0},
+            "apply": {"ms": app_avg, "ms_min": min(app_ms), "Mchanged_per_s": M / (app_avg * 1e-3) / 1e6,
+                      "GBps_algorithmic": 8.0 * M / (app_avg * 1e-3) / 1e9},
+            "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": traffic, "peak_source": peak_kind, "kernel": "extract_kernel"},
+            "reconstruction_vs_truth": {"false_negatives": fn, "false_positives": fp, "variant": wl.variant},
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
+            "launch": lay.last_launch(),
+        }
+        print(json.dumps(out), flush=True)
+    if dist:
+        dist.destroy_process_group()
+
+
+def run_e2e(args, wl, st, device, dte, world, dist):
+    """Same metric through dte_extract_delta_host: pinned host theta/m/v -> device -> extract ->
+    apply -> lists back to the host, copies inside the timed region."""
+    plan = wl.plan
+    budget = int(args.e2e_gb * 1e9 / 12)
+    chosen, n = [], 0
+    for p in range(plan.n_tensors):
+        if n + plan.numel(p) > budget and chosen:
+            break
+        chosen.append(p); n += plan.numel(p)
+    sub = plans.Plan()
+    remap = {}
+    for p in chosen:
+        remap[p] = sub.add_tensor(plan.tensor_names[p], plan.tensor_shapes[p])
+    kmap = {}
+    for o in plan.ops:
+        if o[0] in remap:
+            if o[1] not in kmap:
+                kmap[o[1]] = sub.add_shard(plan.shard_names[o[1]], plan.shard_receivers[o[1]], plan.shard_numels[o[1]])
+            sub.ops.append((remap[o[0]], kmap[o[1]]) + tuple(o[2:]))
+    lay = dte.Layout.from_plan(sub, device.index)
+    th, mm, vv = ([lst[p].cpu().pin_memory() for p in chosen] for lst in (st.theta, st.m, st.v))
+    ws = torch.empty(lay.host_workspace_bytes, dtype=torch.uint8, device=device)
+    N = lay.num_elements
+    delta = lay.new_delta(int(N * args.capacity_frac) + 1024)
+    res = dte.HostResult(lay.num_lists, delta.capacity)
+    shards = [torch.zeros(nn, dtype=torch.int16, device=device) for nn in sub.shard_numels]
+    tab = lay.shard_table(shards)
+    hp = wl.hp.as_args()
+    stream = torch.cuda.current_stream()
+
+    def step():
+        dte.dte_extract_delta_host(lay, th, mm, vv, *hp, ws, delta, res)
+        dte.dte_apply(lay, delta, tab)
+
+    for _ in range(2):
+        step()
+    torch.cuda.synchronize()
+    steps = max(2, min(args.steps, 5))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    if dist: dist.barrier()
+    torch.cuda.synchronize()
+    e0.record(stream)
+    for _ in range(steps):
+        step()
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    if dist:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    M = int(res.counters[0])
+    h2d = 12 * sub.total_source_elements()
+    d2h = 6 * M + 8 * (lay.num_lists + 1) + 32
+    return {"value": world * (12.0 * N + 6.0 * M) / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps,
+            "workload": f"first {len(chosen)} source tensors of {wl.name} held in pinned host memory "
+                        f"({N} scanned elements); PCIe-bound"}
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,190 @@
+/*
+ * dte.h - C ABI of the B200 delta-transfer hot path.
+ *
+ * One pass over a trainer's live AdamW state produces, for every receiver-local
+ * inference tensor, the ordered list of BF16 elements that changed in the last
+ * optimizer step; a second call scatters such lists into BF16 shard buffers.
+ *
+ * The operations follow the paper's problem statement:
+ *   - Eq. 2 (Section 4.1): the previous fp32 master weight is reconstructed from the
+ *     current weight and the AdamW moments by inverting the decoupled AdamW step;
+ *   - Eq. 4 (Section 4.2.1): both versions are cast to BF16, their 16-bit patterns are
+ *     compared, and changed indices with their *target* values are extracted;
+ *   - Eq. 5-6 (Section 4.2.2): each changed index is unravelled, matched against the
+ *     precomputed hyper-rectangular overlaps of the transfer plan, and ravelled into
+ *     receiver-local coordinates;
+ *   - Eq. 7 (Section 4.3): the receiver scatters the values into its live shard.
+ *
+ * Conventions
+ *   - "device pointer" = CUDA global memory of the layout's device; "host pointer" =
+ *     ordinary or pinned host memory.  The library never frees or keeps caller memory.
+ *   - All tensors are row-major and contiguous.  fp32 inputs must be 16-byte aligned.
+ *   - Every call that takes a stream enqueues on it (void* = cudaStream_t; NULL = the
+ *     default stream) and returns without synchronising unless stated otherwise.
+ *   - Functions return DTE_OK or an error detected on the host.  Conditions only the
+ *     device can detect are reported as DTE_DEV_* bits in dte_delta.counters[2].
+ *   - A layout may be used by one extract or apply call at a time (its scratch memory
+ *     is per layout).  Different layouts are independent.
+ *   - There is no CPU fallback: every entry point needs a CUDA device.
+ */
+#ifndef DTE_H_
+#define DTE_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define DTE_API __attribute__((visibility("default")))
+#else
+#define DTE_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum dte_status {
+    DTE_OK = 0,
+    DTE_ERR_INVALID_ARG = 1, /* null pointer, bad hyper-parameter, misaligned tensor      */
+    DTE_ERR_LAYOUT = 2,      /* the tensor / shard / operation tables are inconsistent    */
+    DTE_ERR_CAPACITY = 3,    /* a caller-provided buffer is too small (host-detected)     */
+    DTE_ERR_BOUNDS = 4,      /* reserved for host-side bound checks                       */
+    DTE_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (host variant reports) */
+    DTE_ERR_CUDA = 6         /* a CUDA runtime call failed; see dte_last_error()          */
+} dte_status;
+
+/* Device-detected conditions, OR-ed into dte_delta.counters[2]. */
+#define DTE_DEV_OVERFLOW 1u /* more changed elements than `capacity`; extra ones dropped */
+#define DTE_DEV_BOUNDS 2u   /* apply met an offset >= numel of its shard; entry skipped  */
+#define DTE_DEV_TIMEOUT 4u  /* a bounded wait inside the extract kernel ran out          */
+
+/* Source tensor p of the canonical training-side space: fp32, row-major.  ndim is 1 or 2;
+ * for ndim == 1 shape[1] must be 1.  `group` (parameter group) is reserved: must be 0. */
+typedef struct dte_tensor_desc {
+    uint64_t shape[2];
+    uint32_t ndim;
+    uint32_t group;
+} dte_tensor_desc;
+
+/* Receiver-local destination tensor q, flattened; BF16; numel < 2^32.  One output list
+ * per shard descriptor, in descriptor order.  `receiver` is informational. */
+typedef struct dte_shard_desc {
+    uint64_t numel;
+    uint32_t receiver;
+    uint32_t reserved;
+} dte_shard_desc;
+
+/* One operation o of the transfer plan (Section 4.2.2): the overlap of source tensor
+ * `src_tensor` and destination `dst_shard`.  A source coordinate u with
+ *     src_origin <= u < src_origin + extent      (component-wise, Eq. 5 and the test after it)
+ * maps to the receiver-local flat index (Eq. 6)
+ *     j = dst_base + (u0 - src_origin[0] + dst_origin[0]) * dst_ld + (u1 - src_origin[1] + dst_origin[1]).
+ * The destination region must be one contiguous flat range: either whole destination rows
+ * (dst_origin[1] == 0 and extent[1] == dst_ld) or a single row (extent[0] == 1).
+ * Regions of different operations in the same shard must not overlap; slots no operation
+ * covers are never emitted and never written. */
+typedef struct dte_op_desc {
+    uint32_t src_tensor;
+    uint32_t dst_shard;
+    uint64_t src_origin[2];
+    uint64_t extent[2];
+    uint64_t dst_base;
+    uint64_t dst_ld;
+    uint64_t dst_origin[2];
+} dte_op_desc;
+
+typedef struct dte_layout dte_layout;
+
+/* Output of extract / input of apply.  All pointers are device pointers owned by the
+ * caller.  List k (shard k) occupies entries [list_ptr[k], list_ptr[k+1]) of `offsets`
+ * (receiver-local element offsets, strictly ascending within a list) and `values` (BF16
+ * bit patterns of theta_t, Eq. 4).  Empty lists keep their slot.
+ *   offsets  : capacity x uint32        values : capacity x uint16
+ *   list_ptr : (n_shards + 1) x uint64
+ *   counters : 4 x uint64 = { total changed, elements scanned, DTE_DEV_* bits, 0 }
+ * If the total exceeds `capacity`, entries at positions >= capacity are dropped,
+ * DTE_DEV_OVERFLOW is set, and list_ptr / counters[0] still hold the exact sizes, so
+ * the caller can grow the buffers and call again. */
+typedef struct dte_delta {
+    uint32_t* offsets;
+    uint16_t* values;
+    uint64_t capacity;
+    uint64_t* list_ptr;
+    uint64_t* counters;
+} dte_delta;
+
+/* Compiles the plan into device tables on `device` (Section 4.2.2: the plan is computed
+ * once from shard metadata, before any synchronisation).  Host arrays in, handle out.
+ * Allocates the layout's device tables and scratch with cudaMalloc; synchronous.
+ * Errors: DTE_ERR_INVALID_ARG (null arrays, ndim, group != 0), DTE_ERR_LAYOUT (operation
+ * outside its tensor or shard, non-contiguous or overlapping destination regions,
+ * numel >= 2^32), DTE_ERR_CUDA. */
+DTE_API dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n_tensors,
+                             const dte_shard_desc* shards, size_t n_shards,
+                             const dte_op_desc* ops, size_t n_ops, int device, dte_layout** out);
+
+/* Frees the handle and its device memory.  NULL is ignored. */
+DTE_API void dte_layout_destroy(dte_layout* layout);
+
+/* Number of output lists (== n_shards). */
+DTE_API size_t dte_layout_num_lists(const dte_layout* layout);
+/* Elements one extract call scans (sum of extents; replicated tensors count per copy). */
+DTE_API uint64_t dte_layout_num_elements(const dte_layout* layout);
+/* Bytes of device workspace dte_extract_delta_host needs (12 bytes per source element,
+ * each tensor padded to 256 bytes). */
+DTE_API uint64_t dte_layout_host_workspace_bytes(const dte_layout* layout);
+
+/* The call-uniform fp32 scalars of Eq. 2, derived in double and rounded once:
+ * out5 = { 1-beta1^step, 1-beta2^step, 1-lr*wd, lr, eps }.  Host only.
+ * Errors (DTE_ERR_INVALID_ARG): step < 1, betas outside [0,1), eps < 0, non-finite
+ * inputs, lr*wd >= 1, or a bias correction / decay that rounds to <= 0. */
+DTE_API dte_status dte_derive_constants(int64_t step, double lr, double beta1, double beta2, double eps,
+                                double wd, float* out5);
+
+/* Eq. 2 + Eq. 4 + Eq. 5-6 in one streaming pass.  theta / m / v: HOST arrays of
+ * n_tensors DEVICE pointers (fp32, 16-byte aligned; entries of tensors no operation
+ * reads may be NULL).  `step` is the 1-based index of the optimizer step that produced
+ * theta.  Arithmetic: IEEE binary32, every operation rounded to nearest-even on its own,
+ * no fused multiply-add across operations, subnormals kept; BF16 by round-to-nearest-even
+ * with NaN -> 0x7FC0; +0 and -0 are different patterns.  Deterministic: the same inputs
+ * give the same bytes.  Writes every field of `out` described above. */
+DTE_API dte_status dte_extract_delta(const dte_layout* layout, const float* const* theta,
+                             const float* const* m, const float* const* v, int64_t step,
+                             double lr, double beta1, double beta2, double eps, double wd,
+                             const dte_delta* out, void* cuda_stream);
+
+/* Eq. 7: shard[k][offsets[e]] = values[e] for every entry e of every list k.
+ * shard_ptrs: HOST array of n_shards DEVICE pointers (BF16 buffers, numel as declared;
+ * shards whose lists are necessarily empty may be NULL).  Reads list sizes on the device,
+ * so it can be enqueued right after extract without a host round trip.  Refuses to write
+ * anything (and sets DTE_DEV_OVERFLOW again) if `delta` overflowed its capacity. */
+DTE_API dte_status dte_apply(const dte_layout* layout, const dte_delta* delta,
+                     uint16_t* const* shard_ptrs, void* cuda_stream);
+
+/* End-to-end variant for optimizer state that lives in HOST memory (pinned for full
+ * copy speed).  Copies theta / m / v (HOST arrays of n_tensors HOST pointers) into
+ * `workspace` (device, >= dte_layout_host_workspace_bytes), runs the same extract into
+ * `out` (device buffers, as above), then copies counters, list_ptr and the filled part
+ * of offsets / values to the given host buffers (offsets_h / values_h hold `capacity`
+ * entries; either may be NULL to skip that copy).  SYNCHRONISES the stream before
+ * returning.  Returns DTE_ERR_CAPACITY if the delta overflowed. */
+DTE_API dte_status dte_extract_delta_host(const dte_layout* layout, const float* const* theta_h,
+                                  const float* const* m_h, const float* const* v_h, int64_t step,
+                                  double lr, double beta1, double beta2, double eps, double wd,
+                                  void* workspace, uint64_t workspace_bytes, const dte_delta* out,
+                                  uint32_t* offsets_h, uint16_t* values_h, uint64_t* list_ptr_h,
+                                  uint64_t* counters_h, void* cuda_stream);
+
+/* Static strings. */
+DTE_API const char* dte_status_string(dte_status s);
+/* Message of the calling thread's most recent failed call ("" if none). */
+DTE_API const char* dte_last_error(void);
+
+/* Launch statistics of the most recent extract on this layout (host bookkeeping):
+ * out3 = { tiles, CTAs launched, kernels launched by the call }. */
+DTE_API void dte_layout_last_launch(const dte_layout* layout, uint64_t* out3);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DTE_H_ */

@@ -1,0 +1,286 @@
+"""Thin ctypes binding of libdte.so: argument marshalling only.
+
+Every step of the path runs in the CUDA library; torch is used for device
+memory and streams.  The names mirror the C ABI (include/dte.h).  There is no
+fallback: importing works without a GPU (so that symbols can be checked), but
+every compute call needs the library and a CUDA device and raises otherwise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import List, Optional, Sequence
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+DTE_OK = 0
+DTE_DEV_OVERFLOW, DTE_DEV_BOUNDS, DTE_DEV_TIMEOUT = 1, 2, 4
+
+SYMBOLS = [
+    "dte_layout_create", "dte_layout_destroy", "dte_layout_num_lists", "dte_layout_num_elements",
+    "dte_layout_host_workspace_bytes", "dte_derive_constants", "dte_extract_delta", "dte_apply",
+    "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
+]
+
+
+class TensorDesc(C.Structure):
+    _fields_ = [("shape", C.c_uint64 * 2), ("ndim", C.c_uint32), ("group", C.c_uint32)]
+
+
+class ShardDesc(C.Structure):
+    _fields_ = [("numel", C.c_uint64), ("receiver", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class OpDesc(C.Structure):
+    _fields_ = [("src_tensor", C.c_uint32), ("dst_shard", C.c_uint32),
+                ("src_origin", C.c_uint64 * 2), ("extent", C.c_uint64 * 2),
+                ("dst_base", C.c_uint64), ("dst_ld", C.c_uint64), ("dst_origin", C.c_uint64 * 2)]
+
+
+class DeltaStruct(C.Structure):
+    _fields_ = [("offsets", C.c_void_p), ("values", C.c_void_p), ("capacity", C.c_uint64),
+                ("list_ptr", C.c_void_p), ("counters", C.c_void_p)]
+
+
+class DteError(RuntimeError):
+    def __init__(self, status: int, msg: str):
+        super().__init__(f"dte status {status}: {msg}")
+        self.status = status
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _build.LIB
+
+
+def lib() -> C.CDLL:
+    """Loads libdte.so, building it first if the sources are newer."""
+    global _lib
+    if _lib is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        vp, u64, i64, dbl = C.c_void_p, C.c_uint64, C.c_int64, C.c_double
+        L.dte_layout_create.argtypes = [vp, C.c_size_t, vp, C.c_size_t, vp, C.c_size_t, C.c_int, C.POINTER(vp)]
+        L.dte_layout_create.restype = C.c_int
+        L.dte_layout_destroy.argtypes = [vp]
+        L.dte_layout_destroy.restype = None
+        L.dte_layout_num_lists.argtypes = [vp]
+        L.dte_layout_num_lists.restype = C.c_size_t
+        L.dte_layout_num_elements.argtypes = [vp]
+        L.dte_layout_num_elements.restype = u64
+        L.dte_layout_host_workspace_bytes.argtypes = [vp]
+        L.dte_layout_host_workspace_bytes.restype = u64
+        L.dte_derive_constants.argtypes = [i64, dbl, dbl, dbl, dbl, dbl, vp]
+        L.dte_derive_constants.restype = C.c_int
+        L.dte_extract_delta.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, vp]
+        L.dte_extract_delta.restype = C.c_int
+        L.dte_apply.argtypes = [vp, vp, vp, vp]
+        L.dte_apply.restype = C.c_int
+        L.dte_extract_delta_host.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, u64,
+                                             vp, vp, vp, vp, vp, vp]
+        L.dte_extract_delta_host.restype = C.c_int
+        L.dte_status_string.argtypes = [C.c_int]
+        L.dte_status_string.restype = C.c_char_p
+        L.dte_last_error.argtypes = []
+        L.dte_last_error.restype = C.c_char_p
+        L.dte_layout_last_launch.argtypes = [vp, vp]
+        L.dte_layout_last_launch.restype = None
+        _lib = L
+    return _lib
+
+
+def _check(status: int) -> None:
+    if status != DTE_OK:
+        L = lib()
+        msg = L.dte_last_error().decode() or L.dte_status_string(status).decode()
+        raise DteError(status, msg)
+
+
+def _require_cuda() -> None:
+    if not torch.cuda.is_available():
+        raise RuntimeError("the delta-transfer path needs a CUDA device; there is no CPU fallback")
+
+
+def dte_derive_constants(step, lr, beta1, beta2, eps, wd) -> np.ndarray:
+    out = np.zeros(5, np.float32)
+    _check(lib().dte_derive_constants(int(step), float(lr), float(beta1), float(beta2), float(eps),
+                                      float(wd), out.ctypes.data))
+    return out
+
+
+def _ptr_table(tensors: Sequence[Optional[torch.Tensor]], dtype, device=None):
+    arr = (C.c_void_p * max(1, len(tensors)))()
+    for i, t in enumerate(tensors):
+        if t is None:
+            arr[i] = None
+            continue
+        assert t.dtype == dtype and t.is_contiguous(), "tensor dtype / contiguity"
+        if device is not None:
+            assert t.device == device, f"tensor on {t.device}, layout on {device}"
+        arr[i] = t.data_ptr()
+    return arr
+
+
+class Delta:
+    """Caller-owned device buffers of one extract result (see dte_delta in dte.h)."""
+
+    def __init__(self, n_lists: int, capacity: int, device):
+        dev = torch.device(device)
+        self.capacity = int(capacity)
+        self.n_lists = int(n_lists)
+        self.offsets = torch.empty(max(1, self.capacity), dtype=torch.int32, device=dev)   # uint32 bits
+        self.values = torch.empty(max(1, self.capacity), dtype=torch.int16, device=dev)    # bf16 bits
+        self.list_ptr = torch.zeros(self.n_lists + 1, dtype=torch.int64, device=dev)
+        self.counters = torch.zeros(4, dtype=torch.int64, device=dev)
+        self.struct = DeltaStruct(self.offsets.data_ptr(), self.values.data_ptr(), self.capacity,
+                                  self.list_ptr.data_ptr(), self.counters.data_ptr())
+
+    # host views (synchronise)
+    def total(self) -> int:
+        return int(self.counters[0].item())
+
+    def status_bits(self) -> int:
+        return int(self.counters[2].item())
+
+    def to_host(self):
+        lp = self.list_ptr.cpu().numpy().astype(np.uint64)
+        n = min(int(lp[-1]), self.capacity)
+        off = self.offsets[:n].cpu().numpy().view(np.uint32)
+        val = self.values[:n].cpu().numpy().view(np.uint16)
+        return lp, off, val
+
+
+class Layout:
+    """dte_layout handle built from a plan (tensor shapes, shard sizes, operation rows)."""
+
+    def __init__(self, tensor_shapes, shard_numels, ops, device=0, shard_receivers=None):
+        _require_cuda()
+        self.device = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
+        shapes = [(int(s[0]), int(s[1]) if len(s) > 1 else 1) for s in tensor_shapes]
+        self.tensor_shapes = shapes
+        self.shard_numels = [int(n) for n in shard_numels]
+        T = (TensorDesc * max(1, len(shapes)))()
+        for i, (a, b) in enumerate(shapes):
+            T[i].shape[0], T[i].shape[1] = a, b
+            T[i].ndim = 1 if b == 1 else 2
+            T[i].group = 0
+        S = (ShardDesc * max(1, len(self.shard_numels)))()
+        for k, n in enumerate(self.shard_numels):
+            S[k].numel = n
+            S[k].receiver = int(shard_receivers[k]) if shard_receivers is not None else 0
+        ops = np.asarray(ops, dtype=np.int64).reshape(-1, 10)
+        O = (OpDesc * max(1, ops.shape[0]))()
+        for i, r in enumerate(ops):
+            O[i].src_tensor, O[i].dst_shard = int(r[0]), int(r[1])
+            O[i].src_origin[0], O[i].src_origin[1] = int(r[2]), int(r[3])
+            O[i].extent[0], O[i].extent[1] = int(r[4]), int(r[5])
+            O[i].dst_base, O[i].dst_ld = int(r[6]), int(r[7])
+            O[i].dst_origin[0], O[i].dst_origin[1] = int(r[8]), int(r[9])
+        h = C.c_void_p()
+        _check(lib().dte_layout_create(T, len(shapes), S, len(self.shard_numels), O, ops.shape[0],
+                                       self.device.index or 0, C.byref(h)))
+        self._h = h
+
+    @classmethod
+    def from_plan(cls, plan, device=0):
+        return cls(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), device, plan.shard_receivers)
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().dte_layout_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    @property
+    def num_lists(self) -> int:
+        return int(lib().dte_layout_num_lists(self._h))
+
+    @property
+    def num_elements(self) -> int:
+        return int(lib().dte_layout_num_elements(self._h))
+
+    @property
+    def host_workspace_bytes(self) -> int:
+        return int(lib().dte_layout_host_workspace_bytes(self._h))
+
+    def last_launch(self):
+        out = (C.c_uint64 * 3)()
+        lib().dte_layout_last_launch(self._h, out)
+        return dict(tiles=int(out[0]), ctas=int(out[1]), kernels=int(out[2]))
+
+    def new_delta(self, capacity: int) -> Delta:
+        return Delta(self.num_lists, capacity, self.device)
+
+    def source_tables(self, theta, m, v):
+        """Marshal the three pointer tables once (reusable across calls)."""
+        return (_ptr_table(theta, torch.float32, self.device), _ptr_table(m, torch.float32, self.device),
+                _ptr_table(v, torch.float32, self.device))
+
+    def shard_table(self, shards):
+        tabs = []
+        for s in shards:
+            assert s is None or s.dtype in (torch.bfloat16, torch.int16)
+            tabs.append(s)
+        arr = (C.c_void_p * max(1, len(tabs)))()
+        for i, t in enumerate(tabs):
+            arr[i] = None if t is None else t.data_ptr()
+            assert t is None or (t.is_contiguous() and t.device == self.device)
+        return arr
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return stream.cuda_stream
+
+
+def dte_extract_delta(layout: Layout, tables, step, lr, beta1, beta2, eps, wd, delta: Delta,
+                      stream=None) -> None:
+    """Enqueue one extract.  `tables` = layout.source_tables(theta, m, v)."""
+    th, mm, vv = tables
+    _check(lib().dte_extract_delta(layout._h, th, mm, vv, int(step), float(lr), float(beta1),
+                                   float(beta2), float(eps), float(wd), C.byref(delta.struct),
+                                   _stream_ptr(stream)))
+
+
+def dte_apply(layout: Layout, delta: Delta, shard_table, stream=None) -> None:
+    """Enqueue one apply.  `shard_table` = layout.shard_table(shards)."""
+    _check(lib().dte_apply(layout._h, C.byref(delta.struct), shard_table, _stream_ptr(stream)))
+
+
+class HostResult:
+    def __init__(self, n_lists, capacity, pin=True):
+        self.offsets = torch.empty(max(1, capacity), dtype=torch.int32, pin_memory=pin)
+        self.values = torch.empty(max(1, capacity), dtype=torch.int16, pin_memory=pin)
+        self.list_ptr = torch.zeros(n_lists + 1, dtype=torch.int64, pin_memory=pin)
+        self.counters = torch.zeros(4, dtype=torch.int64, pin_memory=pin)
+
+    def arrays(self):
+        lp = self.list_ptr.numpy().astype(np.uint64)
+        n = int(lp[-1])
+        return lp, self.offsets[:n].numpy().view(np.uint32), self.values[:n].numpy().view(np.uint16)
+
+
+def dte_extract_delta_host(layout: Layout, theta_h, m_h, v_h, step, lr, beta1, beta2, eps, wd,
+                           workspace: torch.Tensor, delta: Delta, result: HostResult,
+                           stream=None) -> None:
+    """Host-resident theta / m / v in, device delta + host copy of the lists out (synchronous)."""
+    th = _ptr_table(theta_h, torch.float32)
+    mm = _ptr_table(m_h, torch.float32)
+    vv = _ptr_table(v_h, torch.float32)
+    assert workspace.device == layout.device and workspace.is_contiguous()
+    _check(lib().dte_extract_delta_host(
+        layout._h, th, mm, vv, int(step), float(lr), float(beta1), float(beta2), float(eps), float(wd),
+        workspace.data_ptr(), workspace.numel() * workspace.element_size(), C.byref(delta.struct),
+        result.offsets.data_ptr(), result.values.data_ptr(), result.list_ptr.data_ptr(),
+        result.counters.data_ptr(), _stream_ptr(stream)))

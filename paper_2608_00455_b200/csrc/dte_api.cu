@@ -1,0 +1,205 @@
+// C entry points that enqueue the kernels: dte_extract_delta, dte_apply and the
+// host-buffer variant dte_extract_delta_host.
+#include <cstring>
+
+#include "dte_internal.cuh"
+
+using namespace dte;
+
+namespace {
+
+dte_status fail(dte_status s, const char* msg) {
+    set_error(msg);
+    return s;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev) {
+        cudaGetDevice(&prev);
+        if (prev != dev) cudaSetDevice(dev); else prev = -1;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+dte_status check_delta(const dte_delta* d) {
+    if (!d) return fail(DTE_ERR_INVALID_ARG, "delta is null");
+    if (!d->list_ptr || !d->counters) return fail(DTE_ERR_INVALID_ARG, "delta.list_ptr / counters is null");
+    if (d->capacity && (!d->offsets || !d->values))
+        return fail(DTE_ERR_INVALID_ARG, "delta.offsets / values is null with capacity > 0");
+    return DTE_OK;
+}
+
+// Upload the per-call source pointer table unless it equals the one already on the device.
+dte_status sync_source_table(dte_layout* L, const float* const* theta, const float* const* m,
+                             const float* const* v, cudaStream_t st) {
+    const size_t n = L->n_tensors;
+    std::vector<const float*> tab(3 * n);
+    for (size_t p = 0; p < n; ++p) {
+        tab[p] = theta[p]; tab[n + p] = m[p]; tab[2 * n + p] = v[p];
+        if (!L->tensor_used[p]) continue;
+        if (!theta[p] || !m[p] || !v[p]) return fail(DTE_ERR_INVALID_ARG, "null theta / m / v pointer for a tensor the plan reads");
+        if (((uintptr_t)theta[p] | (uintptr_t)m[p] | (uintptr_t)v[p]) & 15u)
+            return fail(DTE_ERR_INVALID_ARG, "theta / m / v must be 16-byte aligned");
+    }
+    if (L->ptrs_valid && tab == L->h_ptrs) return DTE_OK;
+    L->ptrs_valid = false;
+    // pageable source: the runtime stages the bytes before returning, so `tab` may die
+    if (n) DTE_CUDA(cudaMemcpyAsync((void*)L->d_ptrs, tab.data(), tab.size() * sizeof(void*), cudaMemcpyHostToDevice, st));
+    L->h_ptrs.swap(tab);
+    L->ptrs_valid = true;
+    return DTE_OK;
+}
+
+dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out, cudaStream_t st) {
+    uint64_t launches = 0;
+    DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
+    if (L->n_tiles == 0) {
+        DTE_CUDA(cudaMemsetAsync(out->list_ptr, 0, (L->n_lists + 1) * sizeof(uint64_t), st));
+        L->last_launch[0] = 0; L->last_launch[1] = 0; L->last_launch[2] = 0;
+        return DTE_OK;
+    }
+    DTE_CUDA(cudaMemsetAsync(L->d_status, 0, ((size_t)L->n_tiles + 1) * sizeof(uint64_t), st));
+    ExtractParams p;
+    p.tiles = L->d_tiles;
+    p.segs = L->d_segs;
+    p.theta = L->d_ptrs;
+    p.m = L->d_ptrs + L->n_tensors;
+    p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
+    p.status = L->d_status;
+    p.ticket = reinterpret_cast<unsigned int*>(L->d_status + L->n_tiles);
+    p.n_tiles = L->n_tiles;
+    p.n_lists = L->n_lists;
+    p.scanned = L->scanned;
+    p.offsets = out->offsets;
+    p.values = out->values;
+    p.capacity = out->capacity;
+    p.list_ptr = out->list_ptr;
+    p.counters = out->counters;
+    p.c = c;
+    const int n_ctas = (int)std::min<uint64_t>(L->n_tiles, (uint64_t)L->max_ctas);
+    dte_status s = launch_extract(p, n_ctas, st);
+    if (s != DTE_OK) return s;
+    ++launches;
+    if (L->has_tileless_lists) {
+        s = launch_fill_empty_lists(out->list_ptr, L->d_next_with_tiles, L->n_lists, st);
+        if (s != DTE_OK) return s;
+        ++launches;
+    }
+    L->last_launch[0] = L->n_tiles;
+    L->last_launch[1] = (uint64_t)n_ctas;
+    L->last_launch[2] = launches;
+    return DTE_OK;
+}
+
+}  // namespace
+
+extern "C" dte_status dte_extract_delta(const dte_layout* layout, const float* const* theta,
+                                        const float* const* m, const float* const* v, int64_t step,
+                                        double lr, double beta1, double beta2, double eps, double wd,
+                                        const dte_delta* out, void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    if (layout->n_tensors && (!theta || !m || !v)) return fail(DTE_ERR_INVALID_ARG, "null pointer table");
+    dte_status s = check_delta(out);
+    if (s != DTE_OK) return s;
+    float c5[5];
+    s = dte_derive_constants(step, lr, beta1, beta2, eps, wd, c5);
+    if (s != DTE_OK) return s;
+    dte_layout* L = const_cast<dte_layout*>(layout);  // scratch and pointer-table cache
+    DeviceGuard g(L->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    s = sync_source_table(L, theta, m, v, st);
+    if (s != DTE_OK) return s;
+    const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
+    return enqueue_extract(L, c, out, st);
+}
+
+extern "C" dte_status dte_apply(const dte_layout* layout, const dte_delta* delta,
+                                uint16_t* const* shard_ptrs, void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    dte_status s = check_delta(delta);
+    if (s != DTE_OK) return s;
+    if (layout->n_lists && !shard_ptrs) return fail(DTE_ERR_INVALID_ARG, "shard pointer table is null");
+    dte_layout* L = const_cast<dte_layout*>(layout);
+    DeviceGuard g(L->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t n = L->n_lists;
+    if (n == 0) return DTE_OK;
+    std::vector<uint16_t*> tab(shard_ptrs, shard_ptrs + n);
+    for (size_t k = 0; k < n; ++k) {
+        if (!tab[k] && L->list_has_tiles[k] && L->shard_numel[k])
+            return fail(DTE_ERR_INVALID_ARG, "null shard pointer for a list that can hold entries");
+        if ((uintptr_t)tab[k] & 1u) return fail(DTE_ERR_INVALID_ARG, "shard pointers must be 2-byte aligned");
+    }
+    if (!(L->shards_valid && tab == L->h_shards)) {
+        L->shards_valid = false;
+        DTE_CUDA(cudaMemcpyAsync((void*)L->d_shards, tab.data(), n * sizeof(void*), cudaMemcpyHostToDevice, st));
+        L->h_shards.swap(tab);
+        L->shards_valid = true;
+    }
+    ApplyParams p;
+    p.offsets = delta->offsets;
+    p.values = delta->values;
+    p.capacity = delta->capacity;
+    p.list_ptr = delta->list_ptr;
+    p.counters = delta->counters;
+    p.shards = L->d_shards;
+    p.shard_numel = L->d_shard_numel;
+    p.n_lists = L->n_lists;
+    return launch_apply(p, L->device, st);
+}
+
+extern "C" dte_status dte_extract_delta_host(const dte_layout* layout, const float* const* theta_h,
+                                             const float* const* m_h, const float* const* v_h,
+                                             int64_t step, double lr, double beta1, double beta2,
+                                             double eps, double wd, void* workspace,
+                                             uint64_t workspace_bytes, const dte_delta* out,
+                                             uint32_t* offsets_h, uint16_t* values_h,
+                                             uint64_t* list_ptr_h, uint64_t* counters_h,
+                                             void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    if (layout->n_tensors && (!theta_h || !m_h || !v_h)) return fail(DTE_ERR_INVALID_ARG, "null pointer table");
+    if (!list_ptr_h || !counters_h) return fail(DTE_ERR_INVALID_ARG, "list_ptr_h / counters_h is null");
+    dte_status s = check_delta(out);
+    if (s != DTE_OK) return s;
+    float c5[5];
+    s = dte_derive_constants(step, lr, beta1, beta2, eps, wd, c5);
+    if (s != DTE_OK) return s;
+    dte_layout* L = const_cast<dte_layout*>(layout);
+    if (workspace_bytes < dte_layout_host_workspace_bytes(L)) return fail(DTE_ERR_CAPACITY, "workspace too small");
+    if (!workspace && workspace_bytes) return fail(DTE_ERR_INVALID_ARG, "workspace is null");
+    if ((uintptr_t)workspace & 255u) return fail(DTE_ERR_INVALID_ARG, "workspace must be 256-byte aligned");
+    DeviceGuard g(L->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t n = L->n_tensors;
+    std::vector<const float*> th(n, nullptr), mm(n, nullptr), vv(n, nullptr);
+    char* w = (char*)workspace;
+    for (size_t p = 0; p < n; ++p) {
+        if (!L->tensor_used[p]) continue;
+        if (!theta_h[p] || !m_h[p] || !v_h[p]) return fail(DTE_ERR_INVALID_ARG, "null host tensor pointer");
+        const size_t bytes = L->tensor_numel[p] * 4, pad = (bytes + 255) / 256 * 256;
+        const float* const src[3] = {theta_h[p], m_h[p], v_h[p]};
+        const float** dst[3] = {&th[p], &mm[p], &vv[p]};
+        for (int a = 0; a < 3; ++a) {
+            DTE_CUDA(cudaMemcpyAsync(w, src[a], bytes, cudaMemcpyHostToDevice, st));
+            *dst[a] = (const float*)w;
+            w += pad;
+        }
+    }
+    s = sync_source_table(L, th.data(), mm.data(), vv.data(), st);
+    if (s != DTE_OK) return s;
+    const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
+    s = enqueue_extract(L, c, out, st);
+    if (s != DTE_OK) return s;
+    DTE_CUDA(cudaMemcpyAsync(counters_h, out->counters, 4 * sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
+    DTE_CUDA(cudaMemcpyAsync(list_ptr_h, out->list_ptr, (L->n_lists + 1) * sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
+    DTE_CUDA(cudaStreamSynchronize(st));
+    if (counters_h[2] & DTE_DEV_TIMEOUT) return fail(DTE_ERR_TIMEOUT, "a bounded wait in the extract kernel ran out");
+    const uint64_t total = counters_h[0];
+    if (total > out->capacity || (counters_h[2] & DTE_DEV_OVERFLOW))
+        return fail(DTE_ERR_CAPACITY, "delta buffers too small; counters[0] holds the required capacity");
+    if (total && offsets_h) DTE_CUDA(cudaMemcpyAsync(offsets_h, out->offsets, total * sizeof(uint32_t), cudaMemcpyDeviceToHost, st));
+    if (total && values_h) DTE_CUDA(cudaMemcpyAsync(values_h, out->values, total * sizeof(uint16_t), cudaMemcpyDeviceToHost, st));
+    DTE_CUDA(cudaStreamSynchronize(st));
+    return DTE_OK;
+}

@@ -1,0 +1,131 @@
+// Internal structures shared by the layout compiler and the kernels.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "dte.h"
+
+namespace dte {
+
+// ---- tiling ---------------------------------------------------------------
+// A tile is a run of <= kTile consecutive receiver-local slots of ONE list, i.e. a
+// contiguous piece of one operation's destination range.  Tiles are numbered in output
+// order (list by list, ascending offset), so the output position of a tile is the
+// exclusive prefix sum of the changed counts of all tiles before it.
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kItems = 4;                              // float4 loads per thread and array
+constexpr int kWarpSpan = 32 * 4 * kItems;             // elements one warp owns: 512
+constexpr int kTile = kWarps * kWarpSpan;              // 4096 elements
+constexpr uint32_t kNone = 0xFFFFFFFFu;
+
+constexpr uint32_t kLenMask = 0xFFFFu;
+constexpr uint32_t kFlagFirstOfList = 1u << 16;        // tile starts its list
+constexpr uint32_t kFlagLastTile = 1u << 17;           // last tile of the whole layout
+constexpr uint32_t kFlagScalar = 1u << 18;             // not 16-byte alignable: scalar loads
+constexpr uint32_t kFlagStrided = 1u << 19;            // crosses source rows (see SegRec)
+
+struct __align__(32) TileDesc {
+    uint64_t src_off;    // element offset in the source tensor of the tile's row start
+    uint32_t tensor;     // source tensor index
+    uint32_t dst_off;    // receiver-local offset of the tile's first element
+    uint32_t len_flags;  // low 16 bits: elements; high bits: kFlag*
+    uint32_t list;       // output list (= shard index)
+    uint32_t seg;        // SegRec index when strided
+    uint32_t col0;       // strided: column (within the operation's extent) of the first element
+};
+static_assert(sizeof(TileDesc) == 32, "TileDesc must be one 32-byte sector");
+
+// A strided operation reads `w` elements from each source row of stride `s`.
+// For a tile element with c = col0 + e:  row = c / w = umulhi(c, magic), col = c - row*w,
+// source element = src_off + row*s + col.  magic = ceil(2^32 / w), verified on the host
+// for every c a tile can produce.
+struct SegRec {
+    uint32_t w, s, magic, pad;
+};
+
+// ---- decoupled look-back state ---------------------------------------------
+// One 64-bit word per tile: top two bits = state, low 62 bits = count.
+constexpr uint64_t kStateShift = 62;
+constexpr uint64_t kStateInvalid = 0, kStateAggregate = 1, kStatePrefix = 2, kStateError = 3;
+constexpr uint64_t kValueMask = (1ull << kStateShift) - 1;
+
+struct Consts {
+    float bc1, bc2, decay, lr, eps;
+};
+
+struct ExtractParams {
+    const TileDesc* tiles;
+    const SegRec* segs;
+    const float* const* theta;   // device table, n_tensors
+    const float* const* m;
+    const float* const* v;
+    uint64_t* status;            // n_tiles look-back words (zeroed before launch)
+    unsigned int* ticket;        // zeroed before launch
+    uint32_t n_tiles;
+    uint32_t n_lists;
+    uint64_t scanned;
+    uint32_t* offsets;
+    uint16_t* values;
+    uint64_t capacity;
+    uint64_t* list_ptr;
+    uint64_t* counters;
+    Consts c;
+};
+
+struct ApplyParams {
+    const uint32_t* offsets;
+    const uint16_t* values;
+    uint64_t capacity;
+    const uint64_t* list_ptr;
+    uint64_t* counters;
+    uint16_t* const* shards;     // device table, n_lists
+    const uint64_t* shard_numel; // device table, n_lists
+    uint32_t n_lists;
+};
+
+void set_error(const std::string& msg);
+dte_status cuda_fail(cudaError_t e, const char* what);
+
+#define DTE_CUDA(call)                                             \
+    do {                                                           \
+        cudaError_t e__ = (call);                                  \
+        if (e__ != cudaSuccess) return dte::cuda_fail(e__, #call); \
+    } while (0)
+
+dte_status launch_extract(const ExtractParams& p, int n_ctas, cudaStream_t st);
+dte_status extract_max_ctas(int device, int* n_ctas);
+dte_status launch_fill_empty_lists(uint64_t* list_ptr, const uint32_t* next_with_tiles,
+                                   uint32_t n_lists, cudaStream_t st);
+dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
+
+}  // namespace dte
+
+struct dte_layout {
+    int device = 0;
+    uint32_t n_tensors = 0, n_lists = 0, n_tiles = 0, n_segs = 0;
+    uint64_t scanned = 0;
+    std::vector<uint64_t> tensor_numel;
+    std::vector<uint8_t> tensor_used;
+    std::vector<uint64_t> shard_numel;
+    std::vector<uint8_t> list_has_tiles;
+    bool has_tileless_lists = false;
+    int max_ctas = 0;
+    // device memory owned by the layout
+    dte::TileDesc* d_tiles = nullptr;
+    dte::SegRec* d_segs = nullptr;
+    uint64_t* d_status = nullptr;          // n_tiles words + 1 word holding the ticket
+    const float** d_ptrs = nullptr;        // 3 * n_tensors source pointers
+    uint16_t** d_shards = nullptr;         // n_lists
+    uint64_t* d_shard_numel = nullptr;     // n_lists
+    uint32_t* d_next_with_tiles = nullptr; // n_lists (+1)
+    // host mirrors of the pointer tables last uploaded
+    std::vector<const float*> h_ptrs;
+    std::vector<uint16_t*> h_shards;
+    bool ptrs_valid = false, shards_valid = false;
+    uint64_t last_launch[3] = {0, 0, 0};
+};

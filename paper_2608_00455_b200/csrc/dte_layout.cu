@@ -1,0 +1,294 @@
+// Host side: error plumbing, constant derivation, and the layout compiler that turns the
+// transfer plan (Section 4.2.2) into a destination-ordered tile table.
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+
+#include "dte_internal.cuh"
+
+namespace dte {
+
+static thread_local std::string g_last_error;
+
+void set_error(const std::string& msg) { g_last_error = msg; }
+
+dte_status cuda_fail(cudaError_t e, const char* what) {
+    set_error(std::string(what) + ": " + cudaGetErrorString(e));
+    return DTE_ERR_CUDA;
+}
+
+static dte_status fail(dte_status s, const std::string& msg) {
+    set_error(msg);
+    return s;
+}
+
+struct Piece {                 // one operation seen from its destination list
+    uint64_t dst_start, len;   // flat destination range
+    uint64_t src_start;        // element offset of (a_s0, a_s1) in the source tensor
+    uint64_t w, s, rows;       // strided view; contiguous pieces have rows == 1, w == len
+    uint32_t tensor;
+    size_t op;
+};
+
+}  // namespace dte
+
+using namespace dte;
+
+extern "C" const char* dte_status_string(dte_status s) {
+    switch (s) {
+        case DTE_OK: return "ok";
+        case DTE_ERR_INVALID_ARG: return "invalid argument";
+        case DTE_ERR_LAYOUT: return "inconsistent layout";
+        case DTE_ERR_CAPACITY: return "buffer too small";
+        case DTE_ERR_BOUNDS: return "index out of bounds";
+        case DTE_ERR_TIMEOUT: return "timed out";
+        case DTE_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+extern "C" const char* dte_last_error(void) { return g_last_error.c_str(); }
+
+extern "C" dte_status dte_derive_constants(int64_t step, double lr, double beta1, double beta2,
+                                           double eps, double wd, float* out5) {
+    if (!out5) return fail(DTE_ERR_INVALID_ARG, "out5 is null");
+    if (step < 1) return fail(DTE_ERR_INVALID_ARG, "step must be >= 1 (1-based optimizer step)");
+    if (!std::isfinite(lr) || !std::isfinite(beta1) || !std::isfinite(beta2) ||
+        !std::isfinite(eps) || !std::isfinite(wd))
+        return fail(DTE_ERR_INVALID_ARG, "non-finite hyper-parameter");
+    if (beta1 < 0.0 || beta1 >= 1.0 || beta2 < 0.0 || beta2 >= 1.0)
+        return fail(DTE_ERR_INVALID_ARG, "betas must lie in [0, 1)");
+    if (eps < 0.0) return fail(DTE_ERR_INVALID_ARG, "eps must be >= 0");
+    if (lr * wd >= 1.0) return fail(DTE_ERR_INVALID_ARG, "lr * wd must be < 1");
+    const double t = (double)step;
+    const float bc1 = (float)(1.0 - std::pow(beta1, t));
+    const float bc2 = (float)(1.0 - std::pow(beta2, t));
+    const float decay = (float)(1.0 - lr * wd);
+    if (!(bc1 > 0.f) || !(bc2 > 0.f) || !(decay > 0.f))
+        return fail(DTE_ERR_INVALID_ARG, "bias correction or decay factor rounds to <= 0");
+    out5[0] = bc1;
+    out5[1] = bc2;
+    out5[2] = decay;
+    out5[3] = (float)lr;
+    out5[4] = (float)eps;
+    return DTE_OK;
+}
+
+extern "C" void dte_layout_destroy(dte_layout* L) {
+    if (!L) return;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    cudaSetDevice(L->device);
+    cudaFree(L->d_tiles);
+    cudaFree(L->d_segs);
+    cudaFree(L->d_status);
+    cudaFree((void*)L->d_ptrs);
+    cudaFree((void*)L->d_shards);
+    cudaFree(L->d_shard_numel);
+    cudaFree(L->d_next_with_tiles);
+    if (prev >= 0) cudaSetDevice(prev);
+    delete L;
+}
+
+extern "C" size_t dte_layout_num_lists(const dte_layout* L) { return L ? L->n_lists : 0; }
+extern "C" uint64_t dte_layout_num_elements(const dte_layout* L) { return L ? L->scanned : 0; }
+
+extern "C" uint64_t dte_layout_host_workspace_bytes(const dte_layout* L) {
+    if (!L) return 0;
+    uint64_t b = 0;
+    for (size_t p = 0; p < L->tensor_numel.size(); ++p)
+        if (L->tensor_used[p]) b += 3 * ((L->tensor_numel[p] * 4 + 255) / 256 * 256);
+    return b;
+}
+
+extern "C" void dte_layout_last_launch(const dte_layout* L, uint64_t* out3) {
+    for (int i = 0; i < 3; ++i) out3[i] = L ? L->last_launch[i] : 0;
+}
+
+template <class T>
+static dte_status upload(T** dst, const std::vector<T>& src, size_t min_elems = 1) {
+    size_t n = std::max(src.size(), min_elems);
+    DTE_CUDA(cudaMalloc((void**)dst, n * sizeof(T)));
+    if (!src.empty())
+        DTE_CUDA(cudaMemcpy(*dst, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice));
+    return DTE_OK;
+}
+
+extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n_tensors,
+                                        const dte_shard_desc* shards, size_t n_shards,
+                                        const dte_op_desc* ops, size_t n_ops, int device,
+                                        dte_layout** out) {
+    if (!out) return fail(DTE_ERR_INVALID_ARG, "out is null");
+    *out = nullptr;
+    if ((n_tensors && !tensors) || (n_shards && !shards) || (n_ops && !ops))
+        return fail(DTE_ERR_INVALID_ARG, "null descriptor array");
+    if (n_tensors >= kNone || n_shards >= kNone)
+        return fail(DTE_ERR_LAYOUT, "too many tensors or shards");
+
+    std::vector<uint64_t> numel(n_tensors);
+    for (size_t p = 0; p < n_tensors; ++p) {
+        const dte_tensor_desc& t = tensors[p];
+        if (t.ndim != 1 && t.ndim != 2) return fail(DTE_ERR_INVALID_ARG, "tensor ndim must be 1 or 2");
+        if (t.ndim == 1 && t.shape[1] != 1) return fail(DTE_ERR_INVALID_ARG, "1-D tensor needs shape[1] == 1");
+        if (t.group != 0) return fail(DTE_ERR_INVALID_ARG, "parameter groups are reserved: group must be 0");
+        if (t.shape[1] != 0 && t.shape[0] > (uint64_t(1) << 62) / t.shape[1])
+            return fail(DTE_ERR_LAYOUT, "tensor too large");
+        numel[p] = t.shape[0] * t.shape[1];
+    }
+    for (size_t k = 0; k < n_shards; ++k)
+        if (shards[k].numel >= (uint64_t(1) << 32))
+            return fail(DTE_ERR_LAYOUT, "shard numel must be < 2^32 (offsets are uint32)");
+
+    // --- operations -> destination pieces, grouped by list -------------------
+    std::vector<std::vector<Piece>> by_list(n_shards);
+    std::vector<uint8_t> used(n_tensors, 0);
+    for (size_t o = 0; o < n_ops; ++o) {
+        const dte_op_desc& op = ops[o];
+        const std::string tag = "operation " + std::to_string(o) + ": ";
+        if (op.src_tensor >= n_tensors || op.dst_shard >= n_shards)
+            return fail(DTE_ERR_LAYOUT, tag + "unknown tensor or shard");
+        const uint64_t n0 = tensors[op.src_tensor].shape[0], n1 = tensors[op.src_tensor].shape[1];
+        const uint64_t e0 = op.extent[0], e1 = op.extent[1];
+        if (e0 == 0 || e1 == 0) continue;  // empty overlap: legal, contributes nothing
+        if (op.src_origin[0] > n0 || e0 > n0 - op.src_origin[0] || op.src_origin[1] > n1 ||
+            e1 > n1 - op.src_origin[1])
+            return fail(DTE_ERR_LAYOUT, tag + "overlap leaves the source tensor");
+        const bool whole_rows = (op.dst_origin[1] == 0 && e1 == op.dst_ld);
+        const bool one_row = (e0 == 1 && op.dst_origin[1] <= op.dst_ld && e1 <= op.dst_ld - op.dst_origin[1]);
+        if (!whole_rows && !one_row)
+            return fail(DTE_ERR_LAYOUT, tag + "destination region is not a contiguous flat range");
+        const uint64_t numel_q = shards[op.dst_shard].numel;
+        // all terms < 2^32 after these checks, so the products below cannot overflow
+        if (op.dst_base > numel_q || op.dst_ld > numel_q + 1 || op.dst_origin[0] > numel_q)
+            return fail(DTE_ERR_LAYOUT, tag + "destination region leaves the shard");
+        Piece pc;
+        pc.dst_start = op.dst_base + op.dst_origin[0] * op.dst_ld + op.dst_origin[1];
+        pc.len = e0 * e1;
+        if (pc.dst_start > numel_q || pc.len > numel_q - pc.dst_start)
+            return fail(DTE_ERR_LAYOUT, tag + "destination region leaves the shard");
+        pc.src_start = op.src_origin[0] * n1 + op.src_origin[1];
+        pc.tensor = op.src_tensor;
+        pc.op = o;
+        if (e1 == n1 || e0 == 1) {          // source run is contiguous too
+            pc.w = pc.len; pc.s = pc.len; pc.rows = 1;
+        } else {
+            if (n1 >= (uint64_t(1) << 32)) return fail(DTE_ERR_LAYOUT, tag + "strided source row too long");
+            pc.w = e1; pc.s = n1; pc.rows = e0;
+        }
+        used[op.src_tensor] = 1;
+        by_list[op.dst_shard].push_back(pc);
+    }
+
+    std::vector<TileDesc> tiles;
+    std::vector<SegRec> segs;
+    std::vector<uint8_t> has_tiles(n_shards, 0);
+    uint64_t scanned = 0;
+    for (size_t k = 0; k < n_shards; ++k) {
+        auto& P = by_list[k];
+        std::sort(P.begin(), P.end(), [](const Piece& a, const Piece& b) { return a.dst_start < b.dst_start; });
+        for (size_t i = 1; i < P.size(); ++i)
+            if (P[i].dst_start < P[i - 1].dst_start + P[i - 1].len)
+                return fail(DTE_ERR_LAYOUT, "operations " + std::to_string(P[i - 1].op) + " and " +
+                                                std::to_string(P[i].op) + " overlap in shard " + std::to_string(k));
+        bool first = true;
+        for (const Piece& pc : P) {
+            scanned += pc.len;
+            auto push = [&](uint64_t src_off, uint64_t dst_off, uint64_t len, uint32_t flags,
+                            uint32_t seg, uint32_t col0) {
+                TileDesc t;
+                t.src_off = src_off;
+                t.tensor = pc.tensor;
+                t.dst_off = (uint32_t)dst_off;
+                t.len_flags = (uint32_t)len | flags | (first ? kFlagFirstOfList : 0u);
+                t.list = (uint32_t)k;
+                t.seg = seg;
+                t.col0 = col0;
+                tiles.push_back(t);
+                first = false;
+            };
+            if (pc.rows == 1) {
+                const bool vec = (pc.src_start % 4 == 0);
+                for (uint64_t s = 0; s < pc.len; s += kTile) {
+                    const uint64_t len = std::min<uint64_t>(kTile, pc.len - s);
+                    push(pc.src_start + s, pc.dst_start + s, len,
+                         (vec && len % 4 == 0) ? 0u : kFlagScalar, kNone, 0);
+                }
+            } else if (pc.w >= 4ull * kTile) {
+                // long rows: cut tiles at row ends, each tile is a contiguous source run
+                for (uint64_t r = 0; r < pc.rows; ++r)
+                    for (uint64_t c0 = 0; c0 < pc.w; c0 += kTile) {
+                        const uint64_t len = std::min<uint64_t>(kTile, pc.w - c0);
+                        const uint64_t so = pc.src_start + r * pc.s + c0;
+                        push(so, pc.dst_start + r * pc.w + c0, len,
+                             (so % 4 == 0 && len % 4 == 0) ? 0u : kFlagScalar, kNone, 0);
+                    }
+            } else {
+                SegRec sr;
+                sr.w = (uint32_t)pc.w;
+                sr.s = (uint32_t)pc.s;
+                sr.magic = pc.w >= 2 ? (uint32_t)(((uint64_t(1) << 32) + pc.w - 1) / pc.w) : 0u;
+                sr.pad = 0;
+                for (uint64_t c = 0; sr.w >= 2 && c < pc.w + kTile; ++c)
+                    if ((uint32_t)((c * sr.magic) >> 32) != (uint32_t)(c / pc.w))
+                        return fail(DTE_ERR_LAYOUT, "internal: row divisor check failed");
+                const uint32_t seg = (uint32_t)segs.size();
+                segs.push_back(sr);
+                const bool vec = (pc.w % 4 == 0 && pc.s % 4 == 0 && pc.src_start % 4 == 0);
+                const uint64_t n = pc.rows * pc.w;
+                for (uint64_t s = 0; s < n; s += kTile) {
+                    const uint64_t len = std::min<uint64_t>(kTile, n - s);
+                    const uint64_t row0 = s / pc.w, col0 = s % pc.w;
+                    push(pc.src_start + row0 * pc.s, pc.dst_start + s, len,
+                         kFlagStrided | ((vec && len % 4 == 0) ? 0u : kFlagScalar), seg, (uint32_t)col0);
+                }
+            }
+        }
+        has_tiles[k] = !first;
+    }
+    if (tiles.size() >= kNone) return fail(DTE_ERR_LAYOUT, "too many tiles");
+    if (!tiles.empty()) tiles.back().len_flags |= kFlagLastTile;
+
+    int prev = -1;
+    DTE_CUDA(cudaGetDevice(&prev));
+    DTE_CUDA(cudaSetDevice(device));
+    dte_layout* L = new dte_layout();
+    L->device = device;
+    L->n_tensors = (uint32_t)n_tensors;
+    L->n_lists = (uint32_t)n_shards;
+    L->n_tiles = (uint32_t)tiles.size();
+    L->n_segs = (uint32_t)segs.size();
+    L->scanned = scanned;
+    L->tensor_numel = numel;
+    L->tensor_used = used;
+    L->shard_numel.resize(n_shards);
+    for (size_t k = 0; k < n_shards; ++k) L->shard_numel[k] = shards[k].numel;
+    L->list_has_tiles = has_tiles;
+    // next_with_tiles[k] = smallest k' >= k whose list has tiles, or n_lists
+    std::vector<uint32_t> nxt(n_shards + 1, (uint32_t)n_shards);
+    for (size_t k = n_shards; k-- > 0;) {
+        nxt[k] = has_tiles[k] ? (uint32_t)k : nxt[k + 1];
+        if (!has_tiles[k]) L->has_tileless_lists = true;
+    }
+    dte_status st = DTE_OK;
+    auto guard = [&](dte_status s) { if (st == DTE_OK) st = s; };
+    guard(upload(&L->d_tiles, tiles));
+    guard(upload(&L->d_segs, segs));
+    guard(upload(&L->d_shard_numel, L->shard_numel));
+    guard(upload(&L->d_next_with_tiles, nxt));
+    if (st == DTE_OK) {
+        cudaError_t e = cudaMalloc((void**)&L->d_status, (tiles.size() + 1) * sizeof(uint64_t));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_ptrs, std::max<size_t>(1, 3 * n_tensors) * sizeof(void*));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_shards, std::max<size_t>(1, n_shards) * sizeof(void*));
+        if (e != cudaSuccess) st = cuda_fail(e, "cudaMalloc(layout scratch)");
+    }
+    if (st == DTE_OK) st = extract_max_ctas(device, &L->max_ctas);
+    if (prev >= 0) cudaSetDevice(prev);
+    if (st != DTE_OK) {
+        std::string keep = g_last_error;
+        dte_layout_destroy(L);
+        set_error(keep);
+        return st;
+    }
+    *out = L;
+    return DTE_OK;
+}

@@ -1,0 +1,60 @@
+"""The C-ABI library loads without a GPU and exports every symbol include/dte.h declares;
+host-only entry points behave as documented."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import paper_2608_00455_b200 as dte
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_symbols():
+    text = open(os.path.join(ROOT, "include", "dte.h")).read()
+    return sorted(set(re.findall(r"DTE_API[^;(]*?\b(dte_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared_symbols()
+    assert len(names) >= 12
+    assert sorted(names) == sorted(dte.SYMBOLS)
+    L = ctypes.CDLL(dte.library_path()) if os.path.exists(dte.library_path()) else dte.lib()
+    for n in names:
+        assert hasattr(L, n), n
+
+
+@pytest.mark.parametrize("args", [(1, 1e-6, 0.9, 0.999, 1e-8, 0.01), (100, 1e-6, 0.9, 0.999, 1e-8, 0.01),
+                                  (500, 1e-4, 0.9, 0.999, 1e-8, 0.1), (7, 3e-3, 0.5, 0.5, 0.0, 0.0),
+                                  (165, 1e-5, 0.95, 0.98, 1e-6, 0.05)])
+def test_constants_bit_identical_to_oracle(args):
+    a = dte.dte_derive_constants(*args)
+    b = oracle.derive_constants(*args)
+    assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+@pytest.mark.parametrize("args", [(0, 1e-6, 0.9, 0.999, 1e-8, 0.01), (1, 1e-6, 1.0, 0.999, 1e-8, 0.01),
+                                  (1, 1e-6, 0.9, -0.1, 1e-8, 0.01), (1, 2.0, 0.9, 0.999, 1e-8, 0.5),
+                                  (1, 1e-6, 0.9, 0.999, -1e-8, 0.01), (1, float("nan"), 0.9, 0.999, 1e-8, 0.01),
+                                  (1, 1e-6, 0.0, 0.999, 1e-8, 0.01 * 0 + float("inf"))])
+def test_bad_hyper_parameters_are_rejected(args):
+    with pytest.raises(dte.DteError) as e:
+        dte.dte_derive_constants(*args)
+    assert e.value.status == 1
+
+
+def test_status_strings():
+    L = dte.lib()
+    assert L.dte_status_string(0) == b"ok"
+    assert L.dte_status_string(2) == b"inconsistent layout"
+
+
+def test_compute_calls_fail_loudly_without_a_gpu():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("GPU present")
+    with pytest.raises(RuntimeError):
+        dte.Layout([(4, 4)], [16], [(0, 0, 0, 0, 4, 4, 0, 4, 0, 0)])

@@ -1,0 +1,227 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the same
+seeded inputs - bit-exact in the changed set, offsets, values, order and applied shards."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2608_00455_b200 as dte
+from synth import configs, plans
+from synth.tensors import Hyper, Spec
+from gpu_util import (assert_lists_equal, expected_shards, initial_shards, oracle_extract,
+                      run_extract)
+
+pytestmark = pytest.mark.gpu
+
+
+def _apply_and_check(plan, st, lay, d, got, want):
+    """Apply on the GPU and with the oracle from the same start; compare every shard."""
+    start = initial_shards(plan, st)
+    bufs = [s.clone() for s in start]
+    dte.dte_apply(lay, d, lay.shard_table(bufs))
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    host = [s.cpu().numpy().view(np.uint16).copy() for s in start]
+    oracle.apply(plan.shard_numels, *want, host)
+    for k in range(plan.n_shards):
+        assert np.array_equal(bufs[k].cpu().numpy().view(np.uint16), host[k]), plan.shard_names[k]
+    # idempotent (Eq. 4 sends target values)
+    again = [b.clone() for b in bufs]
+    dte.dte_apply(lay, d, lay.shard_table(again))
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(again, bufs))
+    return bufs
+
+
+def _full_parity(wl, capacity=None):
+    st = wl.materialize("cuda")
+    lay, d = run_extract(wl.plan, st, wl.hp, capacity)
+    assert d.status_bits() == 0
+    got = d.to_host()
+    want = oracle_extract(wl.plan, st, wl.hp)
+    assert_lists_equal(got, want, wl.plan)
+    cnt = d.counters.cpu().numpy()
+    assert cnt[0] == int(want[0][-1]) and cnt[1] == wl.plan.total_scanned_elements()
+    bufs = _apply_and_check(wl.plan, st, lay, d, got, want)
+    return st, lay, d, got, bufs
+
+
+def test_config1_single_matrix_tp2():
+    wl = configs.config1()
+    st, lay, d, got, bufs = _full_parity(wl)
+    total = int(got[0][-1])
+    assert 0.001 < total / 16777216 < 0.02
+    # mirror-association generator: the reconstruction recovers theta_{t-1} almost always,
+    # so the receivers end up equal to BF16(theta_t) except for a handful of elements
+    want = expected_shards(wl.plan, st)
+    stale = sum(int((a != b).sum().item()) for a, b in zip(bufs, want))
+    assert stale <= 8
+
+
+@pytest.mark.parametrize("name", ["dense_tp4", "dense_tp2", "moe", "matrix_tp3_ragged"])
+def test_small_plans_with_ragged_widths(name):
+    plan = {
+        "dense_tp4": lambda: plans.qwen3_dense_plan(2, 4, True, configs.SMALL_DENSE),
+        "dense_tp2": lambda: plans.qwen3_dense_plan(3, 2, True, configs.SMALL_DENSE),
+        "moe": lambda: plans.qwen3_moe_plan(2, 4, 4, configs.SMALL_MOE),
+        # 4099 x 1027: nothing is a multiple of 4 -> scalar tiles, ragged tails
+        "matrix_tp3_ragged": lambda: plans.single_matrix_plan(3 * 1367, 1027, 3),
+    }[name]()
+    wl = configs.Workload(name, plan, Hyper(step=100, lr=1e-5, wd=0.01), configs._specs(plan), 21)
+    _full_parity(wl)
+
+
+def test_config2_full_layer_tp4():
+    wl = configs.config2()
+    st, lay, d, got, bufs = _full_parity(wl, capacity=8_000_000)
+    assert lay.num_lists == 32
+
+
+@pytest.mark.parametrize("point", [(1e-8, 1, 0.1), (1e-6, 100, 0.01), (1e-4, 1, 0.1), (1e-4, 100, 0.01)])
+def test_config5_edge_sweep_reduced_dims(point):
+    lr, step, wd = point
+    wl = configs.config5(lr, step, wd, 1e-3, dims=configs.SMALL_DENSE)
+    _full_parity(wl)
+
+
+def test_config5_nonfinite_robustness():
+    wl = configs.config5(1e-4, 1, 0.1, 1e-2, dims=configs.SMALL_DENSE, nonfinite=True)
+    _full_parity(wl)
+
+
+def test_row_parallel_non_multiple_of_four_and_single_rows():
+    # column splits whose widths are odd, a one-row operation, and an uncovered gap
+    p = plans.Plan()
+    a = p.add_tensor("a", (37, 1001))
+    b = p.add_tensor("b", (5000,))
+    k0 = p.add_shard("a.cols", 0, 37 * 333)
+    p.add_op(a, k0, (0, 5), (37, 333), 0, 333, (0, 0))
+    k1 = p.add_shard("mixed", 1, 9000)
+    p.add_op(b, k1, (100, 0), (3000, 1), 0, 1, (10, 0))       # 1-D slice lands at offset 10
+    p.add_op(a, k1, (3, 7), (1, 900), 4000, 2000, (0, 50))    # one row, inside a wider row
+    k2 = p.add_shard("empty", 2, 0)
+    k3 = p.add_shard("untouched", 3, 64)
+    k4 = p.add_shard("a.tail", 0, 36 * 1001)
+    p.add_op(a, k4, (1, 0), (36, 1001), 0, 1001, (0, 0))
+    wl = configs.Workload("odd", p, Hyper(step=3, lr=3e-4, wd=0.1), [Spec(), Spec()], 5)
+    st, lay, d, got, bufs = _full_parity(wl)
+    lp = got[0]
+    assert lp[2] == lp[3] == lp[4]          # empty and untouched lists keep their slot
+
+
+def test_all_changed_and_none_changed():
+    plan = plans.qwen3_dense_plan(1, 4, False, configs.SMALL_DENSE)
+    # beta = 0.5, t = 1, m = v = 0.5, eps = 0: u = 1 exactly; lr = 8 moves every element far
+    # enough to change its BF16 pattern -> the lists enumerate every receiver slot
+    hp = Hyper(step=1, lr=8.0, beta1=0.5, beta2=0.5, eps=0.0, wd=0.0)
+    wl = configs.Workload("all", plan, hp, configs._specs(plan), 3)
+    st = wl.materialize("cuda")
+    st.m = [torch.full_like(x, 0.5) for x in st.m]
+    st.v = [torch.full_like(x, 0.5) for x in st.v]
+    lay, d = run_extract(plan, st, hp)
+    got = d.to_host()
+    assert int(got[0][-1]) == plan.total_scanned_elements() and d.status_bits() == 0
+    assert_lists_equal(got, oracle_extract(plan, st, hp), plan)
+    for k, n in enumerate(plan.shard_numels):
+        assert np.array_equal(got[1][int(got[0][k]):int(got[0][k + 1])], np.arange(n, dtype=np.uint32))
+    # zero moments (eps > 0): nothing changes
+    hp0 = Hyper(step=100, lr=1e-3, wd=0.0)
+    st.m = [torch.zeros_like(x) for x in st.m]
+    st.v = [torch.zeros_like(x) for x in st.v]
+    lay, d = run_extract(plan, st, hp0)
+    lp, off, val = d.to_host()
+    assert int(lp[-1]) == 0 and np.all(lp == 0) and d.status_bits() == 0
+    assert int(oracle_extract(plan, st, hp0)[0][-1]) == 0
+
+
+def test_capacity_overflow_reports_exact_sizes_and_apply_refuses():
+    wl = configs.config2(dims=configs.SMALL_DENSE, hp=Hyper(step=100, lr=1e-4, wd=0.01))
+    st = wl.materialize("cuda")
+    want = oracle_extract(wl.plan, st, wl.hp)
+    total = int(want[0][-1])
+    cap = total // 3
+    lay, d = run_extract(wl.plan, st, wl.hp, capacity=cap)
+    canary = torch.full((16,), 0x5A5A, dtype=torch.int32, device="cuda")
+    assert d.status_bits() & dte.DTE_DEV_OVERFLOW
+    assert d.total() == total
+    assert np.array_equal(d.list_ptr.cpu().numpy().astype(np.uint64), want[0])
+    # the part that fits is the prefix of the right answer
+    assert np.array_equal(d.offsets[:cap].cpu().numpy().view(np.uint32), want[1][:cap])
+    assert np.array_equal(d.values[:cap].cpu().numpy().view(np.uint16), want[2][:cap])
+    bufs = initial_shards(wl.plan, st)
+    before = [b.clone() for b in bufs]
+    dte.dte_apply(lay, d, lay.shard_table(bufs))
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(bufs, before))
+    # growing the buffers and calling again succeeds
+    lay, d = run_extract(wl.plan, st, wl.hp, capacity=total, layout=lay)
+    assert d.status_bits() == 0
+    assert_lists_equal(d.to_host(), want, wl.plan)
+    assert int(canary.sum().item()) == 16 * 0x5A5A
+
+
+def test_apply_flags_out_of_range_offsets():
+    plan = plans.single_matrix_plan(64, 64, 2)
+    wl = configs.Workload("b", plan, Hyper(step=1, lr=0.5, wd=0.0), configs._specs(plan, Spec(sigma_g=1.0)), 3)
+    st = wl.materialize("cuda")
+    lay, d = run_extract(plan, st, wl.hp)
+    d.offsets[5] = 2048          # == numel of shard 0: out of range
+    bufs = [torch.zeros(n, dtype=torch.int16, device="cuda") for n in plan.shard_numels]
+    guard = torch.zeros(4096, dtype=torch.int16, device="cuda")
+    dte.dte_apply(lay, d, lay.shard_table(bufs))
+    torch.cuda.synchronize()
+    assert d.status_bits() & dte.DTE_DEV_BOUNDS
+    assert int(guard.abs().sum().item()) == 0
+
+
+def test_deterministic_bytes_over_repeated_calls():
+    wl = configs.config1(rows=2048, cols=4096)
+    st = wl.materialize("cuda")
+    lay, d = run_extract(wl.plan, st, wl.hp, capacity=1 << 20)
+    ref = [x.clone() for x in (d.offsets[:d.total()], d.values[:d.total()], d.list_ptr)]
+    for _ in range(10):
+        d.offsets.zero_()
+        d.values.zero_()
+        run_extract(wl.plan, st, wl.hp, layout=lay, delta=d)
+        assert torch.equal(d.offsets[:d.total()], ref[0])
+        assert torch.equal(d.values[:d.total()], ref[1])
+        assert torch.equal(d.list_ptr, ref[2])
+
+
+def test_host_buffer_variant_matches_device_variant():
+    wl = configs.config2(dims=configs.SMALL_DENSE, hp=Hyper(step=100, lr=1e-5, wd=0.01))
+    st = wl.materialize("cuda")
+    lay, d = run_extract(wl.plan, st, wl.hp)
+    want = d.to_host()
+    th, mm, vv = ([x.cpu().pin_memory() for x in a] for a in (st.theta, st.m, st.v))
+    ws = torch.empty(lay.host_workspace_bytes, dtype=torch.uint8, device="cuda")
+    d2 = lay.new_delta(lay.num_elements)
+    res = dte.HostResult(lay.num_lists, d2.capacity)
+    dte.dte_extract_delta_host(lay, th, mm, vv, *wl.hp.as_args(), ws, d2, res)
+    got = res.arrays()
+    assert_lists_equal(got, want, wl.plan)
+    assert int(res.counters[0]) == int(want[0][-1])
+    assert_lists_equal(got, oracle_extract(wl.plan, st, wl.hp), wl.plan)
+
+
+def test_layout_errors():
+    ok_ops = [(0, 0, 0, 0, 8, 8, 0, 8, 0, 0)]
+    for shapes, numels, ops in [
+        ([(8, 8)], [64], [(0, 0, 0, 0, 9, 8, 0, 8, 0, 0)]),             # leaves the source
+        ([(8, 8)], [63], ok_ops),                                         # leaves the shard
+        ([(8, 8)], [64], [(0, 0, 0, 0, 8, 4, 0, 8, 0, 0)]),             # partial rows: not contiguous
+        ([(8, 8)], [64], [(0, 0, 0, 0, 4, 8, 0, 8, 0, 0), (0, 0, 2, 0, 4, 8, 0, 8, 3, 0)]),  # overlap
+        ([(8, 8)], [64], [(1, 0, 0, 0, 8, 8, 0, 8, 0, 0)]),             # unknown tensor
+        ([(8, 8)], [1 << 32], ok_ops),                                    # offsets would not fit uint32
+    ]:
+        with pytest.raises(dte.DteError) as e:
+            dte.Layout(shapes, numels, ops)
+        assert e.value.status == 2
+    lay = dte.Layout([(8, 8)], [64], ok_ops)
+    t = torch.zeros(65, dtype=torch.float32, device="cuda")
+    with pytest.raises(dte.DteError):                                     # misaligned theta
+        dte.dte_extract_delta(lay, lay.source_tables([t[1:]], [t[1:]], [t[1:]]), 1, 1e-3, 0.9, 0.999, 1e-8, 0.0,
+                              lay.new_delta(64))
+    with pytest.raises(dte.DteError):                                     # step 0
+        dte.dte_extract_delta(lay, lay.source_tables([t[:64]], [t[:64]], [t[:64]]), 0, 1e-3, 0.9, 0.999, 1e-8, 0.0,
+                              lay.new_delta(64))
