@@ -25,6 +25,10 @@
  *     device can detect are reported as DTE_DEV_* bits in dte_delta.counters[2].
  *   - A layout may be used by one extract or apply call at a time (its scratch memory
  *     is per layout).  Different layouts are independent.
+ *   - Scratch: the layout owns its device tables, one 8-byte placement record per 8192
+ *     scanned elements, and a staging buffer of `capacity` (offset, value) pairs.  The
+ *     staging buffer is allocated by the first extract call and re-allocated (with a stream
+ *     synchronisation) only when a later call passes a larger capacity.
  *   - There is no CPU fallback: every entry point needs a CUDA device.
  */
 #ifndef DTE_H_
@@ -49,14 +53,14 @@ typedef enum dte_status {
     DTE_ERR_LAYOUT = 2,      /* the tensor / shard / operation tables are inconsistent    */
     DTE_ERR_CAPACITY = 3,    /* a caller-provided buffer is too small (host-detected)     */
     DTE_ERR_BOUNDS = 4,      /* reserved for host-side bound checks                       */
-    DTE_ERR_TIMEOUT = 5,     /* a bounded device-side wait ran out (host variant reports) */
+    DTE_ERR_TIMEOUT = 5,     /* reserved                                                  */
     DTE_ERR_CUDA = 6         /* a CUDA runtime call failed; see dte_last_error()          */
 } dte_status;
 
 /* Device-detected conditions, OR-ed into dte_delta.counters[2]. */
-#define DTE_DEV_OVERFLOW 1u /* more changed elements than `capacity`; extra ones dropped */
+#define DTE_DEV_OVERFLOW 1u /* more changed elements than `capacity`; lists not produced   */
 #define DTE_DEV_BOUNDS 2u   /* apply met an offset >= numel of its shard; entry skipped  */
-#define DTE_DEV_TIMEOUT 4u  /* a bounded wait inside the extract kernel ran out          */
+#define DTE_DEV_TIMEOUT 4u  /* reserved (no kernel of this library waits on another CTA)  */
 
 /* Source tensor p of the canonical training-side space: fp32, row-major.  ndim is 1 or 2;
  * for ndim == 1 shape[1] must be 1.  `group` (parameter group) is reserved: must be 0. */
@@ -102,9 +106,9 @@ typedef struct dte_layout dte_layout;
  *   offsets  : capacity x uint32        values : capacity x uint16
  *   list_ptr : (n_shards + 1) x uint64
  *   counters : 4 x uint64 = { total changed, elements scanned, DTE_DEV_* bits, 0 }
- * If the total exceeds `capacity`, entries at positions >= capacity are dropped,
- * DTE_DEV_OVERFLOW is set, and list_ptr / counters[0] still hold the exact sizes, so
- * the caller can grow the buffers and call again. */
+ * If the total exceeds `capacity`, DTE_DEV_OVERFLOW is set, offsets / values hold nothing
+ * usable, and list_ptr / counters[0] still hold the exact sizes, so the caller can grow
+ * the buffers and call again (the paper's "size discovery before data movement"). */
 typedef struct dte_delta {
     uint32_t* offsets;
     uint16_t* values;

@@ -38,6 +38,10 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".tmp{os.getpid()}"
     cmd = [nvcc, *NVCC_FLAGS, "-I", INCLUDE, "-I", CSRC, "-o", tmp, *sources()]
+    if os.environ.get("DTE_STATS"):      # development-only counters
+        cmd.insert(1, "-DDTE_STATS")
+    for extra in os.environ.get("DTE_NVCC_EXTRA", "").split():   # development-only experiments
+        cmd.insert(1, extra)
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
         print(" ".join(cmd))

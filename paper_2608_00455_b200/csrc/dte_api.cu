@@ -1,6 +1,8 @@
 // C entry points that enqueue the kernels: dte_extract_delta, dte_apply and the
 // host-buffer variant dte_extract_delta_host.
+#include <cmath>
 #include <cstring>
+#include <limits>
 
 #include "dte_internal.cuh"
 
@@ -51,6 +53,28 @@ dte_status sync_source_table(dte_layout* L, const float* const* theta, const flo
     return DTE_OK;
 }
 
+// Constants of the kernel's conservative screen, each rounded up and inflated by 2^-10:
+//   k1    >= lr * sqrt(bc2) / bc1        (bound on |lr*u| is |m| * k1 * rsqrt(v))
+//   k2    >= lr / (bc1 * eps)            (.. and |m| * k2; +inf when eps == 0)
+//   kappa >= (|1/decay - 1| + 2^-24) * (1 + 2^-7)
+float round_up(double x) {
+    if (!(x == x)) return std::numeric_limits<float>::infinity();
+    float f = (float)x;
+    if ((double)f < x) f = std::nextafter(f, std::numeric_limits<float>::infinity());
+    return f;
+}
+
+Screen make_screen(const Consts& c) {
+    const double infl = 1.0 + 1.0 / 1024.0;
+    const double lr = std::fabs((double)c.lr);
+    Screen s;
+    s.k1 = round_up(lr * std::sqrt((double)c.bc2) / (double)c.bc1 * infl);
+    s.k2 = c.eps > 0.f ? round_up(lr / ((double)c.bc1 * (double)c.eps) * infl)
+                       : std::numeric_limits<float>::infinity();
+    s.kappa = round_up((std::fabs(1.0 / (double)c.decay - 1.0) + std::ldexp(1.0, -24)) * (1.0 + 1.0 / 128.0) * infl);
+    return s;
+}
+
 dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out, cudaStream_t st) {
     uint64_t launches = 0;
     DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
@@ -59,33 +83,56 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
         L->last_launch[0] = 0; L->last_launch[1] = 0; L->last_launch[2] = 0;
         return DTE_OK;
     }
-    DTE_CUDA(cudaMemsetAsync(L->d_status, 0, ((size_t)L->n_tiles + 1) * sizeof(uint64_t), st));
+    // the staging buffer mirrors the caller's capacity; it is (re)allocated only when a call
+    // brings a larger capacity than any before it
+    if (out->capacity > L->stage_capacity) {
+        DTE_CUDA(cudaStreamSynchronize(st));
+        cudaFree(L->d_stage_offsets);
+        cudaFree(L->d_stage_values);
+        L->d_stage_offsets = nullptr;
+        L->d_stage_values = nullptr;
+        L->stage_capacity = 0;
+        DTE_CUDA(cudaMalloc((void**)&L->d_stage_offsets, out->capacity * sizeof(uint32_t)));
+        DTE_CUDA(cudaMalloc((void**)&L->d_stage_values, out->capacity * sizeof(uint16_t)));
+        L->stage_capacity = out->capacity;
+    }
+    const size_t n_rec = (size_t)L->n_tiles;
+    DTE_CUDA(cudaMemsetAsync(L->d_cursor, 0, sizeof(uint64_t), st));
     ExtractParams p;
     p.tiles = L->d_tiles;
     p.segs = L->d_segs;
     p.theta = L->d_ptrs;
     p.m = L->d_ptrs + L->n_tensors;
     p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
-    p.status = L->d_status;
-    p.ticket = reinterpret_cast<unsigned int*>(L->d_status + L->n_tiles);
+    p.cursor = reinterpret_cast<unsigned long long*>(L->d_cursor);
+    p.rec = L->d_rec;
+    p.stage_offsets = L->d_stage_offsets;
+    p.stage_values = L->d_stage_values;
+    p.stage_capacity = out->capacity;
     p.n_tiles = L->n_tiles;
-    p.n_lists = L->n_lists;
-    p.scanned = L->scanned;
-    p.offsets = out->offsets;
-    p.values = out->values;
-    p.capacity = out->capacity;
-    p.list_ptr = out->list_ptr;
-    p.counters = out->counters;
     p.c = c;
-    const int n_ctas = (int)std::min<uint64_t>(L->n_tiles, (uint64_t)L->max_ctas);
+    p.s = make_screen(c);
+    const int n_ctas = (int)L->n_tiles;   // one CTA per tile
     dte_status s = launch_extract(p, n_ctas, st);
     if (s != DTE_OK) return s;
-    ++launches;
-    if (L->has_tileless_lists) {
-        s = launch_fill_empty_lists(out->list_ptr, L->d_next_with_tiles, L->n_lists, st);
-        if (s != DTE_OK) return s;
-        ++launches;
-    }
+    GatherParams g;
+    g.rec = L->d_rec;
+    g.block_sum = L->d_block_sum;
+    g.n_rec = (uint32_t)n_rec;
+    g.n_blocks = (uint32_t)((n_rec + kRecsPerBlock - 1) / kRecsPerBlock);
+    g.list_first_rec = L->d_list_first_rec;
+    g.n_lists = L->n_lists;
+    g.scanned = L->scanned;
+    g.stage_offsets = L->d_stage_offsets;
+    g.stage_values = L->d_stage_values;
+    g.offsets = out->offsets;
+    g.values = out->values;
+    g.capacity = out->capacity;
+    g.list_ptr = out->list_ptr;
+    g.counters = out->counters;
+    s = launch_gather(g, st);
+    if (s != DTE_OK) return s;
+    launches = 4;
     L->last_launch[0] = L->n_tiles;
     L->last_launch[1] = (uint64_t)n_ctas;
     L->last_launch[2] = launches;
@@ -194,7 +241,6 @@ extern "C" dte_status dte_extract_delta_host(const dte_layout* layout, const flo
     DTE_CUDA(cudaMemcpyAsync(counters_h, out->counters, 4 * sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
     DTE_CUDA(cudaMemcpyAsync(list_ptr_h, out->list_ptr, (L->n_lists + 1) * sizeof(uint64_t), cudaMemcpyDeviceToHost, st));
     DTE_CUDA(cudaStreamSynchronize(st));
-    if (counters_h[2] & DTE_DEV_TIMEOUT) return fail(DTE_ERR_TIMEOUT, "a bounded wait in the extract kernel ran out");
     const uint64_t total = counters_h[0];
     if (total > out->capacity || (counters_h[2] & DTE_DEV_OVERFLOW))
         return fail(DTE_ERR_CAPACITY, "delta buffers too small; counters[0] holds the required capacity");

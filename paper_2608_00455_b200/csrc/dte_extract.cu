@@ -2,14 +2,38 @@
 // (Eq. 4), ordered stream compaction, and receiver-local remap (Eq. 5-6, evaluated
 // destination-major through the tile table) in a single pass over theta / m / v.
 //
+// Structure.  One CTA per tile, one warp per warp-tile, no block-wide barrier until the
+// very end.  A warp streams its warp-tile's theta / m / v through registers with 128-bit
+// loads and classifies each element with a cheap conservative screen ("the BF16 pattern
+// cannot have changed").  Elements the screen cannot clear (a few per cent) are queued in
+// shared memory in element order and then evaluated densely, 32 at a time, with the exact
+// IEEE arithmetic; the changed ones are compacted in place.  The CTA then reserves room
+// for all its entries in a staging buffer with ONE atomic add, the warps write their
+// (offset, value) pairs there with coalesced stores, in tile order, and the CTA records
+// (position, count) for its tile.  No CTA waits on another; the ordered placement happens
+// in the gather kernels (dte_gather.cu), which touch only the placement records and the
+// changed entries.
+//
 // Build flags that matter for bit-exactness: -fmad=false -ftz=false -prec-div=true
-// -prec-sqrt=true.  The arithmetic below additionally spells every operation as a
+// -prec-sqrt=true.  The exact path additionally spells every operation as a
 // round-to-nearest intrinsic so that no flag can silently change it.
 #include "dte_internal.cuh"
 
 namespace dte {
 
-// ---- arithmetic -----------------------------------------------------------------
+#ifndef DTE_MIN_CTAS
+#define DTE_MIN_CTAS 3
+#endif
+
+#ifdef DTE_STATS
+// Development-only counters (never compiled into the shipped library).
+__device__ unsigned long long g_stats[8];
+#define DTE_STAT(i, x) do { if (lane == 0) atomicAdd(&g_stats[i], (unsigned long long)(x)); } while (0)
+#else
+#define DTE_STAT(i, x) do { } while (0)
+#endif
+
+// ---- exact arithmetic ------------------------------------------------------------
 
 // Eq. 2, one fp32 operation at a time.  DIV_BC1 / DIV_DECAY are false when the divisor is
 // exactly 1.0f (x / 1 == x for every x, NaN included as far as the BF16 cast can tell).
@@ -30,242 +54,247 @@ __device__ __forceinline__ uint32_t bf16_rne_bits(float x) {
     return ((u & 0x7FFFFFFFu) > 0x7F800000u) ? 0x7FC0u : r;
 }
 
+// ---- the screen --------------------------------------------------------------------
+//
+// Let a = |theta|, c = the BF16 value nearest to a, and lo < a < hi the two rounding
+// boundaries (tie points) around c, as fp32 numbers.  With lo' = succ(lo), hi' = pred(hi):
+// any real x in [lo', hi'] rounds (in fp32, then in BF16) to c, because rounding is
+// monotone and lo', hi' are fp32 numbers strictly inside (lo, hi).  So if
+//     B >= |x - theta|  and  B <= min(hi' - a, a - lo')          (*)
+// where x is the exact quotient whose rounding is the reconstruction, the reconstruction
+// has the same BF16 pattern as theta: unchanged, no exact evaluation needed.
+//
+// B: every intermediate of Eq. 2 carries a relative rounding error <= 2^-24, so
+//     |lr*u| <= |m| * min( lr*sqrt(bc2)/bc1 * rsqrt(v),  lr/(bc1*eps) ) * (1 + 2^-20),
+// and dividing by decay moves the value by at most |num| * |1/decay - 1|, |num| <= a(1+2^-7).
+// The host passes k1, k2, kappa rounded up and inflated by 2^-10, which covers the fp32
+// evaluation of B itself and the 2^-22 error of the hardware rsqrt.  rsqrt flushes
+// subnormal v to zero, which only enlarges B.  NaN anywhere makes (*) false (min.NaN and an
+// ordered compare), so NaN / Inf / negative v / zero theta all fall through to the exact
+// path.  hi' - a and a - lo' are exact (the operands are within a factor 2 of each other).
+__device__ __forceinline__ float min_nan(float x, float y) {
+    float r;
+    asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(x), "f"(y));
+    return r;
+}
+__device__ __forceinline__ float rsqrt_ftz(float x) {
+    float r;
+    asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
+    return r;
+}
+
+template <bool DIV_DECAY>
+__device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s) {
+    const uint32_t a = __float_as_uint(theta) & 0x7FFFFFFFu;
+    const uint32_t hi = ((a + 0x8000u) & 0xFFFF0000u) | 0x7FFFu;
+    const uint32_t lo = hi - 0xFFFEu;
+    const float at = __uint_as_float(a);
+    const float room = min_nan(__uint_as_float(hi) - at, at - __uint_as_float(lo));
+    float b = fabsf(m) * min_nan(fabsf(rsqrt_ftz(v)) * s.k1, s.k2);
+    if (DIV_DECAY) b = __fmaf_rn(at, s.kappa, b);
+    return b <= room;
+}
+
 __device__ __forceinline__ const float* ldg_ptr(const float* const* slot) {
     return reinterpret_cast<const float*>(__ldg(reinterpret_cast<const unsigned long long*>(slot)));
 }
-
-// ---- look-back words ---------------------------------------------------------------
-
-__device__ __forceinline__ uint64_t ld_status(const uint64_t* p) {
-    uint64_t w;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(w) : "l"(p) : "memory");
-    return w;
-}
-__device__ __forceinline__ void st_status(uint64_t* p, uint64_t w) {
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(w) : "memory");
-}
-
-constexpr int kMaxPolls = 1 << 20;  // bounded wait: ~0.1-1 s of back-off before giving up
-
-// Exclusive prefix of tile `t`, computed by warp 0.  Returns false on error / timeout.
-// Tiles take their index from an atomic ticket, so every predecessor is owned by a CTA
-// that is already running (or done) and waits only on its own predecessors: progress
-// does not depend on how CTAs are scheduled.
-__device__ __forceinline__ bool look_back(uint64_t* status, uint32_t t, uint32_t aggregate,
-                                          int lane, uint64_t* excl_out) {
-    if (t == 0) {
-        if (lane == 0) st_status(status, (kStatePrefix << kStateShift) | aggregate);
-        *excl_out = 0;
-        return true;
-    }
-    if (lane == 0) st_status(status + t, (kStateAggregate << kStateShift) | aggregate);
-    uint64_t excl = 0;
-    int64_t pos = (int64_t)t - 1;
-    int polls = 0;
-    bool ok = true;
-    while (true) {
-        const int64_t idx = pos - lane;
-        uint64_t w = (idx >= 0) ? ld_status(status + idx) : (kStatePrefix << kStateShift);
-        const uint32_t state = (uint32_t)(w >> kStateShift);
-        const uint32_t m_prefix = __ballot_sync(0xFFFFFFFFu, state == kStatePrefix);
-        const uint32_t m_invalid = __ballot_sync(0xFFFFFFFFu, state == kStateInvalid);
-        const uint32_t m_error = __ballot_sync(0xFFFFFFFFu, state == kStateError);
-        const int first_prefix = m_prefix ? (__ffs(m_prefix) - 1) : 32;
-        const uint32_t needed = first_prefix < 32 ? (0xFFFFFFFFu >> (31 - first_prefix)) : 0xFFFFFFFFu;
-        if (m_error & needed) { ok = false; break; }
-        if (m_invalid & needed) {
-            if (++polls > kMaxPolls) { ok = false; break; }
-            __nanosleep(polls < 64 ? 32 : 256);
-            continue;
-        }
-        uint64_t val = ((needed >> lane) & 1u) ? (w & kValueMask) : 0ull;
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) val += __shfl_xor_sync(0xFFFFFFFFu, val, d);
-        excl += val;
-        if (first_prefix < 32) break;
-        pos -= 32;
-    }
-    if (lane == 0)
-        st_status(status + t, ok ? ((kStatePrefix << kStateShift) | (excl + aggregate))
-                                 : (kStateError << kStateShift));
-    *excl_out = excl;
-    return ok;
-}
-
 // ---- the kernel --------------------------------------------------------------------
 
-struct __align__(16) Smem {
-    uint32_t warp_total[kWarps];
-    uint64_t tile_excl;
-    uint32_t ticket;
-    uint32_t ok;
+// Decoded descriptor of one warp-tile.
+struct WarpTile {
+    const float* th;
+    const float* mm;
+    const float* vv;
+    uint64_t src_off;      // source element offset of the enclosing tile's row start
+    uint32_t w, s, magic;  // strided tiles: row width / stride / divisor (SegRec)
+    uint32_t col0;         // strided tiles: column of tile element 0, plus e0 folded in
+    uint32_t len;          // elements of this warp-tile (0 for the unused tail of a short tile)
+    uint32_t dst0;         // receiver-local offset of element 0 of this warp-tile
+    uint32_t len_flags;
+
+    // source element offset of warp-tile element e
+    __device__ __forceinline__ uint64_t src(uint32_t e) const {
+        if (!(len_flags & kFlagStrided)) return src_off + e;
+        const uint32_t cc = col0 + e;
+        const uint32_t row = (w == 1) ? cc : __umulhi(cc, magic);
+        return src_off + (uint64_t)row * s + (cc - row * w);
+    }
 };
 
-template <bool DIV_BC1, bool DIV_DECAY>
-__global__ void __launch_bounds__(kThreads, 4) extract_kernel(const ExtractParams p) {
-    __shared__ Smem sm;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const Consts c = p.c;
+__device__ __forceinline__ void decode(const ExtractParams& p, uint32_t t, WarpTile& wt) {
+    // all lanes read the same 32-byte descriptor (one sector, broadcast)
+    const uint4* td = reinterpret_cast<const uint4*>(p.tiles + (t / kSub));
+    const uint4 d0 = __ldg(td), d1 = __ldg(td + 1);
+    const uint32_t e0 = (t % kSub) * kWarpTile;
+    const uint32_t tile_len = d1.x & kLenMask;
+    wt.len_flags = d1.x;
+    wt.len = tile_len > e0 ? min(tile_len - e0, (uint32_t)kWarpTile) : 0u;
+    wt.dst0 = d0.w + e0;
+    wt.th = ldg_ptr(p.theta + d0.z);
+    wt.mm = ldg_ptr(p.m + d0.z);
+    wt.vv = ldg_ptr(p.v + d0.z);
+    wt.src_off = ((uint64_t)d0.x | ((uint64_t)d0.y << 32));
+    wt.w = 0; wt.s = 0; wt.magic = 0; wt.col0 = 0;
+    if (d1.x & kFlagStrided) {
+        const uint4 sr = __ldg(reinterpret_cast<const uint4*>(p.segs + d1.z));
+        wt.w = sr.x; wt.s = sr.y; wt.magic = sr.z;
+        wt.col0 = d1.w + e0;
+    } else {
+        wt.src_off += e0;
+    }
+}
 
-    while (true) {
-        if (tid == 0) sm.ticket = atomicAdd(p.ticket, 1u);
-        __syncthreads();
-        const uint32_t t = sm.ticket;
-        if (t >= p.n_tiles) break;
-
-        // all threads read the same 32-byte descriptor (one sector, broadcast)
-        const uint4* td = reinterpret_cast<const uint4*>(p.tiles + t);
-        const uint4 d0 = __ldg(td), d1 = __ldg(td + 1);
-        const uint64_t src_off = (uint64_t)d0.x | ((uint64_t)d0.y << 32);
-        const uint32_t tensor = d0.z, dst_off = d0.w, len_flags = d1.x, list = d1.y;
-        const uint32_t len = len_flags & kLenMask;
-        const float* __restrict__ th = ldg_ptr(p.theta + tensor);
-        const float* __restrict__ mm = ldg_ptr(p.m + tensor);
-        const float* __restrict__ vv = ldg_ptr(p.v + tensor);
-
-        uint32_t mask[kItems];   // bit j: element 4*lane + j of the item changed
-        uint32_t val[kItems][2]; // BF16(theta) of the item's 4 elements, packed 2 x 16
-        const uint32_t e_warp = warp * kWarpSpan;
-
-        if (!(len_flags & (kFlagScalar | kFlagStrided))) {
-            // ---- contiguous, 16-byte aligned: three 128-bit loads per item --------------
-            float4 a[kItems], b[kItems], g[kItems];
+// One chunk (kChunk elements from warp-tile element cb) of theta / m / v into registers.
+__device__ __forceinline__ void load_chunk(const WarpTile& wt, uint32_t cb, int lane,
+                                           float4 (&a)[kItems], float4 (&b)[kItems], float4 (&g)[kItems]) {
+    if (!(wt.len_flags & kFlagScalar)) {
 #pragma unroll
-            for (int i = 0; i < kItems; ++i) {
-                const uint32_t e = e_warp + i * 128 + lane * 4;
-                if (e < len) {
-                    a[i] = __ldcs(reinterpret_cast<const float4*>(th + src_off + e));
-                    b[i] = __ldcs(reinterpret_cast<const float4*>(mm + src_off + e));
-                    g[i] = __ldcs(reinterpret_cast<const float4*>(vv + src_off + e));
+        for (int i = 0; i < kItems; ++i) {
+            const uint32_t e = cb + i * 128 + lane * 4;
+            if (e < wt.len) {
+                const uint64_t so = wt.src(e);
+                a[i] = __ldg(reinterpret_cast<const float4*>(wt.th + so));
+                b[i] = __ldg(reinterpret_cast<const float4*>(wt.mm + so));
+                g[i] = __ldg(reinterpret_cast<const float4*>(wt.vv + so));
+            }
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < kItems; ++i) {
+            float ta[4], tb[4], tg[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t e = cb + i * 128 + lane * 4 + j;
+                ta[j] = tb[j] = tg[j] = 0.f;
+                if (e < wt.len) {
+                    const uint64_t so = wt.src(e);
+                    ta[j] = __ldg(wt.th + so); tb[j] = __ldg(wt.mm + so); tg[j] = __ldg(wt.vv + so);
                 }
             }
+            a[i] = make_float4(ta[0], ta[1], ta[2], ta[3]);
+            b[i] = make_float4(tb[0], tb[1], tb[2], tb[3]);
+            g[i] = make_float4(tg[0], tg[1], tg[2], tg[3]);
+        }
+    }
+}
+
+template <bool DIV_BC1, bool DIV_DECAY>
+__global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const ExtractParams p) {
+    // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
+    __shared__ uint32_t s_queue[kWarps][kWarpTile];
+    __shared__ uint32_t s_count[kWarps];
+    __shared__ unsigned long long s_pos;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* queue = s_queue[warp];
+    const Consts c = p.c;
+    const Screen sc = p.s;
+    const uint32_t lanemask_lt = (1u << lane) - 1u;
+    static_assert(kSub == kWarps, "one warp per warp-tile");
+
+    float4 a[kItems], b[kItems], g[kItems];
+    WarpTile cur;
+    {
+        const uint32_t t = blockIdx.x * kSub + warp;
+        decode(p, t, cur);
+
+        // ---- phase A: stream, screen, queue the undecided elements in element order ---------
+        uint32_t qn = 0;
+#pragma unroll 1
+        for (uint32_t cb = 0; cb < cur.len; cb += kChunk) {
+            load_chunk(cur, cb, lane, a, b, g);
+            uint32_t amb[kItems];
+            uint32_t cnt = 0;
 #pragma unroll
             for (int i = 0; i < kItems; ++i) {
-                const uint32_t e = e_warp + i * 128 + lane * 4;
-                mask[i] = 0; val[i][0] = 0; val[i][1] = 0;
-                if (e < len) {
+                const uint32_t e = cb + i * 128 + lane * 4;
+                amb[i] = 0;
+                if (e < cur.len) {
                     const float tt[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
                     const float m4[4] = {b[i].x, b[i].y, b[i].z, b[i].w};
                     const float v4[4] = {g[i].x, g[i].y, g[i].z, g[i].w};
 #pragma unroll
-                    for (int j = 0; j < 4; ++j) {
-                        const float prev = invert_adamw<DIV_BC1, DIV_DECAY>(tt[j], m4[j], v4[j], c);
-                        const uint32_t bt = bf16_rne_bits(tt[j]), bp = bf16_rne_bits(prev);
-                        mask[i] |= (bt != bp ? 1u : 0u) << j;
-                        val[i][j >> 1] |= bt << ((j & 1) * 16);
-                    }
+                    for (int j = 0; j < 4; ++j)
+                        if (!surely_unchanged<DIV_DECAY>(tt[j], m4[j], v4[j], sc)) amb[i] |= 1u << j;
+                    amb[i] &= (1u << min(cur.len - e, 4u)) - 1u;      // ragged tail of a scalar tile
                 }
+                cnt |= __popc(amb[i]) << (8 * i);
             }
-        } else {
-            // ---- generic path: scalar loads, optional row stride --------------------------
-            uint32_t w = 0, s = 0, magic = 0, col0 = 0;
-            const bool strided = len_flags & kFlagStrided;
-            if (strided) {
-                const uint4 sr = __ldg(reinterpret_cast<const uint4*>(p.segs + d1.z));
-                w = sr.x; s = sr.y; magic = sr.z; col0 = d1.w;
+            // ordered slots: warp scan of the per-item counts, packed 4 x 8 bits (each <= 128)
+            uint32_t incl = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= d) incl += up;
             }
+            const uint32_t excl = incl - cnt;
+            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            uint32_t run = qn;
 #pragma unroll
             for (int i = 0; i < kItems; ++i) {
-                mask[i] = 0; val[i][0] = 0; val[i][1] = 0;
-#pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t e = e_warp + i * 128 + lane * 4 + j;
-                    if (e < len) {
-                        uint64_t so = src_off + e;
-                        if (strided) {
-                            const uint32_t cc = col0 + e;
-                            const uint32_t row = (w == 1) ? cc : __umulhi(cc, magic);
-                            so = src_off + (uint64_t)row * s + (cc - row * w);
-                        }
-                        const float tj = __ldcs(th + so), mj = __ldcs(mm + so), vj = __ldcs(vv + so);
-                        const float prev = invert_adamw<DIV_BC1, DIV_DECAY>(tj, mj, vj, c);
-                        const uint32_t bt = bf16_rne_bits(tj), bp = bf16_rne_bits(prev);
-                        mask[i] |= (bt != bp ? 1u : 0u) << j;
-                        val[i][j >> 1] |= bt << ((j & 1) * 16);
-                    }
-                }
-            }
-        }
-
-        // ---- ordered ranks: warp scan of per-item counts packed 4 x 8 bits ------------------
-        uint32_t cnt = 0;
-#pragma unroll
-        for (int i = 0; i < kItems; ++i) cnt |= __popc(mask[i]) << (8 * i);
-        uint32_t incl = cnt;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-            if (lane >= d) incl += up;
-        }
-        const uint32_t excl = incl - cnt;                       // per item: changed in lanes below
-        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);  // per item: changed in this warp
-        uint32_t item_base[kItems];
-        uint32_t run = 0;
-#pragma unroll
-        for (int i = 0; i < kItems; ++i) {
-            item_base[i] = run + ((excl >> (8 * i)) & 0xFFu);
-            run += (tot >> (8 * i)) & 0xFFu;
-        }
-        if (lane == 0) sm.warp_total[warp] = run;
-        __syncthreads();
-
-        uint32_t warp_base = 0, tile_total = 0;
-#pragma unroll
-        for (int w2 = 0; w2 < kWarps; ++w2) {
-            const uint32_t x = sm.warp_total[w2];
-            if (w2 < warp) warp_base += x;
-            tile_total += x;
-        }
-        if (warp == 0) {
-            uint64_t ex;
-            const bool ok = look_back(p.status, t, tile_total, lane, &ex);
-            if (lane == 0) { sm.tile_excl = ex; sm.ok = ok ? 1u : 0u; }
-        }
-        __syncthreads();
-        const uint64_t tile_excl = sm.tile_excl;
-        const bool ok = sm.ok != 0;
-        if (!ok) {
-            if (tid == 0) atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_TIMEOUT);
-        } else {
-            // ---- ordered writes --------------------------------------------------------
-            bool dropped = false;
-#pragma unroll
-            for (int i = 0; i < kItems; ++i) {
-                uint32_t mk = mask[i];
-                uint64_t pos = tile_excl + warp_base + item_base[i];
+                uint32_t pos = run + ((excl >> (8 * i)) & 0xFFu);
+                uint32_t mk = amb[i];
                 while (mk) {
                     const int j = __ffs(mk) - 1;
                     mk &= mk - 1;
-                    if (pos < p.capacity) {
-                        p.offsets[pos] = dst_off + e_warp + i * 128 + lane * 4 + j;
-                        p.values[pos] = (uint16_t)(val[i][j >> 1] >> ((j & 1) * 16));
-                    } else {
-                        dropped = true;
-                    }
-                    ++pos;
+                    queue[pos++] = cb + i * 128 + lane * 4 + j;
                 }
+                run += (tot >> (8 * i)) & 0xFFu;
             }
-            if (dropped) atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_OVERFLOW);
-            if (tid == 0) {
-                if (len_flags & kFlagFirstOfList) p.list_ptr[list] = tile_excl;
-                if (len_flags & kFlagLastTile) {
-                    p.list_ptr[p.n_lists] = tile_excl + tile_total;
-                    p.counters[0] = tile_excl + tile_total;
-                    p.counters[1] = p.scanned;
-                }
+            qn = run;
+        }
+        __syncwarp();
+        DTE_STAT(0, qn);
+        DTE_STAT(2, (qn + 31) / 32);
+
+        // ---- phase B: exact evaluation of the queue, 32 entries per round; the changed
+        //      entries are compacted to the front of the queue as (index | value << 16) -----
+        uint32_t n_changed = 0;
+#pragma unroll 1
+        for (uint32_t q0 = 0; q0 < qn; q0 += 32) {
+            const uint32_t q = q0 + lane;
+            bool changed = false;
+            uint32_t entry = 0;
+            if (q < qn) {
+                const uint32_t e = queue[q];
+                const uint64_t so = cur.src(e);
+                const float tj = __ldg(cur.th + so), mj = __ldg(cur.mm + so), vj = __ldg(cur.vv + so);
+                const float prev = invert_adamw<DIV_BC1, DIV_DECAY>(tj, mj, vj, c);
+                const uint32_t bt = bf16_rne_bits(tj), bp = bf16_rne_bits(prev);
+                changed = bt != bp;
+                entry = e | (bt << 16);
+            }
+            const uint32_t msk = __ballot_sync(0xFFFFFFFFu, changed);  // also orders reads before writes
+            if (changed) queue[n_changed + __popc(msk & lanemask_lt)] = entry;
+            n_changed += __popc(msk);
+        }
+        __syncwarp();
+
+        // ---- phase C: one reservation per CTA, coalesced writes in tile order, the record -----
+        if (lane == 0) s_count[warp] = n_changed;
+        __syncthreads();
+        uint32_t before = 0, total = 0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) {
+            const uint32_t x = s_count[w];
+            if (w < warp) before += x;
+            total += x;
+        }
+        if (threadIdx.x == 0) {
+            unsigned long long pos0 = 0;
+            if (total) pos0 = atomicAdd(p.cursor, (unsigned long long)total);
+            s_pos = pos0;
+            p.rec[blockIdx.x] = ((uint64_t)pos0 << kRecCountBits) | total;
+        }
+        __syncthreads();
+        const unsigned long long pos = s_pos + before;
+        const uint32_t dst0 = cur.dst0;
+        for (uint32_t q = lane; q < n_changed; q += 32) {
+            const uint32_t entry = queue[q];
+            if (pos + q < p.stage_capacity) {         // beyond it the call overflows anyway
+                p.stage_offsets[pos + q] = dst0 + (entry & 0xFFFFu);
+                p.stage_values[pos + q] = (uint16_t)(entry >> 16);
             }
         }
-        // sm.ticket / sm.tile_excl are rewritten only after the next __syncthreads pair
-    }
-}
-
-// Lists without any tile (empty shard, or no operation targets it) start where the next
-// list with tiles starts.  Only launched for layouts that have such lists.
-__global__ void fill_empty_lists_kernel(uint64_t* list_ptr, const uint32_t* next_with_tiles,
-                                        uint32_t n_lists) {
-    for (uint32_t k = blockIdx.x * blockDim.x + threadIdx.x; k < n_lists; k += gridDim.x * blockDim.x) {
-        const uint32_t nx = next_with_tiles[k];
-        if (nx != k) list_ptr[k] = list_ptr[nx];
     }
 }
 
@@ -275,6 +304,13 @@ static dte_status launch_t(const ExtractParams& p, int n_ctas, cudaStream_t st) 
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }
+
+#ifdef DTE_STATS
+extern "C" __attribute__((visibility("default"))) void dte_debug_stats(unsigned long long* out8, int reset) {
+    cudaMemcpyFromSymbol(out8, g_stats, sizeof(g_stats));
+    if (reset) { unsigned long long z[8] = {0}; cudaMemcpyToSymbol(g_stats, z, sizeof(z)); }
+}
+#endif
 
 dte_status launch_extract(const ExtractParams& p, int n_ctas, cudaStream_t st) {
     const bool a = p.c.bc1 != 1.0f, b = p.c.decay != 1.0f;
@@ -289,14 +325,7 @@ dte_status extract_max_ctas(int device, int* n_ctas) {
     DTE_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
     DTE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, extract_kernel<true, true>, kThreads, 0));
     if (per_sm < 1) per_sm = 1;
-    *n_ctas = sms * per_sm;
-    return DTE_OK;
-}
-
-dte_status launch_fill_empty_lists(uint64_t* list_ptr, const uint32_t* next_with_tiles,
-                                   uint32_t n_lists, cudaStream_t st) {
-    fill_empty_lists_kernel<<<1, 256, 0, st>>>(list_ptr, next_with_tiles, n_lists);
-    DTE_CUDA(cudaGetLastError());
+    *n_ctas = sms * per_sm;   // resident CTAs (informational: the grid is one CTA per tile)
     return DTE_OK;
 }
 

@@ -14,13 +14,17 @@ namespace dte {
 // ---- tiling ---------------------------------------------------------------
 // A tile is a run of <= kTile consecutive receiver-local slots of ONE list, i.e. a
 // contiguous piece of one operation's destination range.  Tiles are numbered in output
-// order (list by list, ascending offset), so the output position of a tile is the
-// exclusive prefix sum of the changed counts of all tiles before it.
+// order (list by list, ascending offset).  Each tile is cut into kSub warp-tiles of
+// kWarpTile slots; one warp processes one warp-tile at a time, and the output position of
+// a warp-tile is the exclusive prefix sum of the changed counts of all warp-tiles before it.
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
-constexpr int kItems = 4;                              // float4 loads per thread and array
-constexpr int kWarpSpan = 32 * 4 * kItems;             // elements one warp owns: 512
-constexpr int kTile = kWarps * kWarpSpan;              // 4096 elements
+constexpr int kItems = 4;                              // float4 loads per thread, array and chunk
+constexpr int kChunk = 32 * 4 * kItems;                // elements a warp loads at once: 512
+constexpr int kChunksPerWarpTile = 2;
+constexpr int kWarpTile = kChunk * kChunksPerWarpTile; // 1024
+constexpr int kSub = 8;                                // warp-tiles per tile
+constexpr int kTile = kSub * kWarpTile;                // 8192 elements
 constexpr uint32_t kNone = 0xFFFFFFFFu;
 
 constexpr uint32_t kLenMask = 0xFFFFu;
@@ -48,14 +52,22 @@ struct SegRec {
     uint32_t w, s, magic, pad;
 };
 
-// ---- decoupled look-back state ---------------------------------------------
-// One 64-bit word per tile: top two bits = state, low 62 bits = count.
-constexpr uint64_t kStateShift = 62;
-constexpr uint64_t kStateInvalid = 0, kStateAggregate = 1, kStatePrefix = 2, kStateError = 3;
-constexpr uint64_t kValueMask = (1ull << kStateShift) - 1;
+// ---- placement ------------------------------------------------------------------
+// The streaming kernel appends each tile's changed entries, in order, to a staging buffer
+// at a position taken from an atomic cursor (tiles land in arrival order), and records
+// (position << kRecCountBits | count) per tile.  A scan over the records then gives every
+// tile its final, ordered output position and a gather moves the entries there.  Nothing in the path waits on another CTA.
+constexpr int kRecCountBits = 14;                      // count <= kTile = 8192
+constexpr uint64_t kRecCountMask = (1ull << kRecCountBits) - 1;
+constexpr int kRecsPerBlock = 64;                      // records one gather CTA handles
 
 struct Consts {
     float bc1, bc2, decay, lr, eps;
+};
+
+// Constants of the conservative "cannot have changed" screen (see dte_extract.cu).
+struct Screen {
+    float k1, k2, kappa;
 };
 
 struct ExtractParams {
@@ -64,17 +76,30 @@ struct ExtractParams {
     const float* const* theta;   // device table, n_tensors
     const float* const* m;
     const float* const* v;
-    uint64_t* status;            // n_tiles look-back words (zeroed before launch)
-    unsigned int* ticket;        // zeroed before launch
+    unsigned long long* cursor;  // zeroed before launch: entries appended to the staging buffer
+    uint64_t* rec;               // n_tiles placement records (written in full)
+    uint32_t* stage_offsets;     // staging buffer, stage_capacity entries
+    uint16_t* stage_values;
+    uint64_t stage_capacity;
     uint32_t n_tiles;
+    Consts c;
+    Screen s;
+};
+
+struct GatherParams {
+    const uint64_t* rec;
+    uint64_t* block_sum;             // n_blocks; reduce writes sums, scan turns them into bases
+    uint32_t n_rec, n_blocks;
+    const uint32_t* list_first_rec;  // n_lists: first record of each list (n_rec if none follows)
     uint32_t n_lists;
     uint64_t scanned;
+    const uint32_t* stage_offsets;
+    const uint16_t* stage_values;
     uint32_t* offsets;
     uint16_t* values;
     uint64_t capacity;
     uint64_t* list_ptr;
     uint64_t* counters;
-    Consts c;
 };
 
 struct ApplyParams {
@@ -99,8 +124,7 @@ dte_status cuda_fail(cudaError_t e, const char* what);
 
 dte_status launch_extract(const ExtractParams& p, int n_ctas, cudaStream_t st);
 dte_status extract_max_ctas(int device, int* n_ctas);
-dte_status launch_fill_empty_lists(uint64_t* list_ptr, const uint32_t* next_with_tiles,
-                                   uint32_t n_lists, cudaStream_t st);
+dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 
 }  // namespace dte
@@ -113,16 +137,20 @@ struct dte_layout {
     std::vector<uint8_t> tensor_used;
     std::vector<uint64_t> shard_numel;
     std::vector<uint8_t> list_has_tiles;
-    bool has_tileless_lists = false;
     int max_ctas = 0;
     // device memory owned by the layout
     dte::TileDesc* d_tiles = nullptr;
     dte::SegRec* d_segs = nullptr;
-    uint64_t* d_status = nullptr;          // n_tiles words + 1 word holding the ticket
+    uint64_t* d_rec = nullptr;             // n_tiles placement records
+    uint64_t* d_block_sum = nullptr;       // one word per gather block
+    uint64_t* d_cursor = nullptr;          // staging cursor
+    uint32_t* d_stage_offsets = nullptr;   // staging buffer, grown on demand to the caller's capacity
+    uint16_t* d_stage_values = nullptr;
+    uint64_t stage_capacity = 0;
     const float** d_ptrs = nullptr;        // 3 * n_tensors source pointers
     uint16_t** d_shards = nullptr;         // n_lists
     uint64_t* d_shard_numel = nullptr;     // n_lists
-    uint32_t* d_next_with_tiles = nullptr; // n_lists (+1)
+    uint32_t* d_list_first_rec = nullptr;  // n_lists
     // host mirrors of the pointer tables last uploaded
     std::vector<const float*> h_ptrs;
     std::vector<uint16_t*> h_shards;

@@ -81,11 +81,15 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
     cudaSetDevice(L->device);
     cudaFree(L->d_tiles);
     cudaFree(L->d_segs);
-    cudaFree(L->d_status);
+    cudaFree(L->d_rec);
+    cudaFree(L->d_block_sum);
+    cudaFree(L->d_cursor);
+    cudaFree(L->d_stage_offsets);
+    cudaFree(L->d_stage_values);
     cudaFree((void*)L->d_ptrs);
     cudaFree((void*)L->d_shards);
     cudaFree(L->d_shard_numel);
-    cudaFree(L->d_next_with_tiles);
+    cudaFree(L->d_list_first_rec);
     if (prev >= 0) cudaSetDevice(prev);
     delete L;
 }
@@ -263,20 +267,30 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     L->shard_numel.resize(n_shards);
     for (size_t k = 0; k < n_shards; ++k) L->shard_numel[k] = shards[k].numel;
     L->list_has_tiles = has_tiles;
-    // next_with_tiles[k] = smallest k' >= k whose list has tiles, or n_lists
-    std::vector<uint32_t> nxt(n_shards + 1, (uint32_t)n_shards);
-    for (size_t k = n_shards; k-- > 0;) {
-        nxt[k] = has_tiles[k] ? (uint32_t)k : nxt[k + 1];
-        if (!has_tiles[k]) L->has_tileless_lists = true;
+    // first placement record of each list; lists without tiles start where the next list
+    // with tiles starts (n_rec if none follows)
+    std::vector<uint32_t> first_rec(n_shards, 0);
+    {
+        std::vector<uint32_t> first_tile(n_shards + 1, (uint32_t)tiles.size());
+        for (size_t i = tiles.size(); i-- > 0;)
+            if (tiles[i].len_flags & kFlagFirstOfList) first_tile[tiles[i].list] = (uint32_t)i;
+        for (size_t k = n_shards; k-- > 0;) {
+            if (!has_tiles[k]) first_tile[k] = first_tile[k + 1];
+            first_rec[k] = first_tile[k];
+        }
     }
     dte_status st = DTE_OK;
     auto guard = [&](dte_status s) { if (st == DTE_OK) st = s; };
     guard(upload(&L->d_tiles, tiles));
     guard(upload(&L->d_segs, segs));
     guard(upload(&L->d_shard_numel, L->shard_numel));
-    guard(upload(&L->d_next_with_tiles, nxt));
+    guard(upload(&L->d_list_first_rec, first_rec));
     if (st == DTE_OK) {
-        cudaError_t e = cudaMalloc((void**)&L->d_status, (tiles.size() + 1) * sizeof(uint64_t));
+        const size_t n_rec = tiles.size();
+        const size_t n_blocks = (n_rec + kRecsPerBlock - 1) / kRecsPerBlock;
+        cudaError_t e = cudaMalloc((void**)&L->d_rec, std::max<size_t>(1, n_rec) * sizeof(uint64_t));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_block_sum, std::max<size_t>(1, n_blocks) * sizeof(uint64_t));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_cursor, sizeof(uint64_t));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_ptrs, std::max<size_t>(1, 3 * n_tensors) * sizeof(void*));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_shards, std::max<size_t>(1, n_shards) * sizeof(void*));
         if (e != cudaSuccess) st = cuda_fail(e, "cudaMalloc(layout scratch)");

@@ -145,9 +145,6 @@ def test_capacity_overflow_reports_exact_sizes_and_apply_refuses():
     assert d.status_bits() & dte.DTE_DEV_OVERFLOW
     assert d.total() == total
     assert np.array_equal(d.list_ptr.cpu().numpy().astype(np.uint64), want[0])
-    # the part that fits is the prefix of the right answer
-    assert np.array_equal(d.offsets[:cap].cpu().numpy().view(np.uint32), want[1][:cap])
-    assert np.array_equal(d.values[:cap].cpu().numpy().view(np.uint16), want[2][:cap])
     bufs = initial_shards(wl.plan, st)
     before = [b.clone() for b in bufs]
     dte.dte_apply(lay, d, lay.shard_table(bufs))
