@@ -157,6 +157,35 @@ DTE_API dte_status dte_extract_delta(const dte_layout* layout, const float* cons
                              double lr, double beta1, double beta2, double eps, double wd,
                              const dte_delta* out, void* cuda_stream);
 
+/* Allocation-free variant of dte_extract_delta.  The paper has no counterpart: this exists
+ * for callers that may not allocate device memory at the point where they extract - a
+ * trainer whose framework has claimed the whole GPU for its own caching allocator, so that a
+ * raw cudaMalloc would fail or fragment it; a process running under a fixed memory budget; a
+ * latency-critical loop that cannot afford the implicit synchronisation of cudaMalloc /
+ * cudaFree.  dte_extract_delta grows a per-layout staging buffer when a call brings a larger
+ * `capacity`; this entry point never does.  Its placement records, block sums, cursor and
+ * staging buffer live in one fixed array inside the library's device image (about 12.5 MiB;
+ * every GPU that loads the library holds it until the process exits), and it calls no
+ * cudaMalloc, cudaFree or other device-allocating routine.
+ *   Limits: the layout may have at most DTE_STATIC_MAX_TILES tiles (a tile is up to 8192
+ * consecutive destination slots of one operation, so up to 536,870,912 scanned elements when
+ * the tiles are full) and out->capacity at most DTE_STATIC_MAX_CAPACITY entries.  Larger
+ * requests return DTE_ERR_CAPACITY with the numbers in dte_last_error(); nothing is enqueued.
+ *   The first call on a device looks up the array's address on that device (a host-side
+ * query, once per device and process); make that first call before starting a stream capture.
+ *   All calls on a device share the array, and it keeps what the last call left.  The call
+ * clears the one word that must start at zero and overwrites the rest before reading it, so
+ * back-to-back calls on one stream are safe; two calls that can overlap on the GPU (different
+ * streams, different layouts or host threads) race on the array and corrupt each other.
+ *   Arguments, results and all other error behaviour are those of dte_extract_delta; the
+ * caller still provides every input and output buffer. */
+#define DTE_STATIC_MAX_TILES 65536u
+#define DTE_STATIC_MAX_CAPACITY 2097152u
+DTE_API dte_status dte_extract_delta_static(const dte_layout* layout, const float* const* theta,
+                                            const float* const* m, const float* const* v, int64_t step,
+                                            double lr, double beta1, double beta2, double eps, double wd,
+                                            const dte_delta* out, void* cuda_stream);
+
 /* Eq. 7: shard[k][offsets[e]] = values[e] for every entry e of every list k.
  * shard_ptrs: HOST array of n_shards DEVICE pointers (BF16 buffers, numel as declared;
  * shards whose lists are necessarily empty may be NULL).  Reads list sizes on the device,

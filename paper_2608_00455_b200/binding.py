@@ -23,6 +23,7 @@ SYMBOLS = [
     "dte_layout_create", "dte_layout_destroy", "dte_layout_num_lists", "dte_layout_num_elements",
     "dte_layout_host_workspace_bytes", "dte_derive_constants", "dte_extract_delta", "dte_apply",
     "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
+    "dte_extract_delta_static",
 ]
 
 
@@ -79,6 +80,8 @@ def lib() -> C.CDLL:
         L.dte_derive_constants.restype = C.c_int
         L.dte_extract_delta.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, vp]
         L.dte_extract_delta.restype = C.c_int
+        L.dte_extract_delta_static.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, vp]
+        L.dte_extract_delta_static.restype = C.c_int
         L.dte_apply.argtypes = [vp, vp, vp, vp]
         L.dte_apply.restype = C.c_int
         L.dte_extract_delta_host.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, u64,
@@ -251,6 +254,25 @@ def dte_extract_delta(layout: Layout, tables, step, lr, beta1, beta2, eps, wd, d
     _check(lib().dte_extract_delta(layout._h, th, mm, vv, int(step), float(lr), float(beta1),
                                    float(beta2), float(eps), float(wd), C.byref(delta.struct),
                                    _stream_ptr(stream)))
+
+
+STATIC_MAX_TILES = 65536
+STATIC_MAX_CAPACITY = 2097152
+
+
+def dte_extract_delta_static(layout: Layout, tables, step, lr, beta1, beta2, eps, wd, delta: Delta,
+                             stream=None) -> None:
+    """dte_extract_delta for callers that must not allocate device memory.
+
+    Same arguments and results; the call's scratch is a fixed array inside the library, so
+    it is limited to layouts of at most STATIC_MAX_TILES tiles and deltas of at most
+    STATIC_MAX_CAPACITY entries (DteError with status 3 beyond that), and two calls that can
+    overlap on one GPU must not be issued.  See dte_extract_delta_static in include/dte.h.
+    """
+    th, mm, vv = tables
+    _check(lib().dte_extract_delta_static(layout._h, th, mm, vv, int(step), float(lr), float(beta1),
+                                          float(beta2), float(eps), float(wd), C.byref(delta.struct),
+                                          _stream_ptr(stream)))
 
 
 def dte_apply(layout: Layout, delta: Delta, shard_table, stream=None) -> None:

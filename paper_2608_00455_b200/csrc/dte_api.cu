@@ -249,3 +249,123 @@ extern "C" dte_status dte_extract_delta_host(const dte_layout* layout, const flo
     DTE_CUDA(cudaStreamSynchronize(st));
     return DTE_OK;
 }
+
+// ---- allocation-free extract --------------------------------------------------------------
+//
+// Same computation as dte_extract_delta, for callers that must not allocate device memory
+// while they run.  Everything the ordinary call keeps in per-layout scratch that it may
+// have to (re)allocate - the placement records, the gather's block sums, the staging cursor
+// and the staging buffer - lives here in one fixed array in the library's device image.
+// Each GPU that loads the library carries the array until the process exits.
+
+namespace {
+
+constexpr uint64_t kStaticMaxTiles = DTE_STATIC_MAX_TILES;
+constexpr uint64_t kStaticMaxCapacity = DTE_STATIC_MAX_CAPACITY;
+constexpr uint64_t kStaticCursorOff = 0;                                       // 256 bytes reserved
+constexpr uint64_t kStaticRecOff = 256;
+constexpr uint64_t kStaticBlockSumOff = kStaticRecOff + kStaticMaxTiles * 8;
+constexpr uint64_t kStaticStageOffOff =
+    kStaticBlockSumOff + ((kStaticMaxTiles + kRecsPerBlock - 1) / kRecsPerBlock) * 8;
+constexpr uint64_t kStaticStageValOff = kStaticStageOffOff + kStaticMaxCapacity * 4;
+constexpr uint64_t kStaticScratchBytes = (kStaticStageValOff + kStaticMaxCapacity * 2 + 255) / 256 * 256;
+static_assert(kStaticBlockSumOff % 8 == 0 && kStaticStageOffOff % 8 == 0 && kStaticStageValOff % 4 == 0,
+              "sub-buffers must keep their natural alignment");
+
+// In host code this name is only a handle for the runtime's symbol table, never a device
+// address: the address each device gave the array comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_addr[kMaxDevices] = {nullptr};
+
+// First use on a device (that device current): ask the runtime where the array lives there.
+dte_status static_scratch_address(int device, unsigned char** out) {
+    if (device < 0 || device >= kMaxDevices) return fail(DTE_ERR_INVALID_ARG, "device ordinal out of range");
+    if (!g_static_addr[device]) {
+        void* ptr = nullptr;
+        DTE_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (!ptr) return fail(DTE_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
+        g_static_addr[device] = static_cast<unsigned char*>(ptr);
+    }
+    *out = g_static_addr[device];
+    return DTE_OK;
+}
+
+}  // namespace
+
+extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const float* const* theta,
+                                               const float* const* m, const float* const* v,
+                                               int64_t step, double lr, double beta1, double beta2,
+                                               double eps, double wd, const dte_delta* out,
+                                               void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    if (layout->n_tensors && (!theta || !m || !v)) return fail(DTE_ERR_INVALID_ARG, "null pointer table");
+    dte_status s = check_delta(out);
+    if (s != DTE_OK) return s;
+    if (layout->n_tiles > kStaticMaxTiles) {
+        set_error("dte_extract_delta_static: the layout has " + std::to_string(layout->n_tiles) +
+                  " tiles, the fixed scratch holds " + std::to_string(kStaticMaxTiles) +
+                  "; use dte_extract_delta");
+        return DTE_ERR_CAPACITY;
+    }
+    if (out->capacity > kStaticMaxCapacity) {
+        set_error("dte_extract_delta_static: capacity " + std::to_string(out->capacity) +
+                  " exceeds the fixed staging buffer of " + std::to_string(kStaticMaxCapacity) +
+                  " entries; use dte_extract_delta");
+        return DTE_ERR_CAPACITY;
+    }
+    float c5[5];
+    s = dte_derive_constants(step, lr, beta1, beta2, eps, wd, c5);
+    if (s != DTE_OK) return s;
+    dte_layout* L = const_cast<dte_layout*>(layout);
+    DeviceGuard g(L->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    unsigned char* base = nullptr;
+    s = static_scratch_address(L->device, &base);
+    if (s != DTE_OK) return s;
+    s = sync_source_table(L, theta, m, v, st);
+    if (s != DTE_OK) return s;
+    DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
+    if (L->n_tiles == 0) {
+        DTE_CUDA(cudaMemsetAsync(out->list_ptr, 0, (L->n_lists + 1) * sizeof(uint64_t), st));
+        return DTE_OK;
+    }
+    // the array keeps whatever the previous call left: only the cursor has to start at zero
+    // (records and block sums are rewritten in full, staged entries are read only where this
+    // call wrote them)
+    DTE_CUDA(cudaMemsetAsync(base + kStaticCursorOff, 0, sizeof(uint64_t), st));
+    const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
+    ExtractParams p;
+    p.tiles = L->d_tiles;
+    p.segs = L->d_segs;
+    p.theta = L->d_ptrs;
+    p.m = L->d_ptrs + L->n_tensors;
+    p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
+    p.cursor = reinterpret_cast<unsigned long long*>(base + kStaticCursorOff);
+    p.rec = reinterpret_cast<uint64_t*>(base + kStaticRecOff);
+    p.stage_offsets = reinterpret_cast<uint32_t*>(base + kStaticStageOffOff);
+    p.stage_values = reinterpret_cast<uint16_t*>(base + kStaticStageValOff);
+    p.stage_capacity = out->capacity;
+    p.n_tiles = L->n_tiles;
+    p.c = c;
+    p.s = make_screen(c);
+    s = launch_extract(p, (int)L->n_tiles, st);
+    if (s != DTE_OK) return s;
+    GatherParams gp;
+    gp.rec = p.rec;
+    gp.block_sum = reinterpret_cast<uint64_t*>(base + kStaticBlockSumOff);
+    gp.n_rec = L->n_tiles;
+    gp.n_blocks = (L->n_tiles + kRecsPerBlock - 1) / kRecsPerBlock;
+    gp.list_first_rec = L->d_list_first_rec;
+    gp.n_lists = L->n_lists;
+    gp.scanned = L->scanned;
+    gp.stage_offsets = p.stage_offsets;
+    gp.stage_values = p.stage_values;
+    gp.offsets = out->offsets;
+    gp.values = out->values;
+    gp.capacity = out->capacity;
+    gp.list_ptr = out->list_ptr;
+    gp.counters = out->counters;
+    return launch_gather(gp, st);
+}
