@@ -35,7 +35,7 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per scanned element of the extract kernel, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over a 2.3 GB case, per element).
-NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT = None
+NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT = 12.112
 
 
 def log(*a):
@@ -226,10 +226,21 @@ def run_reference(args, rank):
     print(json.dumps(out), flush=True)
 
 
+def aggregate_over_ranks(ms_local: float, units_local: float, dist, device):
+    """Weak scaling: the job's time is the slowest rank's, its units the sum over ranks."""
+    if dist is None:
+        return ms_local, units_local
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device)
+    u = torch.tensor([units_local], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    dist.all_reduce(u, op=dist.ReduceOp.SUM)
+    return float(t.item()), float(u.item())
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=30)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="dte", choices=["dte", "reference"])
     ap.add_argument("--workload", default="full")
@@ -324,13 +335,10 @@ def main():
     ext_ms = [e[0].elapsed_time(e[1]) for e in evs]
     app_ms = [e[1].elapsed_time(e[2]) for e in evs]
     launches = lay.last_launch()["kernels"] * args.steps + args.steps
-    if dist:
-        t = torch.tensor([total_ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
-    ms_per_step = total_ms / args.steps
     bytes_per_step = 12.0 * N + 6.0 * M
-    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    total_ms, bytes_all = aggregate_over_ranks(total_ms, bytes_per_step, dist, device)
+    ms_per_step = total_ms / args.steps
+    value = bytes_all / (ms_per_step * 1e-3) / 1e9
     ext_avg = sum(ext_ms) / len(ext_ms)
     app_avg = sum(app_ms) / len(app_ms)
     peak, peak_kind = measured_peak()
@@ -437,14 +445,11 @@ def run_e2e(args, wl, st, device, dte, world, dist):
     e1.record(stream)
     torch.cuda.synchronize()
     ms = e0.elapsed_time(e1) / steps
-    if dist:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
     M = int(res.counters[0])
+    ms, bytes_all = aggregate_over_ranks(ms, 12.0 * N + 6.0 * M, dist, device)
     h2d = 12 * sub.total_source_elements()
     d2h = 6 * M + 8 * (lay.num_lists + 1) + 32
-    return {"value": world * (12.0 * N + 6.0 * M) / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
+    return {"value": bytes_all / (ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": ms,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": steps,
             "workload": f"first {len(chosen)} source tensors of {wl.name} held in pinned host memory "
                         f"({N} scanned elements); PCIe-bound"}

@@ -1,0 +1,132 @@
+"""Full-size parity in the launch configuration bench.py times: the whole Qwen3-8B-shaped state
+(config 3, 98 GB) and the Qwen3-30B-A3B slice (config 4, 90 GB) resident on one GPU.  The oracle
+checks complete lists of sampled tensors; properties that hold at any size cover the rest."""
+import gc
+
+import numpy as np
+import pytest
+import torch
+
+import bench
+import oracle
+import paper_2608_00455_b200 as dte
+from synth import configs
+from gpu_util import assert_lists_equal
+
+pytestmark = pytest.mark.gpu
+
+
+def _free():
+    gc.collect()
+    torch.cuda.empty_cache()
+
+
+def _need(gb):
+    free, total = torch.cuda.mem_get_info()
+    if free < gb * 1e9:
+        pytest.skip(f"needs {gb} GB of free device memory, {free / 1e9:.0f} GB available")
+
+
+def _global_properties(plan, lay, d):
+    """list_ptr monotone and consistent with the counters; every list strictly ascending and in range."""
+    assert d.status_bits() == 0
+    lp = d.list_ptr.cpu().numpy().astype(np.int64)
+    cnt = d.counters.cpu().numpy()
+    assert lp[0] == 0 and np.all(np.diff(lp) >= 0) and lp[-1] == cnt[0]
+    assert cnt[1] == plan.total_scanned_elements() == lay.num_elements
+    off = d.offsets[:int(lp[-1])].to(torch.int64) & 0xFFFFFFFF
+    dif = off[1:] - off[:-1]
+    starts = torch.from_numpy(lp[1:-1]).to(off.device)
+    starts = starts[(starts > 0) & (starts < off.numel())]
+    ok = dif > 0
+    ok[starts - 1] = True                       # list boundaries may go down
+    assert bool(ok.all())
+    numel = torch.tensor(plan.shard_numels, device=off.device)
+    counts = torch.from_numpy(np.diff(lp)).to(off.device)
+    bound = torch.repeat_interleave(numel, counts)
+    assert bool((off < bound).all())
+    return lp
+
+
+def _sampled_lists_equal(wl, st, d, tensors):
+    """Oracle on `tensors` only; compare every list that those tensors fill completely."""
+    plan = wl.plan
+    shapes, ops, host = bench.oracle_inputs(plan, st, tensors)
+    c = oracle.derive_constants(*wl.hp.as_args())
+    want = oracle.extract(shapes, plan.shard_numels, ops, *host, c)
+    chosen = set(tensors)
+    lists = [k for k in sorted(set(int(x) for x in ops[:, 1]))
+             if all(int(o[0]) in chosen for o in plan.ops if o[1] == k)]
+    assert lists
+    got = d.to_host()
+    assert_lists_equal(got, want, plan, lists)
+    return lists, want
+
+
+def _apply_end_state(plan, st, lay, d, shards, sample_shards):
+    """After apply the sampled receiver tensors equal remapped BF16(theta_t) except for the
+    elements the reconstruction missed (mirror generator: none to a handful)."""
+    dte.dte_apply(lay, d, lay.shard_table(shards))
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    ops_by_shard = {}
+    for o in plan.ops:
+        ops_by_shard.setdefault(o[1], []).append(o)
+    stale = 0
+    for k in sample_shards:
+        exp = torch.zeros_like(shards[k])
+        for (src, _, a0, a1, e0, e1, base, ld, r0, r1) in ops_by_shard[k]:
+            s2 = st.theta[src].reshape(plan.tensor_shapes[src])[a0:a0 + e0, a1:a1 + e1]
+            exp.as_strided((e0, e1), (ld, 1), base + r0 * ld + r1).copy_(s2.to(torch.bfloat16).view(torch.int16))
+        stale += int((exp != shards[k]).sum().item())
+    return stale
+
+
+def test_config3_full_qwen3_8b_state():
+    _need(150)
+    wl = configs.config3("cuda")
+    plan = wl.plan
+    st, shards = bench.materialize_resident(wl, torch.device("cuda", 0), dte)
+    lay = dte.Layout.from_plan(plan, 0)
+    N = lay.num_elements
+    assert N == 8191035392
+    d = lay.new_delta(int(N * 0.03))
+    dte.dte_extract_delta(lay, lay.source_tables(st.theta, st.m, st.v), *wl.hp.as_args(), d)
+    torch.cuda.synchronize()
+    lp = _global_properties(plan, lay, d)
+    assert 0.01 < lp[-1] / N < 0.02
+    # all 11 tensors of layer 17 (row- and column-split, replicated norms) and embed_tokens
+    names = plan.tensor_names
+    sample = [p for p, n in enumerate(names) if n.startswith("layers.17.")] + [names.index("embed_tokens")]
+    lists, _ = _sampled_lists_equal(wl, st, d, sample)
+    assert len(lists) == 18
+    assert _apply_end_state(plan, st, lay, d, shards, lists) <= 8
+    del st, shards, d, lay
+    _free()
+
+
+def test_config4_qwen3_30b_a3b_slice():
+    _need(150)
+    wl = configs.config4("cuda")
+    plan = wl.plan
+    assert (plan.n_shards, len(plan.ops)) == (432, 5040)
+    st, shards = bench.materialize_resident(wl, torch.device("cuda", 0), dte)
+    lay = dte.Layout.from_plan(plan, 0)
+    N = lay.num_elements
+    d = lay.new_delta(int(N * 0.04))
+    dte.dte_extract_delta(lay, lay.source_tables(st.theta, st.m, st.v), *wl.hp.as_args(), d)
+    torch.cuda.synchronize()
+    _global_properties(plan, lay, d)
+    assert wl.notes["cold_experts"] > 0
+    # layer 5 completely: attention, router, norms and all 128 experts (cold ones included)
+    sample = [p for p, n in enumerate(plan.tensor_names) if n.startswith("layers.5.")]
+    lists, want = _sampled_lists_equal(wl, st, d, sample)
+    assert len(lists) == 36
+    # cold experts (zero state) contribute nothing
+    cold = [p for p in sample if "experts" in plan.tensor_names[p] and wl.specs[p].scale == 0.0]
+    assert cold
+    for p in cold[:6]:
+        assert float(st.m[p].abs().max()) == 0.0 and float(st.v[p].abs().max()) == 0.0
+    assert _apply_end_state(plan, st, lay, d, shards, lists) <= 8
+    del st, shards, d, lay
+    _free()
