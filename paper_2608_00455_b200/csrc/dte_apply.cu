@@ -6,6 +6,8 @@
 namespace dte {
 
 constexpr int kApplyThreads = 256;
+constexpr int kApplyPerThread = 8;                      // entries in flight per thread
+constexpr int kApplyChunk = kApplyThreads * kApplyPerThread;
 constexpr int kApplySmemLists = 4096;  // list_ptr entries cached in shared memory
 
 __global__ void __launch_bounds__(kApplyThreads) apply_kernel(const ApplyParams p) {
@@ -24,19 +26,44 @@ __global__ void __launch_bounds__(kApplyThreads) apply_kernel(const ApplyParams 
             atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_OVERFLOW);
         return;
     }
-    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     bool bad = false;
-    for (uint64_t e = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += stride) {
-        // largest k with lp[k] <= e (lists may be empty, so take the upper bound)
-        uint32_t lo = 0, hi = L;
-        while (hi - lo > 1) {
-            const uint32_t mid = (lo + hi) >> 1;
-            if (lp[mid] <= e) lo = mid; else hi = mid;
+    for (uint64_t base = (uint64_t)blockIdx.x * kApplyChunk; base < total; base += (uint64_t)gridDim.x * kApplyChunk) {
+        // all loads of the chunk first: 16 independent requests per thread
+        uint32_t off[kApplyPerThread];
+        uint16_t val[kApplyPerThread];
+#pragma unroll
+        for (int j = 0; j < kApplyPerThread; ++j) {
+            const uint64_t e = base + (uint64_t)j * kApplyThreads + threadIdx.x;
+            if (e < total) {
+                off[j] = __ldcs(p.offsets + e);
+                val[j] = __ldcs(p.values + e);
+            }
         }
-        const uint32_t off = __ldcs(p.offsets + e);
-        const uint16_t val = __ldcs(p.values + e);
-        if ((uint64_t)off < p.shard_numel[lo]) p.shards[lo][off] = val;
-        else bad = true;
+        // list of the thread's first entry: largest k with lp[k] <= e (lists may be empty);
+        // the later entries of the thread only ever move forward from there
+        uint32_t k = 0;
+        {
+            const uint64_t e = base + threadIdx.x;
+            uint32_t lo = 0, hi = L;
+            while (hi - lo > 1) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (lp[mid] <= e) lo = mid; else hi = mid;
+            }
+            k = lo;
+        }
+#pragma unroll
+        for (int j = 0; j < kApplyPerThread; ++j) {
+            const uint64_t e = base + (uint64_t)j * kApplyThreads + threadIdx.x;
+            if (e < total) {
+                while (e >= lp[k + 1]) ++k;          // e < total = lp[L] keeps k < L
+                if ((uint64_t)off[j] < __ldg(p.shard_numel + k)) {
+                    uint16_t* dst = reinterpret_cast<uint16_t*>(__ldg(reinterpret_cast<const unsigned long long*>(p.shards + k)));
+                    dst[off[j]] = val[j];
+                } else {
+                    bad = true;
+                }
+            }
+        }
     }
     if (bad) atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_BOUNDS);
 }
@@ -44,7 +71,7 @@ __global__ void __launch_bounds__(kApplyThreads) apply_kernel(const ApplyParams 
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st) {
     int sms = 0;
     DTE_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    apply_kernel<<<sms * 8, kApplyThreads, 0, st>>>(p);
+    apply_kernel<<<sms * 6, kApplyThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }
