@@ -1,0 +1,68 @@
+"""Adversarial inputs for the extract kernel's conservative screen: theta within a few fp32
+ulps of a BF16 rounding boundary and update terms of about the same size, so that the
+decision "cannot have changed" is taken right at its threshold.  Bit-exact against the oracle."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2608_00455_b200 as dte
+from synth import plans
+from synth.tensors import Hyper
+
+pytestmark = pytest.mark.gpu
+
+
+def _near_boundary_state(n, hp: Hyper, seed, spread_ulps=24, with_specials=True):
+    """theta = BF16 tie point +- a few ulps; m, v chosen so |lr*u| is 0..2*spread ulps of theta."""
+    rng = np.random.default_rng(seed)
+    upper = rng.integers(0x3000, 0x4800, size=n, dtype=np.uint32)         # exponents 2^-31 .. 2^17
+    sign = rng.integers(0, 2, size=n, dtype=np.uint32) << 31
+    delta = rng.integers(-spread_ulps, spread_ulps + 1, size=n).astype(np.int64)
+    bits = ((upper.astype(np.int64) << 16) + 0x8000 + delta).astype(np.uint32) | sign
+    theta = bits.view(np.float32).copy()
+    ulp = np.spacing(np.abs(theta)).astype(np.float64)
+    want_step = rng.uniform(0, 2 * spread_ulps, size=n) * ulp * rng.choice([-1.0, 1.0], size=n)
+    c = oracle.derive_constants(*hp.as_args()).astype(np.float64)
+    v = np.abs(rng.standard_normal(n) * 1e-6).astype(np.float32) + np.float32(1e-12)
+    # lr * (m/bc1) / (sqrt(v/bc2) + eps) ~= want_step  =>  m
+    m = (want_step / c[3] * (np.sqrt(v.astype(np.float64) / c[1]) + c[4]) * c[0]).astype(np.float32)
+    if with_specials:
+        k = n // 64
+        v[:k] = 0.0                                   # eps-dominated denominators
+        m[k:2 * k] = 0.0
+        v[2 * k:3 * k] = np.float32(1e-42)            # subnormal second moment
+        theta[3 * k:3 * k + 16] = 0.0
+        m[3 * k + 16:3 * k + 32] = np.float32(np.inf)
+        v[3 * k + 32:3 * k + 48] = -1.0
+        theta[3 * k + 48:3 * k + 64] = np.float32(np.nan)
+    return theta, m, v
+
+
+@pytest.mark.parametrize("hp", [
+    Hyper(step=500, lr=1e-6, wd=0.01),        # bc1 == 1, decay == 1
+    Hyper(step=100, lr=1e-6, wd=0.01),        # bc1 != 1, decay == 1
+    Hyper(step=500, lr=1e-4, wd=0.1),         # bc1 == 1, decay != 1
+    Hyper(step=1, lr=3e-4, wd=0.3),           # both divisions, extreme bias correction
+    Hyper(step=7, lr=1e-3, wd=0.0, eps=0.0),  # eps == 0
+    Hyper(step=50, lr=1e-5, wd=5.0, beta1=0.5, beta2=0.9),
+], ids=lambda h: f"t{h.step}-lr{h.lr:g}-wd{h.wd:g}-eps{h.eps:g}")
+def test_screen_threshold_cases_match_oracle(hp):
+    rows, cols = 4096, 2048
+    n = rows * cols
+    theta, m, v = _near_boundary_state(n, hp, seed=hp.step)
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    c = oracle.derive_constants(*hp.as_args())
+    want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), [theta], [m], [v], c)
+    lay = dte.Layout.from_plan(plan, 0)
+    d = lay.new_delta(n)
+    t, mm, vv = (torch.from_numpy(a).cuda() for a in (theta, m, v))
+    dte.dte_extract_delta(lay, lay.source_tables([t], [mm], [vv]), *hp.as_args(), d)
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    lp, off, val = d.to_host()
+    assert np.array_equal(lp, want[0])
+    assert np.array_equal(off, want[1])
+    assert np.array_equal(val, want[2])
+    frac = int(lp[-1]) / n
+    assert 0.05 < frac < 0.95, frac            # the cases really straddle the decision
