@@ -246,7 +246,7 @@ def main():
     ap.add_argument("--workload", default="full")
     ap.add_argument("--capacity-frac", type=float, default=0.03)
     ap.add_argument("--e2e-gb", type=float, default=10.0, help="host-resident state for the e2e leg (GB)")
-    ap.add_argument("--cpu-elements", type=float, default=1.2e9, help="oracle sample size (elements)")
+    ap.add_argument("--cpu-elements", type=float, default=2.0e9, help="oracle sample size (elements)")
     ap.add_argument("--ref-elements", type=float, default=4e8, help="--impl reference: elements per step")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")

@@ -71,6 +71,9 @@ __global__ void __launch_bounds__(kApplyThreads) apply_kernel(const ApplyParams 
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st) {
     int sms = 0;
     DTE_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    // 6 CTAs per SM is what the 32 KB list_ptr cache allows; measured on B200: 3, 6 and 12 CTAs
+    // per SM and .cs / .cg / .wt store hints all give the same ~39 G entries/s - isolated
+    // 2-byte writes are bound by the memory system's sector read-modify-write rate
     apply_kernel<<<sms * 6, kApplyThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;

@@ -222,3 +222,56 @@ def test_layout_errors():
     with pytest.raises(dte.DteError):                                     # step 0
         dte.dte_extract_delta(lay, lay.source_tables([t[:64]], [t[:64]], [t[:64]]), 0, 1e-3, 0.9, 0.999, 1e-8, 0.0,
                               lay.new_delta(64))
+
+
+def test_empty_layouts_and_empty_operations():
+    # no operations at all: every list empty, nothing launched
+    lay = dte.Layout([(8, 8)], [64, 0, 5], [])
+    d = lay.new_delta(4)
+    t = torch.ones(64, dtype=torch.float32, device="cuda")
+    d.list_ptr.fill_(7)
+    dte.dte_extract_delta(lay, lay.source_tables([t], [t], [t]), 1, 1e-3, 0.9, 0.999, 1e-8, 0.0, d)
+    torch.cuda.synchronize()
+    assert d.total() == 0 and d.status_bits() == 0 and int(d.list_ptr.abs().sum()) == 0
+    bufs = [torch.zeros(max(1, n), dtype=torch.int16, device="cuda") for n in (64, 0, 5)]
+    dte.dte_apply(lay, d, lay.shard_table(bufs))
+    torch.cuda.synchronize()
+    # an operation with an empty extent is legal and contributes nothing; tensor 1 is unused (NULL)
+    lay = dte.Layout([(8, 8), (4, 4)], [64], [(0, 0, 0, 0, 8, 8, 0, 8, 0, 0), (1, 0, 0, 0, 0, 4, 0, 4, 0, 0)])
+    d = lay.new_delta(64)
+    m = torch.full((64,), 0.5, dtype=torch.float32, device="cuda")
+    dte.dte_extract_delta(lay, lay.source_tables([t, None], [m, None], [m, None]), 1, 8.0, 0.5, 0.5, 0.0, 0.0, d)
+    torch.cuda.synchronize()
+    assert d.total() == 64 and lay.num_elements == 64
+
+
+def test_offsets_up_to_the_uint32_limit():
+    # destination tensor of 2^32 - 1 elements: offsets beyond 2^31 must survive extract and apply
+    free, _ = torch.cuda.mem_get_info()
+    if free < 12e9:
+        pytest.skip("needs 12 GB of device memory")
+    numel = (1 << 32) - 1
+    rows, cols = 40, 1000
+    base = numel - rows * cols                      # the block ends at the very last slot
+    plan = plans.Plan()
+    a = plan.add_tensor("a", (rows, cols))
+    k = plan.add_shard("huge", 0, numel)
+    plan.add_op(a, k, (0, 0), (rows, cols), base, cols, (0, 0))
+    wl = configs.Workload("huge", plan, Hyper(step=100, lr=1e-4, wd=0.01), [Spec()], 17)
+    st = wl.materialize("cuda")
+    lay, d = run_extract(plan, st, wl.hp)
+    got = d.to_host()
+    want = oracle_extract(plan, st, wl.hp)
+    assert_lists_equal(got, want, plan)
+    assert int(got[1].max()) > (1 << 31) and int(got[0][-1]) > 100
+    shard = torch.zeros(numel, dtype=torch.int16, device="cuda")
+    dte.dte_apply(lay, d, lay.shard_table([shard]))
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    tail = shard[base:].cpu().numpy().view(np.uint16)
+    exp = np.zeros(rows * cols, np.uint16)
+    exp[(want[1].astype(np.int64) - base)] = want[2]
+    assert np.array_equal(tail, exp)
+    assert int(shard[:base][-1000000:].abs().sum()) == 0
+    del shard
+    torch.cuda.empty_cache()
