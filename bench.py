@@ -100,6 +100,9 @@ def build_workload(name: str, device):
         return configs.config3(device)
     if name.startswith("layers:"):
         return configs.config3(device, n_layers=int(name.split(":")[1]), with_embeddings=False)
+    if name.startswith("mcore:"):        # mcore:<sender TP>:<receiver TP>:<dp slices>[:<layers>]
+        f = [int(x) for x in name.split(":")[1:]]
+        return configs.config3_mcore(device, f[0], f[1], f[2], n_layers=f[3] if len(f) > 3 else 36)
     if name == "config1":
         return configs.config1()
     if name == "config2":
@@ -118,12 +121,17 @@ def materialize_resident(wl, device, dte):
         ops_by_tensor.setdefault(o[0], []).append(o)
     st = configs.State([None] * plan.n_tensors, [None] * plan.n_tensors, [None] * plan.n_tensors,
                        [None] * plan.n_tensors)
-    for p in range(plan.n_tensors):
-        one = wl.materialize(device, [p])
-        st.theta[p], st.m[p], st.v[p] = one.theta[p], one.m[p], one.v[p]
-        prev = one.prev_bf16[p].view(torch.int16).reshape(plan.tensor_shapes[p])
-        for (_, dst, a0, a1, e0, e1, base, ld, r0, r1) in ops_by_tensor.get(p, []):
-            shards[dst].as_strided((e0, e1), (ld, 1), base + r0 * ld + r1).copy_(prev[a0:a0 + e0, a1:a1 + e1])
+    alias = wl.alias_of or list(range(plan.n_tensors))
+    members = {}
+    for p, a in enumerate(alias):
+        members.setdefault(a, []).append(p)
+    for base, group in members.items():
+        one = wl.materialize(device, [base])
+        prev = one.prev_bf16[base].view(torch.int16).reshape(plan.tensor_shapes[base])
+        for p in group:                  # slices of one shard share its allocation
+            st.theta[p], st.m[p], st.v[p] = one.theta[base], one.m[base], one.v[base]
+            for (_, dst, a0, a1, e0, e1, b0, ld, r0, r1) in ops_by_tensor.get(p, []):
+                shards[dst].as_strided((e0, e1), (ld, 1), b0 + r0 * ld + r1).copy_(prev[a0:a0 + e0, a1:a1 + e1])
         del one, prev
     return st, shards
 

@@ -320,13 +320,5 @@ dte_status launch_extract(const ExtractParams& p, int n_ctas, cudaStream_t st) {
     return launch_t<false, false>(p, n_ctas, st);
 }
 
-dte_status extract_max_ctas(int device, int* n_ctas) {
-    int sms = 0, per_sm = 0;
-    DTE_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-    DTE_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, extract_kernel<true, true>, kThreads, 0));
-    if (per_sm < 1) per_sm = 1;
-    *n_ctas = sms * per_sm;   // resident CTAs (informational: the grid is one CTA per tile)
-    return DTE_OK;
-}
 
 }  // namespace dte

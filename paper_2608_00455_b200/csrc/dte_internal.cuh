@@ -123,7 +123,6 @@ dte_status cuda_fail(cudaError_t e, const char* what);
     } while (0)
 
 dte_status launch_extract(const ExtractParams& p, int n_ctas, cudaStream_t st);
-dte_status extract_max_ctas(int device, int* n_ctas);
 dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 
@@ -137,7 +136,6 @@ struct dte_layout {
     std::vector<uint8_t> tensor_used;
     std::vector<uint64_t> shard_numel;
     std::vector<uint8_t> list_has_tiles;
-    int max_ctas = 0;
     // device memory owned by the layout
     dte::TileDesc* d_tiles = nullptr;
     dte::SegRec* d_segs = nullptr;

@@ -295,7 +295,6 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_shards, std::max<size_t>(1, n_shards) * sizeof(void*));
         if (e != cudaSuccess) st = cuda_fail(e, "cudaMalloc(layout scratch)");
     }
-    if (st == DTE_OK) st = extract_max_ctas(device, &L->max_ctas);
     if (prev >= 0) cudaSetDevice(prev);
     if (st != DTE_OK) {
         std::string keep = g_last_error;

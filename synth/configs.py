@@ -39,6 +39,8 @@ class Workload:
     plant: bool = False
     plant_nonfinite: bool = False
     notes: Dict[str, object] = field(default_factory=dict)
+    # alias_of[p] = tensor whose allocation p shares (distributed-optimizer slices of one shard)
+    alias_of: Optional[List[int]] = None
 
     def materialize(self, device, tensors: Optional[List[int]] = None) -> State:
         """Generate theta_t/m_t/v_t (+BF16 theta_{t-1}) for all (or the listed) tensors."""
@@ -84,6 +86,21 @@ def config3(device, n_layers=36, tp=2, seed=1234, dims=P.QWEN3_8B, with_embeddin
     w = calibrate_sigma_g(WEIGHT, HP_T500, seed, device, target)
     wl = Workload(f"qwen3-8b.full{n_layers}.tp{tp}", plan, HP_T500, _specs(plan, w), seed)
     wl.notes["sigma_g"] = w.sigma_g
+    return wl
+
+
+def config3_mcore(device, tp_send=2, tp_recv=2, dp=1, n_layers=36, seed=1234, dims=P.QWEN3_8B,
+                  target=0.015) -> Workload:
+    """Config 3's state held the way Megatron-Core holds it: fused GQA-interleaved linear_qkv and
+    fused linear_fc1 per sender TP rank, column shards of linear_proj / linear_fc2, and `dp`
+    distributed-optimizer slices per shard (all slices of a shard share one allocation here)."""
+    plan = P.mcore_dense_plan(n_layers, tp_send, tp_recv, True, dims, dp=dp)
+    w = calibrate_sigma_g(WEIGHT, HP_T500, seed, device, target)
+    wl = Workload(f"qwen3-8b.mcore.tp{tp_send}to{tp_recv}.dp{dp}.full{n_layers}", plan, HP_T500,
+                  _specs(plan, w), seed)
+    wl.notes.update(sigma_g=w.sigma_g, operations=len(plan.ops))
+    if dp > 1:
+        wl.alias_of = [(t // dp) * dp for t in range(plan.n_tensors)]
     return wl
 
 

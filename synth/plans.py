@@ -28,6 +28,8 @@ class Plan:
     shard_receivers: List[int] = field(default_factory=list)
     shard_numels: List[int] = field(default_factory=list)
     ops: List[Tuple[int, ...]] = field(default_factory=list)
+    # distributed-optimizer plans: flat element range [lo, hi) each source tensor's owner holds
+    slice_ranges: List[Tuple[int, int]] = field(default_factory=list)
 
     @property
     def n_tensors(self) -> int:
@@ -241,3 +243,169 @@ def scatter_dense(plan: Plan, dense_by_tensor, shards) -> None:
         s2 = s.reshape(plan.tensor_shapes[src])
         view = shards[dst].as_strided((e0, e1), (ld, 1), base + r0 * ld + r1)
         view.copy_(s2[a0:a0 + e0, a1:a1 + e1])
+
+
+# ---- Megatron-Core-native training-side layouts -------------------------------------------------
+#
+# Source tensors in the trainer's own organisation (Appendix B of the paper): per sender TP rank a
+# fused, GQA-interleaved linear_qkv shard [Q_{jg..(j+1)g-1}, K_j, V_j] per kv group j (Eq. 14-16), a
+# fused linear_fc1 shard [gate_s; up_s], column shards of linear_proj / linear_fc2, vocab shards
+# of the embeddings, and - with a distributed optimizer - every such shard cut into `dp`
+# contiguous flat slices, each owned by one data-parallel rank.  The receiver side is unchanged.
+
+def restrict_to_flat_range(op, n1: int, lo: int, hi: int):
+    """The parts of operation `op` whose source elements lie in the flat range [lo, hi) of a
+    row-major source with n1 columns: at most a partial first row, whole middle rows and a
+    partial last row (each a legal operation: whole destination rows or one row)."""
+    src, dst, a0, a1, e0, e1, base, ld, r0, r1 = op
+    out = []
+
+    def emit(row_lo, row_hi, col_lo, col_hi):
+        row_lo, row_hi = max(row_lo, a0), min(row_hi, a0 + e0)
+        col_lo, col_hi = max(col_lo, a1), min(col_hi, a1 + e1)
+        if row_lo >= row_hi or col_lo >= col_hi:
+            return
+        if col_lo == a1 and col_hi == a1 + e1:          # the operation's full width: keep rows together
+            out.append((src, dst, row_lo, a1, row_hi - row_lo, e1, base, ld, r0 + row_lo - a0, r1))
+        else:                                            # partial width: one operation per row
+            for row in range(row_lo, row_hi):
+                out.append((src, dst, row, col_lo, 1, col_hi - col_lo, base, ld, r0 + row - a0,
+                            r1 + col_lo - a1))
+
+    first_full = -(-lo // n1)
+    last_full = hi // n1
+    if first_full > last_full:                           # the range lies inside one row
+        emit(lo // n1, lo // n1 + 1, lo % n1, hi - (lo // n1) * n1)
+        return out
+    if lo % n1:
+        emit(lo // n1, lo // n1 + 1, lo % n1, n1)
+    emit(first_full, last_full, 0, n1)
+    if hi % n1:
+        emit(last_full, last_full + 1, 0, hi % n1)
+    return out
+
+
+def _overlap(lo_a, hi_a, lo_b, hi_b):
+    lo, hi = max(lo_a, lo_b), min(hi_a, hi_b)
+    return (lo, hi) if lo < hi else None
+
+
+def mcore_dense_plan(n_layers: int, tp_send: int, tp_recv: int, with_embeddings: bool,
+                     dims: dict = QWEN3_8B, dp: int = 1, align: int = 4) -> Plan:
+    """Qwen3-dense layers with Megatron-Core-native sources (see above) and the usual receivers.
+
+    Column-split tensors (linear_proj, linear_fc2) map with whole destination rows when the
+    receiver shard lies inside one sender shard (tp_send divides tp_recv); otherwise the
+    builder falls back to one operation per destination row piece.
+    """
+    P_, R = tp_send, tp_recv
+    h, hd, hq, hkv, F = dims["hidden"], dims["head_dim"], dims["q_heads"], dims["kv_heads"], dims["inter"]
+    g = hq // hkv
+    assert hkv % P_ == 0 and hkv % R == 0 and F % P_ == 0 and F % R == 0
+    p = Plan()
+    raw_ops = []       # operations before the data-parallel cut, with the source's column count
+
+    srcs = {}          # (layer, kind, sender) -> tensor index
+    for l in range(n_layers):
+        pre = f"layers.{l}."
+        for s in range(P_):
+            srcs[l, "qkv", s] = p.add_tensor(f"{pre}linear_qkv.tp{s}", ((hq + 2 * hkv) * hd // P_, h))
+            srcs[l, "proj", s] = p.add_tensor(f"{pre}linear_proj.tp{s}", (h, hq * hd // P_))
+            srcs[l, "fc1", s] = p.add_tensor(f"{pre}linear_fc1.tp{s}", (2 * F // P_, h))
+            srcs[l, "fc2", s] = p.add_tensor(f"{pre}linear_fc2.tp{s}", (h, F // P_))
+        for n, shape in (("q_norm", (hd,)), ("k_norm", (hd,)), ("input_layernorm", (h,)),
+                         ("post_attention_layernorm", (h,))):
+            srcs[l, n, 0] = p.add_tensor(pre + n, shape)      # replicated on senders: rank 0's copy is used
+    if with_embeddings:
+        V = dims["vocab"]
+        assert V % P_ == 0 and V % R == 0
+        for s in range(P_):
+            srcs["emb", s] = p.add_tensor(f"embed_tokens.tp{s}", (V // P_, h))
+            srcs["head", s] = p.add_tensor(f"lm_head.tp{s}", (V // P_, h))
+
+    def add(src, dst, a_s, e, base, ld, a_r):
+        raw_ops.append((int(src), int(dst), int(a_s[0]), int(a_s[1]), int(e[0]), int(e[1]), int(base),
+                        int(ld), int(a_r[0]), int(a_r[1])))
+
+    def row_split(dst, dst_row0, dst_cols, kind_key, total_rows, want_lo, want_hi):
+        """Rows [want_lo, want_hi) of a logical [total_rows, cols] tensor whose sender s holds rows
+        [s*total/P, (s+1)*total/P) -> destination rows starting at dst_row0."""
+        per = total_rows // P_
+        for s in range(P_):
+            ov = _overlap(want_lo, want_hi, s * per, (s + 1) * per)
+            if ov:
+                add(srcs[kind_key(s)], dst, (ov[0] - s * per, 0), (ov[1] - ov[0], dst_cols), 0, dst_cols,
+                    (dst_row0 + ov[0] - want_lo, 0))
+
+    def col_split(dst, kind_key, rows, total_cols, want_lo, want_hi):
+        per = total_cols // P_
+        w = want_hi - want_lo
+        for s in range(P_):
+            ov = _overlap(want_lo, want_hi, s * per, (s + 1) * per)
+            if not ov:
+                continue
+            if ov[1] - ov[0] == w:      # whole destination rows
+                add(srcs[kind_key(s)], dst, (0, ov[0] - s * per), (rows, w), 0, w, (0, 0))
+            else:                       # a piece of every destination row: one operation per row
+                for row in range(rows):
+                    add(srcs[kind_key(s)], dst, (row, ov[0] - s * per), (1, ov[1] - ov[0]), 0, w,
+                        (row, ov[0] - want_lo))
+
+    for r in range(R):
+        for l in range(n_layers):
+            pre = f"layers.{l}."
+            # fused qkv_proj by head: kv groups [r*hkv/R, (r+1)*hkv/R)
+            q_rows, kv_rows = hq * hd // R, hkv * hd // R
+            k = p.add_shard(f"r{r}.{pre}qkv_proj", r, (q_rows + 2 * kv_rows) * h)
+            for j in range(r * hkv // R, (r + 1) * hkv // R):
+                s, jl, jr = j // (hkv // P_), j % (hkv // P_), j - r * hkv // R
+                src = srcs[l, "qkv", s]
+                blk = jl * (g + 2) * hd                                   # Eq. 14: [Q x g, K, V] per group
+                add(src, k, (blk, 0), (g * hd, h), 0, h, (jr * g * hd, 0))
+                add(src, k, (blk + g * hd, 0), (hd, h), 0, h, (q_rows + jr * hd, 0))
+                add(src, k, (blk + (g + 1) * hd, 0), (hd, h), 0, h, (q_rows + kv_rows + jr * hd, 0))
+            C = hq * hd
+            k = p.add_shard(f"r{r}.{pre}o_proj", r, h * C // R)
+            col_split(k, lambda s: (l, "proj", s), h, C, r * C // R, (r + 1) * C // R)
+            # fused gate_up_proj: gate rows [r*F/R, ...) then up rows; sender s holds [gate_s; up_s]
+            k = p.add_shard(f"r{r}.{pre}gate_up_proj", r, 2 * F // R * h)
+            per = F // P_
+            for half in range(2):                                         # 0 = gate, 1 = up
+                for s in range(P_):
+                    ov = _overlap(r * F // R, (r + 1) * F // R, s * per, (s + 1) * per)
+                    if ov:
+                        add(srcs[l, "fc1", s], k, (half * per + ov[0] - s * per, 0), (ov[1] - ov[0], h), 0, h,
+                            (half * F // R + ov[0] - r * F // R, 0))
+            k = p.add_shard(f"r{r}.{pre}down_proj", r, h * F // R)
+            col_split(k, lambda s: (l, "fc2", s), h, F, r * F // R, (r + 1) * F // R)
+            for n in ("q_norm", "k_norm", "input_layernorm", "post_attention_layernorm"):
+                src = srcs[l, n, 0]
+                n0 = p.tensor_shapes[src][0]
+                k = p.add_shard(f"r{r}.{pre}{n}", r, n0)
+                add(src, k, (0, 0), (n0, 1), 0, 1, (0, 0))
+        if with_embeddings:
+            V = dims["vocab"]
+            for name, key in (("embed_tokens", "emb"), ("lm_head", "head")):
+                k = p.add_shard(f"r{r}.{name}", r, V // R * h)
+                row_split(k, 0, h, lambda s, key=key: (key, s), V, r * V // R, (r + 1) * V // R)
+
+    if dp == 1:
+        p.ops = raw_ops
+        return p
+    # distributed optimizer: every source tensor is cut into `dp` flat slices (boundaries on
+    # multiples of `align` elements); slice d becomes its own source tensor of the same shape
+    q = Plan(shard_names=p.shard_names, shard_receivers=p.shard_receivers, shard_numels=p.shard_numels)
+    new_index = {}
+    for t, (name, shape) in enumerate(zip(p.tensor_names, p.tensor_shapes)):
+        n = shape[0] * shape[1]
+        cuts = [min(n, -(-(n * d // dp) // align) * align) for d in range(dp)] + [n]
+        for d in range(dp):
+            new_index[t, d] = q.add_tensor(f"{name}.dp{d}", shape)
+            q.slice_ranges.append((cuts[d], cuts[d + 1]))
+    for op in raw_ops:
+        n1 = p.tensor_shapes[op[0]][1]
+        for d in range(dp):
+            lo, hi = q.slice_ranges[new_index[op[0], d]]
+            for piece in restrict_to_flat_range(op, n1, lo, hi):
+                q.ops.append((new_index[op[0], d],) + tuple(piece[1:]))
+    return q
