@@ -256,6 +256,8 @@ def main():
     ap.add_argument("--e2e-gb", type=float, default=10.0, help="host-resident state for the e2e leg (GB)")
     ap.add_argument("--cpu-elements", type=float, default=2.0e9, help="oracle sample size (elements)")
     ap.add_argument("--ref-elements", type=float, default=4e8, help="--impl reference: elements per step")
+    ap.add_argument("--variant", default="mirror", choices=["mirror", "trainer"],
+                    help="association of the generator's forward AdamW step (only changes the inputs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     args = ap.parse_args()
@@ -279,6 +281,7 @@ def main():
 
     t_gen = time.time()
     wl = build_workload(args.workload, device)
+    wl.variant = args.variant
     plan = wl.plan
     st, shards = materialize_resident(wl, device, dte)
     torch.cuda.synchronize()

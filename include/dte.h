@@ -63,7 +63,10 @@ typedef enum dte_status {
 #define DTE_DEV_TIMEOUT 4u  /* reserved (no kernel of this library waits on another CTA)  */
 
 /* Source tensor p of the canonical training-side space: fp32, row-major.  ndim is 1 or 2;
- * for ndim == 1 shape[1] must be 1.  `group` (parameter group) is reserved: must be 0. */
+ * for ndim == 1 shape[1] must be 1.  `group` is the tensor's parameter group (< 65536): the
+ * paper's lambda is a per-group weight-decay coefficient and eta_t a per-group learning rate
+ * (Section 4.1); dte_extract_delta uses one pair for all groups, dte_extract_delta_groups one
+ * pair per group. */
 typedef struct dte_tensor_desc {
     uint64_t shape[2];
     uint32_t ndim;
@@ -120,7 +123,7 @@ typedef struct dte_delta {
 /* Compiles the plan into device tables on `device` (Section 4.2.2: the plan is computed
  * once from shard metadata, before any synchronisation).  Host arrays in, handle out.
  * Allocates the layout's device tables and scratch with cudaMalloc; synchronous.
- * Errors: DTE_ERR_INVALID_ARG (null arrays, ndim, group != 0), DTE_ERR_LAYOUT (operation
+ * Errors: DTE_ERR_INVALID_ARG (null arrays, ndim, group >= 65536), DTE_ERR_LAYOUT (operation
  * outside its tensor or shard, non-contiguous or overlapping destination regions,
  * numel >= 2^32), DTE_ERR_CUDA. */
 DTE_API dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n_tensors,
@@ -132,6 +135,8 @@ DTE_API void dte_layout_destroy(dte_layout* layout);
 
 /* Number of output lists (== n_shards). */
 DTE_API size_t dte_layout_num_lists(const dte_layout* layout);
+/* Number of parameter groups the layout's tensors refer to (largest group index + 1). */
+DTE_API size_t dte_layout_num_groups(const dte_layout* layout);
 /* Elements one extract call scans (sum of extents; replicated tensors count per copy). */
 DTE_API uint64_t dte_layout_num_elements(const dte_layout* layout);
 /* Bytes of device workspace dte_extract_delta_host needs (12 bytes per source element,
@@ -156,6 +161,16 @@ DTE_API dte_status dte_extract_delta(const dte_layout* layout, const float* cons
                              const float* const* m, const float* const* v, int64_t step,
                              double lr, double beta1, double beta2, double eps, double wd,
                              const dte_delta* out, void* cuda_stream);
+
+/* dte_extract_delta with per-parameter-group learning rate and weight decay (Eq. 2: eta_t and
+ * lambda belong to the parameter group of the element).  lr / wd: HOST arrays of n_groups
+ * doubles, n_groups >= dte_layout_num_groups(layout); tensor p uses entry tensors[p].group.
+ * step, beta1, beta2 and eps are shared.  Everything else as dte_extract_delta. */
+DTE_API dte_status dte_extract_delta_groups(const dte_layout* layout, const float* const* theta,
+                                            const float* const* m, const float* const* v, int64_t step,
+                                            double beta1, double beta2, double eps, const double* lr,
+                                            const double* wd, size_t n_groups, const dte_delta* out,
+                                            void* cuda_stream);
 
 /* Allocation-free variant of dte_extract_delta.  The paper has no counterpart: this exists
  * for callers that may not allocate device memory at the point where they extract - a

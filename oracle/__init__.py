@@ -114,7 +114,8 @@ def extract(tensor_shapes, shard_numels, ops, theta, m, v, consts):
     tensor_shapes: [(n0, n1)] per source tensor; shard_numels: [numel] per
     receiver-local tensor; ops: rows of 10 integers {src_tensor, dst_shard,
     a_s0, a_s1, e0, e1, dst_base, dst_ld, a_r0, a_r1}; theta/m/v: lists of
-    fp32 arrays.  Returns (list_ptr uint64[n_shards+1], offsets uint32[M],
+    fp32 arrays; consts: the 5 scalars of derive_constants, or one row of 5
+    per source tensor (per-group learning rate / weight decay).  Returns (list_ptr uint64[n_shards+1], offsets uint32[M],
     values uint16[M]).
     """
     L = lib()
@@ -127,7 +128,11 @@ def extract(tensor_shapes, shard_numels, ops, theta, m, v, consts):
     for p in range(shp.shape[0]):
         n = int(shp[p, 0] * shp[p, 1])
         assert th[p].size == n and mm[p].size == n and vv[p].size == n, "tensor size mismatch"
-    c = _f32(consts)
+    c = np.ascontiguousarray(consts, dtype=np.float32)
+    if c.ndim == 1:                       # one parameter group: the same scalars for every tensor
+        c = np.tile(c.reshape(1, 5), (shp.shape[0], 1))
+    assert c.shape == (shp.shape[0], 5), "consts: 5 scalars, or 5 per source tensor"
+    c = np.ascontiguousarray(c)
     h = L.oracle_extract(shp.shape[0], shp.ctypes.data, num.size, num.ctypes.data, op.shape[0],
                          op.ctypes.data, _ptr_array(th), _ptr_array(mm), _ptr_array(vv),
                          c.ctypes.data)

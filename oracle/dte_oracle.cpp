@@ -142,12 +142,13 @@ uint64_t oracle_changed_mask(const float* theta, const float* m, const float* v,
 // ascending j (the "ordered sparse payload"); a repeated j within one list is
 // a plan error.  Lists are concatenated in shard order; empty lists keep
 // their slot (list_ptr[k] == list_ptr[k+1]).
+// `consts` holds 5 scalars per source tensor (n_tensors x 5): eta_t and lambda of Eq. 2 belong
+// to the element's parameter group, so tensors of different groups carry different scalars.
 void* oracle_extract(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n_shards,
                      const int64_t* shard_numel, uint64_t n_ops, const int64_t* ops,
                      const float* const* theta, const float* const* m, const float* const* v,
-                     const float* c5) {
+                     const float* consts) {
     Result* res = new Result();
-    Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
     std::vector<std::vector<uint64_t>> ops_of(n_tensors);
     for (uint64_t o = 0; o < n_ops; ++o) {
         const int64_t* op = ops + 10 * o;
@@ -162,6 +163,8 @@ void* oracle_extract(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n
         const uint64_t n0 = (uint64_t)tensor_shape[2 * p], n1 = (uint64_t)tensor_shape[2 * p + 1];
         const uint64_t n = n0 * n1;
         if (ops_of[p].empty()) continue;
+        const float* c5 = consts + 5 * p;
+        const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
         for (uint64_t i = 0; i < n; ++i) {
             float prev = invert_one(theta[p][i], m[p][i], v[p][i], c);
             uint16_t bt = bf16_rne(theta[p][i]);

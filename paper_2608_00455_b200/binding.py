@@ -23,7 +23,7 @@ SYMBOLS = [
     "dte_layout_create", "dte_layout_destroy", "dte_layout_num_lists", "dte_layout_num_elements",
     "dte_layout_host_workspace_bytes", "dte_derive_constants", "dte_extract_delta", "dte_apply",
     "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
-    "dte_extract_delta_static",
+    "dte_extract_delta_static", "dte_extract_delta_groups", "dte_layout_num_groups",
 ]
 
 
@@ -82,6 +82,10 @@ def lib() -> C.CDLL:
         L.dte_extract_delta.restype = C.c_int
         L.dte_extract_delta_static.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, vp]
         L.dte_extract_delta_static.restype = C.c_int
+        L.dte_extract_delta_groups.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, vp, vp, C.c_size_t, vp, vp]
+        L.dte_extract_delta_groups.restype = C.c_int
+        L.dte_layout_num_groups.argtypes = [vp]
+        L.dte_layout_num_groups.restype = C.c_size_t
         L.dte_apply.argtypes = [vp, vp, vp, vp]
         L.dte_apply.restype = C.c_int
         L.dte_extract_delta_host.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, u64,
@@ -161,7 +165,7 @@ class Delta:
 class Layout:
     """dte_layout handle built from a plan (tensor shapes, shard sizes, operation rows)."""
 
-    def __init__(self, tensor_shapes, shard_numels, ops, device=0, shard_receivers=None):
+    def __init__(self, tensor_shapes, shard_numels, ops, device=0, shard_receivers=None, tensor_groups=None):
         _require_cuda()
         self.device = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
         shapes = [(int(s[0]), int(s[1]) if len(s) > 1 else 1) for s in tensor_shapes]
@@ -171,7 +175,7 @@ class Layout:
         for i, (a, b) in enumerate(shapes):
             T[i].shape[0], T[i].shape[1] = a, b
             T[i].ndim = 1 if b == 1 else 2
-            T[i].group = 0
+            T[i].group = int(tensor_groups[i]) if tensor_groups is not None else 0
         S = (ShardDesc * max(1, len(self.shard_numels)))()
         for k, n in enumerate(self.shard_numels):
             S[k].numel = n
@@ -190,8 +194,9 @@ class Layout:
         self._h = h
 
     @classmethod
-    def from_plan(cls, plan, device=0):
-        return cls(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), device, plan.shard_receivers)
+    def from_plan(cls, plan, device=0, tensor_groups=None):
+        return cls(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), device, plan.shard_receivers,
+                   tensor_groups)
 
     def close(self):
         if getattr(self, "_h", None):
@@ -207,6 +212,10 @@ class Layout:
     @property
     def num_lists(self) -> int:
         return int(lib().dte_layout_num_lists(self._h))
+
+    @property
+    def num_groups(self) -> int:
+        return int(lib().dte_layout_num_groups(self._h))
 
     @property
     def num_elements(self) -> int:
@@ -254,6 +263,19 @@ def dte_extract_delta(layout: Layout, tables, step, lr, beta1, beta2, eps, wd, d
     _check(lib().dte_extract_delta(layout._h, th, mm, vv, int(step), float(lr), float(beta1),
                                    float(beta2), float(eps), float(wd), C.byref(delta.struct),
                                    _stream_ptr(stream)))
+
+
+def dte_extract_delta_groups(layout: Layout, tables, step, beta1, beta2, eps, lr, wd, delta: Delta,
+                             stream=None) -> None:
+    """Extract with one (lr, wd) pair per parameter group (sequences of equal length)."""
+    th, mm, vv = tables
+    n = len(lr)
+    assert len(wd) == n
+    lr_a = (C.c_double * n)(*[float(x) for x in lr])
+    wd_a = (C.c_double * n)(*[float(x) for x in wd])
+    _check(lib().dte_extract_delta_groups(layout._h, th, mm, vv, int(step), float(beta1), float(beta2),
+                                          float(eps), lr_a, wd_a, n, C.byref(delta.struct),
+                                          _stream_ptr(stream)))
 
 
 STATIC_MAX_TILES = 65536

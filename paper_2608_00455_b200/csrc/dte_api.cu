@@ -75,7 +75,9 @@ Screen make_screen(const Consts& c) {
     return s;
 }
 
-dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out, cudaStream_t st) {
+// `groups`: per-parameter-group constants (NULL: `c` applies to every tensor).
+dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out, cudaStream_t st,
+                           const std::vector<GroupConsts>* groups = nullptr) {
     uint64_t launches = 0;
     DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
     if (L->n_tiles == 0) {
@@ -112,8 +114,23 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
     p.n_tiles = L->n_tiles;
     p.c = c;
     p.s = make_screen(c);
+    p.tensor_group = nullptr;
+    p.groups = nullptr;
+    bool div_bc1 = c.bc1 != 1.0f, div_decay = c.decay != 1.0f;
+    if (groups) {
+        // pageable source: staged by the runtime before the call returns
+        DTE_CUDA(cudaMemcpyAsync(L->d_groups, groups->data(), groups->size() * sizeof(GroupConsts),
+                                 cudaMemcpyHostToDevice, st));
+        p.tensor_group = L->d_tensor_group;
+        p.groups = L->d_groups;
+        div_bc1 = div_decay = false;
+        for (const GroupConsts& g : *groups) {
+            div_bc1 |= g.c.bc1 != 1.0f;
+            div_decay |= g.c.decay != 1.0f;
+        }
+    }
     const int n_ctas = (int)L->n_tiles;   // one CTA per tile
-    dte_status s = launch_extract(p, n_ctas, st);
+    dte_status s = launch_extract(p, div_bc1, div_decay, n_ctas, st);
     if (s != DTE_OK) return s;
     GatherParams g;
     g.rec = L->d_rec;
@@ -159,6 +176,33 @@ extern "C" dte_status dte_extract_delta(const dte_layout* layout, const float* c
     if (s != DTE_OK) return s;
     const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
     return enqueue_extract(L, c, out, st);
+}
+
+extern "C" dte_status dte_extract_delta_groups(const dte_layout* layout, const float* const* theta,
+                                               const float* const* m, const float* const* v,
+                                               int64_t step, double beta1, double beta2, double eps,
+                                               const double* lr, const double* wd, size_t n_groups,
+                                               const dte_delta* out, void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    if (layout->n_tensors && (!theta || !m || !v)) return fail(DTE_ERR_INVALID_ARG, "null pointer table");
+    if (!lr || !wd) return fail(DTE_ERR_INVALID_ARG, "lr / wd array is null");
+    if (n_groups < layout->n_groups) return fail(DTE_ERR_INVALID_ARG, "fewer hyper-parameter groups than the layout's tensors use");
+    dte_status s = check_delta(out);
+    if (s != DTE_OK) return s;
+    std::vector<GroupConsts> groups(layout->n_groups);
+    for (size_t gi = 0; gi < groups.size(); ++gi) {
+        float c5[5];
+        s = dte_derive_constants(step, lr[gi], beta1, beta2, eps, wd[gi], c5);
+        if (s != DTE_OK) return s;
+        groups[gi].c = Consts{c5[0], c5[1], c5[2], c5[3], c5[4]};
+        groups[gi].s = make_screen(groups[gi].c);
+    }
+    dte_layout* L = const_cast<dte_layout*>(layout);
+    DeviceGuard g(L->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    s = sync_source_table(L, theta, m, v, st);
+    if (s != DTE_OK) return s;
+    return enqueue_extract(L, groups[0].c, out, st, &groups);
 }
 
 extern "C" dte_status dte_apply(const dte_layout* layout, const dte_delta* delta,
@@ -350,7 +394,9 @@ extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const f
     p.n_tiles = L->n_tiles;
     p.c = c;
     p.s = make_screen(c);
-    s = launch_extract(p, (int)L->n_tiles, st);
+    p.tensor_group = nullptr;
+    p.groups = nullptr;
+    s = launch_extract(p, c.bc1 != 1.0f, c.decay != 1.0f, (int)L->n_tiles, st);
     if (s != DTE_OK) return s;
     GatherParams gp;
     gp.rec = p.rec;

@@ -111,6 +111,7 @@ struct WarpTile {
     uint32_t len;          // elements of this warp-tile (0 for the unused tail of a short tile)
     uint32_t dst0;         // receiver-local offset of element 0 of this warp-tile
     uint32_t len_flags;
+    uint32_t tensor;
 
     // source element offset of warp-tile element e
     __device__ __forceinline__ uint64_t src(uint32_t e) const {
@@ -130,6 +131,7 @@ __device__ __forceinline__ void decode(const ExtractParams& p, uint32_t t, WarpT
     wt.len_flags = d1.x;
     wt.len = tile_len > e0 ? min(tile_len - e0, (uint32_t)kWarpTile) : 0u;
     wt.dst0 = d0.w + e0;
+    wt.tensor = d0.z;
     wt.th = ldg_ptr(p.theta + d0.z);
     wt.mm = ldg_ptr(p.m + d0.z);
     wt.vv = ldg_ptr(p.v + d0.z);
@@ -178,7 +180,8 @@ __device__ __forceinline__ void load_chunk(const WarpTile& wt, uint32_t cb, int 
     }
 }
 
-template <bool DIV_BC1, bool DIV_DECAY>
+// GROUPS: the constants come from the tile's parameter group instead of the kernel parameters.
+template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS>
 __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const ExtractParams p) {
     // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
     __shared__ uint32_t s_queue[kWarps][kWarpTile];
@@ -186,8 +189,8 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
     __shared__ unsigned long long s_pos;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* queue = s_queue[warp];
-    const Consts c = p.c;
-    const Screen sc = p.s;
+    Consts c = p.c;
+    Screen sc = p.s;
     const uint32_t lanemask_lt = (1u << lane) - 1u;
     static_assert(kSub == kWarps, "one warp per warp-tile");
 
@@ -196,6 +199,13 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
     {
         const uint32_t t = blockIdx.x * kSub + warp;
         decode(p, t, cur);
+        if (GROUPS) {   // one 32-byte record, the same for the whole CTA
+            const uint4* gp = reinterpret_cast<const uint4*>(p.groups + __ldg(p.tensor_group + cur.tensor));
+            const uint4 g0 = __ldg(gp), g1 = __ldg(gp + 1);
+            c.bc1 = __uint_as_float(g0.x); c.bc2 = __uint_as_float(g0.y); c.decay = __uint_as_float(g0.z);
+            c.lr = __uint_as_float(g0.w); c.eps = __uint_as_float(g1.x);
+            sc.k1 = __uint_as_float(g1.y); sc.k2 = __uint_as_float(g1.z); sc.kappa = __uint_as_float(g1.w);
+        }
 
         // ---- phase A: stream, screen, queue the undecided elements in element order ---------
         uint32_t qn = 0;
@@ -298,9 +308,9 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
     }
 }
 
-template <bool A, bool B>
+template <bool A, bool B, bool G>
 static dte_status launch_t(const ExtractParams& p, int n_ctas, cudaStream_t st) {
-    extract_kernel<A, B><<<n_ctas, kThreads, 0, st>>>(p);
+    extract_kernel<A, B, G><<<n_ctas, kThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }
@@ -312,13 +322,19 @@ extern "C" __attribute__((visibility("default"))) void dte_debug_stats(unsigned 
 }
 #endif
 
-dte_status launch_extract(const ExtractParams& p, int n_ctas, cudaStream_t st) {
-    const bool a = p.c.bc1 != 1.0f, b = p.c.decay != 1.0f;
-    if (a && b) return launch_t<true, true>(p, n_ctas, st);
-    if (a) return launch_t<true, false>(p, n_ctas, st);
-    if (b) return launch_t<false, true>(p, n_ctas, st);
-    return launch_t<false, false>(p, n_ctas, st);
+// div_bc1 / div_decay: whether any group in the call has a divisor different from 1.0f.
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, int n_ctas, cudaStream_t st) {
+    const bool a = div_bc1, b = div_decay;
+    if (p.groups) {
+        if (a && b) return launch_t<true, true, true>(p, n_ctas, st);
+        if (a) return launch_t<true, false, true>(p, n_ctas, st);
+        if (b) return launch_t<false, true, true>(p, n_ctas, st);
+        return launch_t<false, false, true>(p, n_ctas, st);
+    }
+    if (a && b) return launch_t<true, true, false>(p, n_ctas, st);
+    if (a) return launch_t<true, false, false>(p, n_ctas, st);
+    if (b) return launch_t<false, true, false>(p, n_ctas, st);
+    return launch_t<false, false, false>(p, n_ctas, st);
 }
-
 
 }  // namespace dte

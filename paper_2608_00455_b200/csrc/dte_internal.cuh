@@ -70,6 +70,13 @@ struct Screen {
     float k1, k2, kappa;
 };
 
+// Per-parameter-group constants, one 32-byte record (exact path + screen).
+struct __align__(32) GroupConsts {
+    Consts c;
+    Screen s;
+};
+static_assert(sizeof(GroupConsts) == 32, "GroupConsts must be one 32-byte sector");
+
 struct ExtractParams {
     const TileDesc* tiles;
     const SegRec* segs;
@@ -82,8 +89,10 @@ struct ExtractParams {
     uint16_t* stage_values;
     uint64_t stage_capacity;
     uint32_t n_tiles;
-    Consts c;
+    Consts c;                    // single-group calls: constants in the kernel parameters
     Screen s;
+    const uint32_t* tensor_group;   // per-group calls: group of each source tensor ...
+    const GroupConsts* groups;      // ... and the constants of each group (NULL otherwise)
 };
 
 struct GatherParams {
@@ -122,7 +131,7 @@ dte_status cuda_fail(cudaError_t e, const char* what);
         if (e__ != cudaSuccess) return dte::cuda_fail(e__, #call); \
     } while (0)
 
-dte_status launch_extract(const ExtractParams& p, int n_ctas, cudaStream_t st);
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, int n_ctas, cudaStream_t st);
 dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 
@@ -149,6 +158,9 @@ struct dte_layout {
     uint16_t** d_shards = nullptr;         // n_lists
     uint64_t* d_shard_numel = nullptr;     // n_lists
     uint32_t* d_list_first_rec = nullptr;  // n_lists
+    uint32_t* d_tensor_group = nullptr;    // n_tensors
+    dte::GroupConsts* d_groups = nullptr;  // n_groups
+    uint32_t n_groups = 1;
     // host mirrors of the pointer tables last uploaded
     std::vector<const float*> h_ptrs;
     std::vector<uint16_t*> h_shards;

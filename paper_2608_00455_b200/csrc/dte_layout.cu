@@ -90,12 +90,15 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
     cudaFree((void*)L->d_shards);
     cudaFree(L->d_shard_numel);
     cudaFree(L->d_list_first_rec);
+    cudaFree(L->d_tensor_group);
+    cudaFree(L->d_groups);
     if (prev >= 0) cudaSetDevice(prev);
     delete L;
 }
 
 extern "C" size_t dte_layout_num_lists(const dte_layout* L) { return L ? L->n_lists : 0; }
 extern "C" uint64_t dte_layout_num_elements(const dte_layout* L) { return L ? L->scanned : 0; }
+extern "C" size_t dte_layout_num_groups(const dte_layout* L) { return L ? L->n_groups : 0; }
 
 extern "C" uint64_t dte_layout_host_workspace_bytes(const dte_layout* L) {
     if (!L) return 0;
@@ -134,7 +137,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         const dte_tensor_desc& t = tensors[p];
         if (t.ndim != 1 && t.ndim != 2) return fail(DTE_ERR_INVALID_ARG, "tensor ndim must be 1 or 2");
         if (t.ndim == 1 && t.shape[1] != 1) return fail(DTE_ERR_INVALID_ARG, "1-D tensor needs shape[1] == 1");
-        if (t.group != 0) return fail(DTE_ERR_INVALID_ARG, "parameter groups are reserved: group must be 0");
+        if (t.group >= 65536) return fail(DTE_ERR_INVALID_ARG, "parameter group index must be < 65536");
         if (t.shape[1] != 0 && t.shape[0] > (uint64_t(1) << 62) / t.shape[1])
             return fail(DTE_ERR_LAYOUT, "tensor too large");
         numel[p] = t.shape[0] * t.shape[1];
@@ -285,12 +288,21 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     guard(upload(&L->d_segs, segs));
     guard(upload(&L->d_shard_numel, L->shard_numel));
     guard(upload(&L->d_list_first_rec, first_rec));
+    {
+        std::vector<uint32_t> grp(n_tensors);
+        for (size_t p = 0; p < n_tensors; ++p) {
+            grp[p] = tensors[p].group;
+            L->n_groups = std::max(L->n_groups, tensors[p].group + 1);
+        }
+        guard(upload(&L->d_tensor_group, grp));
+    }
     if (st == DTE_OK) {
         const size_t n_rec = tiles.size();
         const size_t n_blocks = (n_rec + kRecsPerBlock - 1) / kRecsPerBlock;
         cudaError_t e = cudaMalloc((void**)&L->d_rec, std::max<size_t>(1, n_rec) * sizeof(uint64_t));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_block_sum, std::max<size_t>(1, n_blocks) * sizeof(uint64_t));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_cursor, sizeof(uint64_t));
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_groups, L->n_groups * sizeof(GroupConsts));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_ptrs, std::max<size_t>(1, 3 * n_tensors) * sizeof(void*));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_shards, std::max<size_t>(1, n_shards) * sizeof(void*));
         if (e != cudaSuccess) st = cuda_fail(e, "cudaMalloc(layout scratch)");

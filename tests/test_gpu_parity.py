@@ -275,3 +275,34 @@ def test_offsets_up_to_the_uint32_limit():
     assert int(shard[:base][-1000000:].abs().sum()) == 0
     del shard
     torch.cuda.empty_cache()
+
+
+def test_parameter_groups_lr_and_weight_decay_per_group():
+    # group 0: weights (lr, wd); group 1: norms (smaller lr, no weight decay); group 2: embeddings
+    plan = plans.qwen3_dense_plan(2, 4, True, configs.SMALL_DENSE)
+    groups = [1 if "norm" in n else (2 if n in ("embed_tokens", "lm_head") else 0) for n in plan.tensor_names]
+    lr, wd = [1e-4, 3e-5, 5e-5], [0.1, 0.0, 0.3]
+    step, b1, b2, eps = 50, 0.9, 0.999, 1e-8
+    wl = configs.Workload("groups", plan, Hyper(step=step, lr=lr[0], wd=wd[0]), configs._specs(plan), 41)
+    st = wl.materialize("cuda")
+    lay = dte.Layout.from_plan(plan, 0, tensor_groups=groups)
+    assert lay.num_groups == 3
+    d = lay.new_delta(lay.num_elements)
+    tabs = lay.source_tables(st.theta, st.m, st.v)
+    dte.dte_extract_delta_groups(lay, tabs, step, b1, b2, eps, lr, wd, d)
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    consts = np.stack([oracle.derive_constants(step, lr[g], b1, b2, eps, wd[g]) for g in groups])
+    host = lambda lst: [x.cpu().numpy() for x in lst]
+    want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), host(st.theta), host(st.m),
+                          host(st.v), consts)
+    assert_lists_equal(d.to_host(), want, plan)
+    # the single-pair call on the same layout applies one pair to every group
+    dte.dte_extract_delta(lay, tabs, step, lr[0], b1, b2, eps, wd[0], d)
+    torch.cuda.synchronize()
+    one = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), host(st.theta), host(st.m),
+                         host(st.v), oracle.derive_constants(step, lr[0], b1, b2, eps, wd[0]))
+    assert_lists_equal(d.to_host(), one, plan)
+    assert int(one[0][-1]) != int(want[0][-1])
+    with pytest.raises(dte.DteError):            # fewer pairs than groups
+        dte.dte_extract_delta_groups(lay, tabs, step, b1, b2, eps, lr[:2], wd[:2], d)

@@ -250,3 +250,29 @@ def test_plan_errors_are_reported():
     ops[0, 6] = 40         # pushes the block past the end of the shard
     with pytest.raises(ValueError):
         oracle.extract(plan.tensor_shapes, plan.shard_numels, ops, th, mm, vv, c)
+
+
+def test_per_tensor_constants_equal_one_tensor_at_a_time():
+    """Parameter groups (Section 4.1: lambda and eta_t belong to the element's group): the
+    extract with one row of constants per tensor equals separate single-group extracts of
+    each tensor's operations, list by list."""
+    plan = plans.qwen3_dense_plan(1, 2, False, configs.SMALL_DENSE)
+    wl, st, _, th, mm, vv = _random_sparse_case(plan, 6, lr=1e-4)
+    rows = []
+    for p, name in enumerate(plan.tensor_names):
+        norm = "norm" in name
+        rows.append(oracle.derive_constants(100, 3e-5 if norm else 1e-4, 0.9, 0.999, 1e-8, 0.0 if norm else 0.1))
+    consts = np.stack(rows)
+    assert consts[0, 2] != 1.0 and consts[-1, 2] == 1.0
+    lp, off, val = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), th, mm, vv, consts)
+    merged = [[] for _ in range(plan.n_shards)]
+    ops = plan.ops_array()
+    for p in range(plan.n_tensors):
+        sub = ops[ops[:, 0] == p]
+        l1, o1, v1 = oracle.extract(plan.tensor_shapes, plan.shard_numels, sub, th, mm, vv, consts[p])
+        for k in range(plan.n_shards):
+            merged[k] += list(zip(o1[int(l1[k]):int(l1[k + 1])], v1[int(l1[k]):int(l1[k + 1])]))
+    for k in range(plan.n_shards):
+        got = list(zip(off[int(lp[k]):int(lp[k + 1])], val[int(lp[k]):int(lp[k + 1])]))
+        assert got == sorted(merged[k])
+    assert int(lp[-1]) > 1000
