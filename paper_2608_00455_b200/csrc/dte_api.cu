@@ -53,10 +53,11 @@ dte_status sync_source_table(dte_layout* L, const float* const* theta, const flo
     return DTE_OK;
 }
 
-// Constants of the kernel's conservative screen, each rounded up and inflated by 2^-10:
-//   k1    >= lr * sqrt(bc2) / bc1        (bound on |lr*u| is |m| * k1 * rsqrt(v))
-//   k2    >= lr / (bc1 * eps)            (.. and |m| * k2; +inf when eps == 0)
-//   kappa >= (|1/decay - 1| + 2^-24) * (1 + 2^-7)
+// Constants of the kernel's conservative screen (see dte_extract.cu), each rounded up:
+//   ka    >= 1 / bc1
+//   kb    >= sqrt(bc2) * (1 + 2^-10)
+//   kc    >= 1 / eps                      (+inf when eps == 0)
+//   kappa >= (|1/decay - 1| + 2^-24) * (1 + 2^-7) * (1 + 2^-10)
 float round_up(double x) {
     if (!(x == x)) return std::numeric_limits<float>::infinity();
     float f = (float)x;
@@ -66,11 +67,10 @@ float round_up(double x) {
 
 Screen make_screen(const Consts& c) {
     const double infl = 1.0 + 1.0 / 1024.0;
-    const double lr = std::fabs((double)c.lr);
     Screen s;
-    s.k1 = round_up(lr * std::sqrt((double)c.bc2) / (double)c.bc1 * infl);
-    s.k2 = c.eps > 0.f ? round_up(lr / ((double)c.bc1 * (double)c.eps) * infl)
-                       : std::numeric_limits<float>::infinity();
+    s.ka = round_up(1.0 / (double)c.bc1);
+    s.kb = round_up(std::sqrt((double)c.bc2) * infl);
+    s.kc = c.eps > 0.f ? round_up(1.0 / (double)c.eps) : std::numeric_limits<float>::infinity();
     s.kappa = round_up((std::fabs(1.0 / (double)c.decay - 1.0) + std::ldexp(1.0, -24)) * (1.0 + 1.0 / 128.0) * infl);
     return s;
 }
@@ -196,6 +196,7 @@ extern "C" dte_status dte_extract_delta_groups(const dte_layout* layout, const f
         if (s != DTE_OK) return s;
         groups[gi].c = Consts{c5[0], c5[1], c5[2], c5[3], c5[4]};
         groups[gi].s = make_screen(groups[gi].c);
+        groups[gi].pad[0] = groups[gi].pad[1] = groups[gi].pad[2] = 0.f;
     }
     dte_layout* L = const_cast<dte_layout*>(layout);
     DeviceGuard g(L->device);

@@ -57,21 +57,31 @@ __device__ __forceinline__ uint32_t bf16_rne_bits(float x) {
 // ---- the screen --------------------------------------------------------------------
 //
 // Let a = |theta|, c = the BF16 value nearest to a, and lo < a < hi the two rounding
-// boundaries (tie points) around c, as fp32 numbers.  With lo' = succ(lo), hi' = pred(hi):
-// any real x in [lo', hi'] rounds (in fp32, then in BF16) to c, because rounding is
-// monotone and lo', hi' are fp32 numbers strictly inside (lo, hi).  So if
-//     B >= |x - theta|  and  B <= min(hi' - a, a - lo')          (*)
-// where x is the exact quotient whose rounding is the reconstruction, the reconstruction
-// has the same BF16 pattern as theta: unchanged, no exact evaluation needed.
+// boundaries (tie points) around c, as fp32 numbers.  Any real x with lo < x < hi rounds (in
+// fp32, then in BF16) to c, because rounding is monotone.  The screen proves that the exact
+// quotient whose rounding is the reconstruction lies in [lo'', hi''] = [lo + 2 ulp, hi - 2 ulp]
+// (ulp = fp32 spacing at the boundary), hence the reconstruction has the BF16 pattern of
+// theta: unchanged, no exact evaluation needed.
 //
-// B: every intermediate of Eq. 2 carries a relative rounding error <= 2^-24, so
-//     |lr*u| <= |m| * min( lr*sqrt(bc2)/bc1 * rsqrt(v),  lr/(bc1*eps) ) * (1 + 2^-20),
-// and dividing by decay moves the value by at most |num| * |1/decay - 1|, |num| <= a(1+2^-7).
-// The host passes k1, k2, kappa rounded up and inflated by 2^-10, which covers the fp32
-// evaluation of B itself and the 2^-22 error of the hardware rsqrt.  rsqrt flushes
-// subnormal v to zero, which only enlarges B.  NaN anywhere makes (*) false (min.NaN and an
-// ordered compare), so NaN / Inf / negative v / zero theta all fall through to the exact
-// path.  hi' - a and a - lo' are exact (the operands are within a factor 2 of each other).
+// The bound mirrors Eq. 2 operation by operation and leans on the monotonicity of
+// round-to-nearest: if real x <= real y then RN(x) <= RN(y), overflow and underflow included.
+//     exact                      bound (all operands non-negative)
+//     mhat = RN(m / bc1)         A = RN(|m| * ka),        ka >= 1/bc1          => A >= |mhat|
+//     den  = RN(RN(sqrt(RN(v/bc2))) + eps)
+//                                W = min(|rsqrt(v)| * kb, kc),  kb >= sqrt(bc2)(1+2^-10),
+//                                    kc >= 1/eps                               => W >= 1/den
+//     u    = RN(mhat / den)      U = RN(A * W)                                 => U >= |u|
+//     s    = RN(lr * u)          S = RN(U * |lr|)                              => S >= |s|
+// so theta + s lies within S of theta, and num = RN(theta + s) stays in any fp32 interval
+// that contains [a - S, a + S].  For decay != 1, num/decay differs from theta by at most
+// S + a(1+2^-7)(|1/decay - 1| + 2^-24) <= B = fma(a, kappa, S) up to B's own rounding, which
+// is below one ulp and is absorbed by the second ulp of margin; the first ulp of margin
+// absorbs sub-ulp absolute errors in the subnormal range.  2^-10 in kb covers the 2^-22 error
+// of the hardware rsqrt and the rounding of RN(v/bc2), sqrt and the product.  rsqrt.ftz turns
+// subnormal v into +Inf, so W = kc there (den >= eps always); a negative subnormal v (whose
+// exact square root is NaN) becomes -0, then -Inf, and |B| = Inf.  NaN, Inf, negative v, zero
+// theta, an intermediate that overflows: all make B NaN / Inf or the room NaN (min.NaN and an
+// ordered compare), so those elements fall through to the exact path.
 __device__ __forceinline__ float min_nan(float x, float y) {
     float r;
     asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(x), "f"(y));
@@ -83,16 +93,18 @@ __device__ __forceinline__ float rsqrt_ftz(float x) {
     return r;
 }
 
-template <bool DIV_DECAY>
-__device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s) {
+template <bool DIV_BC1, bool DIV_DECAY>
+__device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s, float abs_lr) {
     const uint32_t a = __float_as_uint(theta) & 0x7FFFFFFFu;
-    const uint32_t hi = ((a + 0x8000u) & 0xFFFF0000u) | 0x7FFFu;
-    const uint32_t lo = hi - 0xFFFEu;
+    const uint32_t hi = ((a + 0x8000u) & 0xFFFF0000u) | 0x7FFEu;   // boundary above, minus 2 ulp
+    const uint32_t lo = hi - 0xFFFCu;                               // boundary below, plus 2 ulp
     const float at = __uint_as_float(a);
-    const float room = min_nan(__uint_as_float(hi) - at, at - __uint_as_float(lo));
-    float b = fabsf(m) * min_nan(fabsf(rsqrt_ftz(v)) * s.k1, s.k2);
+    const float room = min_nan(__uint_as_float(hi) - at, at - __uint_as_float(lo));   // exact differences
+    const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
+    const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);   // -Inf for v = -0 or a negative subnormal
+    float b = __fmul_rn(__fmul_rn(am, w), abs_lr);
     if (DIV_DECAY) b = __fmaf_rn(at, s.kappa, b);
-    return b <= room;
+    return fabsf(b) <= room;            // |b|: a negative v (w = -Inf or NaN) must not pass
 }
 
 __device__ __forceinline__ const float* ldg_ptr(const float* const* slot) {
@@ -199,13 +211,15 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
     {
         const uint32_t t = blockIdx.x * kSub + warp;
         decode(p, t, cur);
-        if (GROUPS) {   // one 32-byte record, the same for the whole CTA
+        if (GROUPS) {   // one 48-byte record, the same for the whole CTA
             const uint4* gp = reinterpret_cast<const uint4*>(p.groups + __ldg(p.tensor_group + cur.tensor));
-            const uint4 g0 = __ldg(gp), g1 = __ldg(gp + 1);
+            const uint4 g0 = __ldg(gp), g1 = __ldg(gp + 1), g2 = __ldg(gp + 2);
             c.bc1 = __uint_as_float(g0.x); c.bc2 = __uint_as_float(g0.y); c.decay = __uint_as_float(g0.z);
             c.lr = __uint_as_float(g0.w); c.eps = __uint_as_float(g1.x);
-            sc.k1 = __uint_as_float(g1.y); sc.k2 = __uint_as_float(g1.z); sc.kappa = __uint_as_float(g1.w);
+            sc.ka = __uint_as_float(g1.y); sc.kb = __uint_as_float(g1.z); sc.kc = __uint_as_float(g1.w);
+            sc.kappa = __uint_as_float(g2.x);
         }
+        const float abs_lr = fabsf(c.lr);
 
         // ---- phase A: stream, screen, queue the undecided elements in element order ---------
         uint32_t qn = 0;
@@ -224,7 +238,7 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
                     const float v4[4] = {g[i].x, g[i].y, g[i].z, g[i].w};
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
-                        if (!surely_unchanged<DIV_DECAY>(tt[j], m4[j], v4[j], sc)) amb[i] |= 1u << j;
+                        if (!surely_unchanged<DIV_BC1, DIV_DECAY>(tt[j], m4[j], v4[j], sc, abs_lr)) amb[i] |= 1u << j;
                     amb[i] &= (1u << min(cur.len - e, 4u)) - 1u;      // ragged tail of a scalar tile
                 }
                 cnt |= __popc(amb[i]) << (8 * i);

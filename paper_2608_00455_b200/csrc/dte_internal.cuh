@@ -67,15 +67,16 @@ struct Consts {
 
 // Constants of the conservative "cannot have changed" screen (see dte_extract.cu).
 struct Screen {
-    float k1, k2, kappa;
+    float ka, kb, kc, kappa;
 };
 
-// Per-parameter-group constants, one 32-byte record (exact path + screen).
-struct __align__(32) GroupConsts {
+// Per-parameter-group constants (exact path + screen), read with three 16-byte loads.
+struct __align__(16) GroupConsts {
     Consts c;
     Screen s;
+    float pad[3];
 };
-static_assert(sizeof(GroupConsts) == 32, "GroupConsts must be one 32-byte sector");
+static_assert(sizeof(GroupConsts) == 48, "GroupConsts is read as three uint4");
 
 struct ExtractParams {
     const TileDesc* tiles;

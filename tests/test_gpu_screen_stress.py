@@ -66,3 +66,44 @@ def test_screen_threshold_cases_match_oracle(hp):
     assert np.array_equal(val, want[2])
     frac = int(lp[-1]) / n
     assert 0.05 < frac < 0.95, frac            # the cases really straddle the decision
+
+
+@pytest.mark.parametrize("hp", [
+    Hyper(step=500, lr=1e-6, wd=0.01),                 # no division by bc1 or decay
+    Hyper(step=3, lr=1e-3, wd=0.2),                    # both
+    Hyper(step=100, lr=1e-6, wd=0.01),                 # bc1 only
+    Hyper(step=500, lr=1e-4, wd=0.1),                  # decay only
+    Hyper(step=7, lr=1e-3, wd=0.0, eps=0.0),           # eps == 0
+    Hyper(step=20, lr=0.5, wd=1.5),                    # decay = 0.25
+    Hyper(step=20, lr=-1e-3, wd=0.5),                  # negative learning rate, decay > 1
+    Hyper(step=2, lr=1e-2, wd=0.01, beta1=0.0, beta2=0.5, eps=1e-30),
+], ids=lambda h: f"t{h.step}-lr{h.lr:g}-wd{h.wd:g}-eps{h.eps:g}")
+def test_random_bit_patterns_match_oracle(hp):
+    """theta, m, v drawn as raw 32-bit patterns: every exponent, subnormals, Inf, NaN, negative
+    second moments.  Nothing here is a plausible optimizer state; the point is that the screen
+    never clears an element whose exact evaluation would differ."""
+    rows, cols = 2048, 4096
+    n = rows * cols
+    rng = np.random.default_rng(99 + hp.step)
+    theta = rng.integers(0, 1 << 32, size=n, dtype=np.uint64).astype(np.uint32).view(np.float32)
+    m = rng.integers(0, 1 << 32, size=n, dtype=np.uint64).astype(np.uint32).view(np.float32)
+    vb = rng.integers(0, 1 << 32, size=n, dtype=np.uint64).astype(np.uint32)
+    vb[: n // 2] &= 0x7FFFFFFF                        # half of the second moments non-negative
+    v = vb.view(np.float32)
+    # a band of moderate magnitudes so that part of the data takes the screened path at all
+    k = n // 4
+    theta[:k] = (rng.standard_normal(k) * 0.02).astype(np.float32)
+    m[:k] = (rng.standard_normal(k) * 10.0 ** rng.uniform(-12, 2, k)).astype(np.float32)
+    v[:k] = np.abs(rng.standard_normal(k) * 10.0 ** rng.uniform(-20, 2, k)).astype(np.float32)
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    c = oracle.derive_constants(*hp.as_args())
+    with np.errstate(all="ignore"):
+        want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), [theta], [m], [v], c)
+    lay = dte.Layout.from_plan(plan, 0)
+    d = lay.new_delta(n)
+    t, mm, vv = (torch.from_numpy(a.copy()).cuda() for a in (theta, m, v))
+    dte.dte_extract_delta(lay, lay.source_tables([t], [mm], [vv]), *hp.as_args(), d)
+    torch.cuda.synchronize()
+    lp, off, val = d.to_host()
+    assert np.array_equal(lp, want[0]) and np.array_equal(off, want[1]) and np.array_equal(val, want[2])
+    assert 0.3 < int(lp[-1]) / n <= 1.0
