@@ -21,8 +21,8 @@ constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kItems = 4;                              // float4 loads per thread, array and chunk
 constexpr int kChunk = 32 * 4 * kItems;                // elements a warp loads at once: 512
-constexpr int kChunksPerWarpTile = 2;
-constexpr int kWarpTile = kChunk * kChunksPerWarpTile; // 1024
+constexpr int kWarpTile = 1024;
+static_assert(kWarpTile % kChunk == 0, "whole chunks per warp-tile");
 constexpr int kSub = 8;                                // warp-tiles per tile
 constexpr int kTile = kSub * kWarpTile;                // 8192 elements
 constexpr uint32_t kNone = 0xFFFFFFFFu;
