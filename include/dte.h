@@ -25,7 +25,7 @@
  *     device can detect are reported as DTE_DEV_* bits in dte_delta.counters[2].
  *   - A layout may be used by one extract or apply call at a time (its scratch memory
  *     is per layout).  Different layouts are independent.
- *   - Scratch: the layout owns its device tables, one 8-byte placement record per 8192
+ *   - Scratch: the layout owns its device tables, one 8-byte placement record per 9216
  *     scanned elements, and a staging buffer of `capacity` (offset, value) pairs.  The
  *     staging buffer is allocated by the first extract call and re-allocated (with a stream
  *     synchronisation) only when a later call passes a larger capacity.
@@ -182,8 +182,8 @@ DTE_API dte_status dte_extract_delta_groups(const dte_layout* layout, const floa
  * staging buffer live in one fixed array inside the library's device image (about 12.5 MiB;
  * every GPU that loads the library holds it until the process exits), and it calls no
  * cudaMalloc, cudaFree or other device-allocating routine.
- *   Limits: the layout may have at most DTE_STATIC_MAX_TILES tiles (a tile is up to 8192
- * consecutive destination slots of one operation, so up to 536,870,912 scanned elements when
+ *   Limits: the layout may have at most DTE_STATIC_MAX_TILES tiles (a tile is up to 9216
+ * consecutive destination slots of one operation, so up to 603,979,776 scanned elements when
  * the tiles are full) and out->capacity at most DTE_STATIC_MAX_CAPACITY entries.  Larger
  * requests return DTE_ERR_CAPACITY with the numbers in dte_last_error(); nothing is enqueued.
  *   The first call on a device looks up the array's address on that device (a host-side

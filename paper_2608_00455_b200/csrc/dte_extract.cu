@@ -22,7 +22,7 @@
 namespace dte {
 
 #ifndef DTE_MIN_CTAS
-#define DTE_MIN_CTAS 3
+#define DTE_MIN_CTAS 4
 #endif
 
 #ifdef DTE_STATS
@@ -198,11 +198,12 @@ __device__ __forceinline__ void load_chunk(const WarpTile& wt, uint32_t cb, int 
 template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS>
 __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const ExtractParams p) {
     // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
-    __shared__ uint32_t s_queue[kWarps][kWarpTile];
+    // (dynamic shared memory: kWarps * kWarpTile words, may exceed the 48 KB static limit)
+    extern __shared__ __align__(16) uint32_t s_queue[];
     __shared__ uint32_t s_count[kWarps];
     __shared__ unsigned long long s_pos;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    uint32_t* queue = s_queue[warp];
+    uint32_t* queue = s_queue + warp * kWarpTile;
     Consts c = p.c;
     Screen sc = p.s;
     const uint32_t lanemask_lt = (1u << lane) - 1u;
@@ -324,9 +325,19 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
     }
 }
 
+constexpr size_t kQueueBytes = (size_t)kWarps * kWarpTile * sizeof(uint32_t);
+
 template <bool A, bool B, bool G>
 static dte_status launch_t(const ExtractParams& p, int n_ctas, cudaStream_t st) {
-    extract_kernel<A, B, G><<<n_ctas, kThreads, 0, st>>>(p);
+    static bool configured[64] = {false};     // per device: allow more than 48 KB of dynamic shared memory
+    int dev = 0;
+    DTE_CUDA(cudaGetDevice(&dev));
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        DTE_CUDA(cudaFuncSetAttribute(extract_kernel<A, B, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      (int)kQueueBytes));
+        configured[dev] = true;
+    }
+    extract_kernel<A, B, G><<<n_ctas, kThreads, kQueueBytes, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }

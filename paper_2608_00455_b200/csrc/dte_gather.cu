@@ -2,7 +2,7 @@
 // per-tile placement records gives every tile its position in the concatenated,
 // list-ordered output (lists in shard order, ascending offsets within a list), and a gather
 // moves its entries from the staging buffer to that position.  Three small launches; the
-// data they touch are the records (8 bytes per 8192 scanned elements) and the changed
+// data they touch are the records (8 bytes per 9216 scanned elements) and the changed
 // entries themselves.  No kernel waits on another CTA.
 #include "dte_internal.cuh"
 
