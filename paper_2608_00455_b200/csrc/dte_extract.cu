@@ -242,7 +242,8 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
 #pragma unroll
                     for (int j = 0; j < 4; ++j)
                         if (!surely_unchanged<DIV_BC1, DIV_DECAY>(tt[j], m4[j], v4[j], sc, abs_lr)) amb[i] |= 1u << j;
-                    amb[i] &= (1u << min(cur.len - e, 4u)) - 1u;      // ragged tail of a scalar tile
+                    if (cur.len_flags & kFlagScalar)                  // ragged tail of a scalar tile
+                        amb[i] &= (1u << min(cur.len - e, 4u)) - 1u;
                 }
                 cnt |= __popc(amb[i]) << (8 * i);
             }
