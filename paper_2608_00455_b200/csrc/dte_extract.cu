@@ -277,23 +277,39 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
         // ---- phase B: exact evaluation of the queue, 32 entries per round; the changed
         //      entries are compacted to the front of the queue as (index | value << 16) -----
         uint32_t n_changed = 0;
+        // the loads of round r + 1 are issued before round r is evaluated (their latency is an
+        // L2 hit, several hundred ns, and rounds are otherwise serial)
+        uint32_t e_cur = 0;
+        float tj = 0.f, mj = 0.f, vj = 0.f;
+        if ((uint32_t)lane < qn) {
+            e_cur = queue[lane];
+            const uint64_t so = cur.src(e_cur);
+            tj = __ldg(cur.th + so); mj = __ldg(cur.mm + so); vj = __ldg(cur.vv + so);
+        }
 #pragma unroll 1
         for (uint32_t q0 = 0; q0 < qn; q0 += 32) {
-            const uint32_t q = q0 + lane;
+            const uint32_t q = q0 + lane, qnext = q + 32;
+            uint32_t e_nxt = 0;
+            float tn = 0.f, mn = 0.f, vn = 0.f;
+            if (qnext < qn) {
+                e_nxt = queue[qnext];
+                const uint64_t so = cur.src(e_nxt);
+                tn = __ldg(cur.th + so); mn = __ldg(cur.mm + so); vn = __ldg(cur.vv + so);
+            }
             bool changed = false;
             uint32_t entry = 0;
             if (q < qn) {
-                const uint32_t e = queue[q];
-                const uint64_t so = cur.src(e);
-                const float tj = __ldg(cur.th + so), mj = __ldg(cur.mm + so), vj = __ldg(cur.vv + so);
                 const float prev = invert_adamw<DIV_BC1, DIV_DECAY>(tj, mj, vj, c);
                 const uint32_t bt = bf16_rne_bits(tj), bp = bf16_rne_bits(prev);
                 changed = bt != bp;
-                entry = e | (bt << 16);
+                entry = e_cur | (bt << 16);
             }
-            const uint32_t msk = __ballot_sync(0xFFFFFFFFu, changed);  // also orders reads before writes
+            // the ballot also orders this round's (and the next round's) queue reads before the
+            // writes below, which land at or before slot q0 + 31
+            const uint32_t msk = __ballot_sync(0xFFFFFFFFu, changed);
             if (changed) queue[n_changed + __popc(msk & lanemask_lt)] = entry;
             n_changed += __popc(msk);
+            e_cur = e_nxt; tj = tn; mj = mn; vj = vn;
         }
         __syncwarp();
 
