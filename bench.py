@@ -280,7 +280,15 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     t_gen = time.time()
-    wl = build_workload(args.workload, device)
+    workload = args.workload
+    free_b, _ = torch.cuda.mem_get_info(device)
+    if workload == "full" and free_b < 128e9:
+        # the full state needs ~115 GB (98.3 GB of theta/m/v + 16.4 GB of shards + lists); on a
+        # smaller or partly occupied GPU run as many layers as fit and say so in config.workload
+        n_fit = max(1, int((free_b * 0.85 - 6e9) // (192946432 * 14.6)))
+        workload = f"layers:{min(36, n_fit)}"
+        log(f"[bench] only {free_b / 1e9:.0f} GB free: falling back to --workload {workload}")
+    wl = build_workload(workload, device)
     wl.variant = args.variant
     plan = wl.plan
     st, shards = materialize_resident(wl, device, dte)

@@ -209,6 +209,17 @@ DTE_API dte_status dte_extract_delta_static(const dte_layout* layout, const floa
 DTE_API dte_status dte_apply(const dte_layout* layout, const dte_delta* delta,
                      uint16_t* const* shard_ptrs, void* cuda_stream);
 
+/* Section 4.3, round 1 of the two-round transfer: the entry count c_o = |I_o| of every
+ * operation of the plan, in plan order, zero-length operations included (both peers keep
+ * the position of an empty operation, so the schedule stays aligned).  `counts`: DEVICE array
+ * of dte_layout_num_ops(layout) uint64.  `delta` must be a complete extract result (no
+ * overflow); entries of operation o are those of list dst_shard(o) whose offset lies in the
+ * operation's destination range, a contiguous run of that list. */
+DTE_API dte_status dte_op_counts(const dte_layout* layout, const dte_delta* delta, uint64_t* counts,
+                                 void* cuda_stream);
+/* Number of operations the layout was created with. */
+DTE_API size_t dte_layout_num_ops(const dte_layout* layout);
+
 /* End-to-end variant for optimizer state that lives in HOST memory (pinned for full
  * copy speed).  Copies theta / m / v (HOST arrays of n_tensors HOST pointers) into
  * `workspace` (device, >= dte_layout_host_workspace_bytes), runs the same extract into

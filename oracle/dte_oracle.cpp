@@ -73,6 +73,7 @@ inline uint16_t bf16_rne(float x) {
 }
 
 struct Result {
+    std::vector<uint64_t> op_count;   // n_ops: c_o = |I_o| (Section 4.3), zeros included
     std::vector<uint64_t> list_ptr;   // n_shards + 1
     std::vector<uint32_t> offsets;
     std::vector<uint16_t> values;
@@ -149,6 +150,7 @@ void* oracle_extract(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n
                      const float* const* theta, const float* const* m, const float* const* v,
                      const float* consts) {
     Result* res = new Result();
+    res->op_count.assign(n_ops, 0);
     std::vector<std::vector<uint64_t>> ops_of(n_tensors);
     for (uint64_t o = 0; o < n_ops; ++o) {
         const int64_t* op = ops + 10 * o;
@@ -187,6 +189,7 @@ void* oracle_extract(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n
                     return res;
                 }
                 lists[k].push_back(Entry{j, bt});
+                res->op_count[o] += 1;
             }
         }
     }
@@ -223,6 +226,12 @@ void oracle_result_copy(void* h, uint64_t* list_ptr, uint32_t* offsets, uint16_t
     std::copy(r->list_ptr.begin(), r->list_ptr.end(), list_ptr);
     std::copy(r->offsets.begin(), r->offsets.end(), offsets);
     std::copy(r->values.begin(), r->values.end(), values);
+}
+
+// c_o for every operation of the plan, in plan order (round 1 of the two-round transfer).
+void oracle_result_op_counts(void* h, uint64_t* out) {
+    Result* r = (Result*)h;
+    std::copy(r->op_count.begin(), r->op_count.end(), out);
 }
 
 void oracle_result_free(void* h) { delete (Result*)h; }

@@ -24,6 +24,7 @@ SYMBOLS = [
     "dte_layout_host_workspace_bytes", "dte_derive_constants", "dte_extract_delta", "dte_apply",
     "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
     "dte_extract_delta_static", "dte_extract_delta_groups", "dte_layout_num_groups",
+    "dte_op_counts", "dte_layout_num_ops",
 ]
 
 
@@ -86,6 +87,10 @@ def lib() -> C.CDLL:
         L.dte_extract_delta_groups.restype = C.c_int
         L.dte_layout_num_groups.argtypes = [vp]
         L.dte_layout_num_groups.restype = C.c_size_t
+        L.dte_op_counts.argtypes = [vp, vp, vp, vp]
+        L.dte_op_counts.restype = C.c_int
+        L.dte_layout_num_ops.argtypes = [vp]
+        L.dte_layout_num_ops.restype = C.c_size_t
         L.dte_apply.argtypes = [vp, vp, vp, vp]
         L.dte_apply.restype = C.c_int
         L.dte_extract_delta_host.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, u64,
@@ -295,6 +300,14 @@ def dte_extract_delta_static(layout: Layout, tables, step, lr, beta1, beta2, eps
     _check(lib().dte_extract_delta_static(layout._h, th, mm, vv, int(step), float(lr), float(beta1),
                                           float(beta2), float(eps), float(wd), C.byref(delta.struct),
                                           _stream_ptr(stream)))
+
+
+def dte_op_counts(layout: Layout, delta: Delta, stream=None) -> torch.Tensor:
+    """Entry count of every operation of the plan (plan order, zeros included), on the device."""
+    n = int(lib().dte_layout_num_ops(layout._h))
+    counts = torch.zeros(max(1, n), dtype=torch.int64, device=layout.device)
+    _check(lib().dte_op_counts(layout._h, C.byref(delta.struct), counts.data_ptr(), _stream_ptr(stream)))
+    return counts[:n]
 
 
 def dte_apply(layout: Layout, delta: Delta, shard_table, stream=None) -> None:

@@ -241,6 +241,17 @@ extern "C" dte_status dte_apply(const dte_layout* layout, const dte_delta* delta
     return launch_apply(p, L->device, st);
 }
 
+extern "C" dte_status dte_op_counts(const dte_layout* layout, const dte_delta* delta, uint64_t* counts,
+                                    void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    dte_status s = check_delta(delta);
+    if (s != DTE_OK) return s;
+    if (layout->n_ops && !counts) return fail(DTE_ERR_INVALID_ARG, "counts is null");
+    DeviceGuard g(layout->device);
+    return launch_op_counts(layout->d_op_ranges, layout->n_ops, delta->offsets, delta->list_ptr, counts,
+                            (cudaStream_t)cuda_stream);
+}
+
 extern "C" dte_status dte_extract_delta_host(const dte_layout* layout, const float* const* theta_h,
                                              const float* const* m_h, const float* const* v_h,
                                              int64_t step, double lr, double beta1, double beta2,

@@ -1,6 +1,8 @@
 // Direct sparse apply (Eq. 7): shard[k][offsets[e]] = values[e] for every entry of every
 // list.  Entry counts are read on the device (list_ptr), so the launch needs no host
 // round trip after extract.
+#include <algorithm>
+
 #include "dte_internal.cuh"
 
 namespace dte {
@@ -75,6 +77,39 @@ dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st) {
     // per SM and .cs / .cg / .wt store hints all give the same ~39 G entries/s - isolated
     // 2-byte writes are bound by the memory system's sector read-modify-write rate
     apply_kernel<<<sms * 6, kApplyThreads, 0, st>>>(p);
+    DTE_CUDA(cudaGetLastError());
+    return DTE_OK;
+}
+
+// ---- per-operation counts (Section 4.3, round 1) ---------------------------------------------
+// c_o = number of entries of the operation's list whose offset lies in the operation's
+// destination range: two binary searches in the (ascending) list.
+__global__ void op_counts_kernel(const OpRange* __restrict__ ranges, uint32_t n_ops,
+                                 const uint32_t* __restrict__ offsets, const uint64_t* __restrict__ list_ptr,
+                                 uint64_t* __restrict__ counts) {
+    for (uint32_t o = blockIdx.x * blockDim.x + threadIdx.x; o < n_ops; o += gridDim.x * blockDim.x) {
+        const OpRange r = ranges[o];
+        const uint64_t a = list_ptr[r.list], b = list_ptr[r.list + 1];
+        uint64_t pos[2];
+        const uint64_t key[2] = {r.begin, r.end};
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {          // first entry with offset >= key
+            uint64_t lo = a, hi = b;
+            while (lo < hi) {
+                const uint64_t mid = (lo + hi) >> 1;
+                if ((uint64_t)offsets[mid] < key[i]) lo = mid + 1; else hi = mid;
+            }
+            pos[i] = lo;
+        }
+        counts[o] = pos[1] - pos[0];
+    }
+}
+
+dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const uint32_t* offsets,
+                            const uint64_t* list_ptr, uint64_t* counts, cudaStream_t st) {
+    if (n_ops == 0) return DTE_OK;
+    const int threads = 128, blocks = (int)std::min<uint32_t>((n_ops + threads - 1) / threads, 4096u);
+    op_counts_kernel<<<blocks, threads, 0, st>>>(ranges, n_ops, offsets, list_ptr, counts);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }

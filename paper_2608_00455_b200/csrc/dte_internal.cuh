@@ -127,6 +127,13 @@ struct ApplyParams {
     uint32_t n_lists;
 };
 
+// Destination range of one operation, in plan order (for the per-operation counts).
+struct OpRange {
+    uint32_t list;
+    uint32_t pad;
+    uint64_t begin, end;   // receiver-local flat range [begin, end); begin == end for empty overlaps
+};
+
 void set_error(const std::string& msg);
 dte_status cuda_fail(cudaError_t e, const char* what);
 
@@ -139,6 +146,8 @@ dte_status cuda_fail(cudaError_t e, const char* what);
 dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, int n_ctas, cudaStream_t st);
 dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
+dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const uint32_t* offsets,
+                            const uint64_t* list_ptr, uint64_t* counts, cudaStream_t st);
 
 }  // namespace dte
 
@@ -166,6 +175,8 @@ struct dte_layout {
     uint32_t* d_tensor_group = nullptr;    // n_tensors
     dte::GroupConsts* d_groups = nullptr;  // n_groups
     uint32_t n_groups = 1;
+    dte::OpRange* d_op_ranges = nullptr;   // n_ops, plan order
+    uint32_t n_ops = 0;
     // host mirrors of the pointer tables last uploaded
     std::vector<const float*> h_ptrs;
     std::vector<uint16_t*> h_shards;

@@ -91,6 +91,7 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
     cudaFree(L->d_shard_numel);
     cudaFree(L->d_list_first_rec);
     cudaFree(L->d_tensor_group);
+    cudaFree(L->d_op_ranges);
     cudaFree(L->d_groups);
     if (prev >= 0) cudaSetDevice(prev);
     delete L;
@@ -98,6 +99,7 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
 
 extern "C" size_t dte_layout_num_lists(const dte_layout* L) { return L ? L->n_lists : 0; }
 extern "C" uint64_t dte_layout_num_elements(const dte_layout* L) { return L ? L->scanned : 0; }
+extern "C" size_t dte_layout_num_ops(const dte_layout* L) { return L ? L->n_ops : 0; }
 extern "C" size_t dte_layout_num_groups(const dte_layout* L) { return L ? L->n_groups : 0; }
 
 extern "C" uint64_t dte_layout_host_workspace_bytes(const dte_layout* L) {
@@ -129,7 +131,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     *out = nullptr;
     if ((n_tensors && !tensors) || (n_shards && !shards) || (n_ops && !ops))
         return fail(DTE_ERR_INVALID_ARG, "null descriptor array");
-    if (n_tensors >= kNone || n_shards >= kNone)
+    if (n_tensors >= kNone || n_shards >= kNone || n_ops >= kNone)
         return fail(DTE_ERR_LAYOUT, "too many tensors or shards");
 
     std::vector<uint64_t> numel(n_tensors);
@@ -148,6 +150,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
 
     // --- operations -> destination pieces, grouped by list -------------------
     std::vector<std::vector<Piece>> by_list(n_shards);
+    std::vector<OpRange> op_ranges(n_ops);
     std::vector<uint8_t> used(n_tensors, 0);
     for (size_t o = 0; o < n_ops; ++o) {
         const dte_op_desc& op = ops[o];
@@ -156,6 +159,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
             return fail(DTE_ERR_LAYOUT, tag + "unknown tensor or shard");
         const uint64_t n0 = tensors[op.src_tensor].shape[0], n1 = tensors[op.src_tensor].shape[1];
         const uint64_t e0 = op.extent[0], e1 = op.extent[1];
+        op_ranges[o] = OpRange{op.dst_shard, 0, 0, 0};
         if (e0 == 0 || e1 == 0) continue;  // empty overlap: legal, contributes nothing
         if (op.src_origin[0] > n0 || e0 > n0 - op.src_origin[0] || op.src_origin[1] > n1 ||
             e1 > n1 - op.src_origin[1])
@@ -173,6 +177,8 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         pc.len = e0 * e1;
         if (pc.dst_start > numel_q || pc.len > numel_q - pc.dst_start)
             return fail(DTE_ERR_LAYOUT, tag + "destination region leaves the shard");
+        op_ranges[o].begin = pc.dst_start;
+        op_ranges[o].end = pc.dst_start + pc.len;
         pc.src_start = op.src_origin[0] * n1 + op.src_origin[1];
         pc.tensor = op.src_tensor;
         pc.op = o;
@@ -288,6 +294,8 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     guard(upload(&L->d_segs, segs));
     guard(upload(&L->d_shard_numel, L->shard_numel));
     guard(upload(&L->d_list_first_rec, first_rec));
+    guard(upload(&L->d_op_ranges, op_ranges));
+    L->n_ops = (uint32_t)n_ops;
     {
         std::vector<uint32_t> grp(n_tensors);
         for (size_t p = 0; p < n_tensors; ++p) {

@@ -306,3 +306,21 @@ def test_parameter_groups_lr_and_weight_decay_per_group():
     assert int(one[0][-1]) != int(want[0][-1])
     with pytest.raises(dte.DteError):            # fewer pairs than groups
         dte.dte_extract_delta_groups(lay, tabs, step, b1, b2, eps, lr[:2], wd[:2], d)
+
+
+def test_op_counts_match_oracle_including_zero_length_operations():
+    plan = plans.qwen3_moe_plan(2, 4, 4, configs.SMALL_MOE)
+    wl = configs.Workload("counts", plan, Hyper(step=100, lr=3e-6, wd=0.01), configs._specs(plan), 23)
+    st = wl.materialize("cuda")
+    for p in range(0, plan.n_tensors, 7):          # some tensors do not change at all
+        st.m[p].zero_()
+        st.v[p].zero_()
+    lay, d = run_extract(plan, st, wl.hp)
+    got = dte.dte_op_counts(lay, d).cpu().numpy().astype(np.uint64)
+    c = oracle.derive_constants(*wl.hp.as_args())
+    host = lambda lst: [x.cpu().numpy() for x in lst]
+    want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), host(st.theta), host(st.m),
+                          host(st.v), c, with_op_counts=True)
+    assert_lists_equal(d.to_host(), want[:3], plan)
+    assert np.array_equal(got, want[3])
+    assert (got == 0).sum() > 10 and int(got.sum()) == d.total()

@@ -276,3 +276,23 @@ def test_per_tensor_constants_equal_one_tensor_at_a_time():
         got = list(zip(off[int(lp[k]):int(lp[k + 1])], val[int(lp[k]):int(lp[k + 1])]))
         assert got == sorted(merged[k])
     assert int(lp[-1]) > 1000
+
+
+def test_op_counts_keep_every_planned_operation():
+    """c_o = |I_o| per operation in plan order, zero-length ones included (Section 4.3): they add
+    up to the list lengths and equal a brute-force count of the list entries that fall into each
+    operation's destination block."""
+    plan = plans.qwen3_moe_plan(1, 4, 4, configs.SMALL_MOE)
+    wl, st, c, th, mm, vv = _random_sparse_case(plan, 8, lr=3e-6)
+    ops = plan.ops_array().copy()
+    ops = np.concatenate([ops, [[0, 0, 0, 0, 0, ops[0, 5], 0, ops[0, 7], 0, 0]]])   # an empty overlap
+    lp, off, val, cnt = oracle.extract(plan.tensor_shapes, plan.shard_numels, ops, th, mm, vv, c,
+                                       with_op_counts=True)
+    assert cnt.shape == (ops.shape[0],) and cnt[-1] == 0 and (cnt == 0).sum() > 1
+    for k in range(plan.n_shards):
+        assert int(cnt[ops[:, 1] == k].sum()) == int(lp[k + 1] - lp[k])
+    for o, (src, dst, a0, a1, e0, e1, base, ld, r0, r1) in enumerate(ops):
+        begin = base + r0 * ld + r1
+        end = begin + e0 * e1          # whole destination rows: a contiguous block
+        seg = off[int(lp[dst]):int(lp[dst + 1])].astype(np.int64)
+        assert int(((seg >= begin) & (seg < end)).sum()) == int(cnt[o])
