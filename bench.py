@@ -360,7 +360,7 @@ def main():
         total_ms = sum(e[0].elapsed_time(e[2]) for e in evs)
     ext_ms = [e[0].elapsed_time(e[1]) for e in evs]
     app_ms = [e[1].elapsed_time(e[2]) for e in evs]
-    launches = lay.last_launch()["kernels"] * args.steps + args.steps
+    launches = (lay.last_launch()["kernels"] + 1) * args.steps     # extract call + apply, per step
     bytes_per_step = 12.0 * N + 6.0 * M
     total_ms, bytes_all = aggregate_over_ranks(total_ms, bytes_per_step, dist, device)
     ms_per_step = total_ms / args.steps

@@ -129,8 +129,14 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
             div_decay |= g.c.decay != 1.0f;
         }
     }
-    const int n_ctas = (int)L->n_tiles;   // one CTA per tile
-    dte_status s = launch_extract(p, div_bc1, div_decay, n_ctas, st);
+    // one CTA per tile; full tiles and packed tiles (short runs sharing a CTA) in two launches
+    const int n_ctas = (int)L->n_tiles;
+    p.n_tiles = L->n_regular;
+    dte_status s = launch_extract(p, div_bc1, div_decay, false, st);
+    if (s != DTE_OK) return s;
+    p.tiles = L->d_packed;
+    p.n_tiles = L->n_packed;
+    s = launch_extract(p, div_bc1, div_decay, true, st);
     if (s != DTE_OK) return s;
     GatherParams g;
     g.rec = L->d_rec;
@@ -149,7 +155,7 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
     g.counters = out->counters;
     s = launch_gather(g, st);
     if (s != DTE_OK) return s;
-    launches = 4;
+    launches = 3 + (L->n_regular ? 1 : 0) + (L->n_packed ? 1 : 0);
     L->last_launch[0] = L->n_tiles;
     L->last_launch[1] = (uint64_t)n_ctas;
     L->last_launch[2] = launches;
@@ -408,7 +414,12 @@ extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const f
     p.s = make_screen(c);
     p.tensor_group = nullptr;
     p.groups = nullptr;
-    s = launch_extract(p, c.bc1 != 1.0f, c.decay != 1.0f, (int)L->n_tiles, st);
+    p.n_tiles = L->n_regular;
+    s = launch_extract(p, c.bc1 != 1.0f, c.decay != 1.0f, false, st);
+    if (s != DTE_OK) return s;
+    p.tiles = L->d_packed;
+    p.n_tiles = L->n_packed;
+    s = launch_extract(p, c.bc1 != 1.0f, c.decay != 1.0f, true, st);
     if (s != DTE_OK) return s;
     GatherParams gp;
     gp.rec = p.rec;

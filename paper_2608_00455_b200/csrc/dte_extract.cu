@@ -112,50 +112,66 @@ __device__ __forceinline__ const float* ldg_ptr(const float* const* slot) {
 }
 // ---- the kernel --------------------------------------------------------------------
 
-// Decoded descriptor of one warp-tile.
+// Row geometry of a strided (column-split) warp-tile; lives in shared memory, one per warp,
+// because it is needed only when addresses are formed and registers are scarce.
+struct StridedGeom {
+    uint32_t w, s, magic;  // row width / source row stride / divisor (SegRec)
+};
+
+// Decoded descriptor of one warp-tile.  th / mm / vv already point at the warp-tile's first
+// element (contiguous) or at the first column of its first source row (strided).
 struct WarpTile {
     const float* th;
     const float* mm;
     const float* vv;
-    uint64_t src_off;      // source element offset of the enclosing tile's row start
-    uint32_t w, s, magic;  // strided tiles: row width / stride / divisor (SegRec)
-    uint32_t col0;         // strided tiles: column of tile element 0, plus e0 folded in
+    const StridedGeom* geom;
+    uint32_t col0;         // strided: column of warp-tile element 0 within the operation's extent
     uint32_t len;          // elements of this warp-tile (0 for the unused tail of a short tile)
     uint32_t dst0;         // receiver-local offset of element 0 of this warp-tile
     uint32_t len_flags;
-    uint32_t tensor;
 
-    // source element offset of warp-tile element e
+    // source element offset (relative to th / mm / vv) of warp-tile element e
     __device__ __forceinline__ uint64_t src(uint32_t e) const {
-        if (!(len_flags & kFlagStrided)) return src_off + e;
-        const uint32_t cc = col0 + e;
-        const uint32_t row = (w == 1) ? cc : __umulhi(cc, magic);
-        return src_off + (uint64_t)row * s + (cc - row * w);
+        if (!(len_flags & kFlagStrided)) return e;
+        const uint32_t w = geom->w, cc = col0 + e;
+        const uint32_t row = (w == 1) ? cc : __umulhi(cc, geom->magic);
+        return (uint64_t)row * geom->s + (cc - row * w);
     }
 };
 
-__device__ __forceinline__ void decode(const ExtractParams& p, uint32_t t, WarpTile& wt) {
-    // all lanes read the same 32-byte descriptor (one sector, broadcast)
-    const uint4* td = reinterpret_cast<const uint4*>(p.tiles + (t / kSub));
+// Returns the source tensor index (needed once, for the parameter group); `tile` receives the
+// index of the placement record.  PACKED: every warp has a descriptor of its own; otherwise
+// the CTA shares one (its address depends on blockIdx only: uniform registers) and warp w
+// takes the w-th kWarpTile slots of it.
+template <bool PACKED>
+__device__ __forceinline__ uint32_t decode(const ExtractParams& p, int lane, int warp, StridedGeom* geom,
+                                           WarpTile& wt, uint32_t& tile) {
+    const uint4* td = reinterpret_cast<const uint4*>(PACKED ? p.tiles + ((size_t)blockIdx.x * kSub + warp)
+                                                            : p.tiles + blockIdx.x);
     const uint4 d0 = __ldg(td), d1 = __ldg(td + 1);
-    const uint32_t e0 = (t % kSub) * kWarpTile;
-    const uint32_t tile_len = d1.x & kLenMask;
+    const uint32_t e0 = PACKED ? 0u : (uint32_t)warp * kWarpTile;
+    const uint32_t run_len = d1.x & kLenMask;
+    tile = d1.y;
     wt.len_flags = d1.x;
-    wt.len = tile_len > e0 ? min(tile_len - e0, (uint32_t)kWarpTile) : 0u;
+    wt.len = run_len > e0 ? min(run_len - e0, (uint32_t)kWarpTile) : 0u;
     wt.dst0 = d0.w + e0;
-    wt.tensor = d0.z;
-    wt.th = ldg_ptr(p.theta + d0.z);
-    wt.mm = ldg_ptr(p.m + d0.z);
-    wt.vv = ldg_ptr(p.v + d0.z);
-    wt.src_off = ((uint64_t)d0.x | ((uint64_t)d0.y << 32));
-    wt.w = 0; wt.s = 0; wt.magic = 0; wt.col0 = 0;
+    wt.geom = geom;
+    wt.col0 = 0;
+    uint64_t off = ((uint64_t)d0.x | ((uint64_t)d0.y << 32));
     if (d1.x & kFlagStrided) {
-        const uint4 sr = __ldg(reinterpret_cast<const uint4*>(p.segs + d1.z));
-        wt.w = sr.x; wt.s = sr.y; wt.magic = sr.z;
+        if (lane == 0) {
+            const uint4 sr = __ldg(reinterpret_cast<const uint4*>(p.segs + d1.z));
+            geom->w = sr.x; geom->s = sr.y; geom->magic = sr.z;
+        }
+        __syncwarp();
         wt.col0 = d1.w + e0;
     } else {
-        wt.src_off += e0;
+        off += e0;
     }
+    wt.th = ldg_ptr(p.theta + d0.z) + off;
+    wt.mm = ldg_ptr(p.m + d0.z) + off;
+    wt.vv = ldg_ptr(p.v + d0.z) + off;
+    return d0.z;
 }
 
 // One chunk (kChunk elements from warp-tile element cb) of theta / m / v into registers.
@@ -195,13 +211,14 @@ __device__ __forceinline__ void load_chunk(const WarpTile& wt, uint32_t cb, int 
 }
 
 // GROUPS: the constants come from the tile's parameter group instead of the kernel parameters.
-template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS>
+template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED>
 __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const ExtractParams p) {
     // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
     // (dynamic shared memory: kWarps * kWarpTile words, may exceed the 48 KB static limit)
     extern __shared__ __align__(16) uint32_t s_queue[];
     __shared__ uint32_t s_count[kWarps];
     __shared__ unsigned long long s_pos;
+    __shared__ StridedGeom s_geom[kWarps];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* queue = s_queue + warp * kWarpTile;
     Consts c = p.c;
@@ -211,11 +228,11 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
 
     float4 a[kItems], b[kItems], g[kItems];
     WarpTile cur;
+    uint32_t tile;
     {
-        const uint32_t t = blockIdx.x * kSub + warp;
-        decode(p, t, cur);
-        if (GROUPS) {   // one 48-byte record, the same for the whole CTA
-            const uint4* gp = reinterpret_cast<const uint4*>(p.groups + __ldg(p.tensor_group + cur.tensor));
+        const uint32_t tensor = decode<PACKED>(p, lane, warp, &s_geom[warp], cur, tile);
+        if (GROUPS) {   // one 48-byte record per parameter group
+            const uint4* gp = reinterpret_cast<const uint4*>(p.groups + __ldg(p.tensor_group + tensor));
             const uint4 g0 = __ldg(gp), g1 = __ldg(gp + 1), g2 = __ldg(gp + 2);
             c.bc1 = __uint_as_float(g0.x); c.bc2 = __uint_as_float(g0.y); c.decay = __uint_as_float(g0.z);
             c.lr = __uint_as_float(g0.w); c.eps = __uint_as_float(g1.x);
@@ -327,7 +344,7 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
             unsigned long long pos0 = 0;
             if (total) pos0 = atomicAdd(p.cursor, (unsigned long long)total);
             s_pos = pos0;
-            p.rec[blockIdx.x] = ((uint64_t)pos0 << kRecCountBits) | total;
+            p.rec[tile] = ((uint64_t)pos0 << kRecCountBits) | total;
         }
         __syncthreads();
         const unsigned long long pos = s_pos + before;
@@ -344,19 +361,24 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
 
 constexpr size_t kQueueBytes = (size_t)kWarps * kWarpTile * sizeof(uint32_t);
 
-template <bool A, bool B, bool G>
-static dte_status launch_t(const ExtractParams& p, int n_ctas, cudaStream_t st) {
+template <bool A, bool B, bool G, bool P>
+static dte_status launch_t(const ExtractParams& p, cudaStream_t st) {
     static bool configured[64] = {false};     // per device: allow more than 48 KB of dynamic shared memory
     int dev = 0;
     DTE_CUDA(cudaGetDevice(&dev));
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        DTE_CUDA(cudaFuncSetAttribute(extract_kernel<A, B, G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        DTE_CUDA(cudaFuncSetAttribute(extract_kernel<A, B, G, P>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)kQueueBytes));
         configured[dev] = true;
     }
-    extract_kernel<A, B, G><<<n_ctas, kThreads, kQueueBytes, st>>>(p);
+    extract_kernel<A, B, G, P><<<p.n_tiles, kThreads, kQueueBytes, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
+}
+
+template <bool A, bool B, bool G>
+static dte_status launch_p(const ExtractParams& p, bool packed, cudaStream_t st) {
+    return packed ? launch_t<A, B, G, true>(p, st) : launch_t<A, B, G, false>(p, st);
 }
 
 #ifdef DTE_STATS
@@ -367,18 +389,20 @@ extern "C" __attribute__((visibility("default"))) void dte_debug_stats(unsigned 
 #endif
 
 // div_bc1 / div_decay: whether any group in the call has a divisor different from 1.0f.
-dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, int n_ctas, cudaStream_t st) {
+// One launch covers p.n_tiles tiles of one kind (p.tiles = their descriptors).
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, cudaStream_t st) {
+    if (p.n_tiles == 0) return DTE_OK;
     const bool a = div_bc1, b = div_decay;
     if (p.groups) {
-        if (a && b) return launch_t<true, true, true>(p, n_ctas, st);
-        if (a) return launch_t<true, false, true>(p, n_ctas, st);
-        if (b) return launch_t<false, true, true>(p, n_ctas, st);
-        return launch_t<false, false, true>(p, n_ctas, st);
+        if (a && b) return launch_p<true, true, true>(p, packed, st);
+        if (a) return launch_p<true, false, true>(p, packed, st);
+        if (b) return launch_p<false, true, true>(p, packed, st);
+        return launch_p<false, false, true>(p, packed, st);
     }
-    if (a && b) return launch_t<true, true, false>(p, n_ctas, st);
-    if (a) return launch_t<true, false, false>(p, n_ctas, st);
-    if (b) return launch_t<false, true, false>(p, n_ctas, st);
-    return launch_t<false, false, false>(p, n_ctas, st);
+    if (a && b) return launch_p<true, true, false>(p, packed, st);
+    if (a) return launch_p<true, false, false>(p, packed, st);
+    if (b) return launch_p<false, true, false>(p, packed, st);
+    return launch_p<false, false, false>(p, packed, st);
 }
 
 }  // namespace dte

@@ -12,11 +12,17 @@
 namespace dte {
 
 // ---- tiling ---------------------------------------------------------------
-// A tile is a run of <= kTile consecutive receiver-local slots of ONE list, i.e. a
-// contiguous piece of one operation's destination range.  Tiles are numbered in output
-// order (list by list, ascending offset).  Each tile is cut into kSub warp-tiles of
-// kWarpTile slots; one warp processes one warp-tile at a time, and the output position of
-// a warp-tile is the exclusive prefix sum of the changed counts of all warp-tiles before it.
+// The destination space (lists in shard order, ascending offset inside a list) is cut into
+// tiles, the work of one CTA each, numbered in output order: the output position of a tile
+// is the exclusive prefix sum of the changed counts of all tiles before it.
+//   regular tile: kTile consecutive receiver-local slots of ONE operation, one descriptor;
+//       warp w takes slots [w * kWarpTile, (w+1) * kWarpTile).  The descriptor address
+//       depends on blockIdx only, so everything decoded from it lives in uniform registers.
+//   packed tile: runs shorter than a tile (ragged ends, small tensors, one-row operations)
+//       are cut into pieces of <= kWarpTile slots; kSub consecutive pieces of one list -
+//       possibly from different operations and source tensors - share a CTA, each warp with
+//       a descriptor of its own (unused slots have length 0).  Handled by a second launch.
+// A tile never spans two lists.
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 // Measured on B200 (8 Qwen3-8B layers, 1.5 % changed): 3 items x 3 chunks at 4 CTAs/SM (64
@@ -32,17 +38,15 @@ static_assert(kTile < 16384, "a tile's changed count must fit kRecCountBits");
 constexpr uint32_t kNone = 0xFFFFFFFFu;
 
 constexpr uint32_t kLenMask = 0xFFFFu;
-constexpr uint32_t kFlagFirstOfList = 1u << 16;        // tile starts its list
-constexpr uint32_t kFlagLastTile = 1u << 17;           // last tile of the whole layout
 constexpr uint32_t kFlagScalar = 1u << 18;             // not 16-byte alignable: scalar loads
 constexpr uint32_t kFlagStrided = 1u << 19;            // crosses source rows (see SegRec)
 
 struct __align__(32) TileDesc {
-    uint64_t src_off;    // element offset in the source tensor of the tile's row start
+    uint64_t src_off;    // element offset in the source tensor of the run's row start
     uint32_t tensor;     // source tensor index
-    uint32_t dst_off;    // receiver-local offset of the tile's first element
-    uint32_t len_flags;  // low 16 bits: elements; high bits: kFlag*
-    uint32_t list;       // output list (= shard index)
+    uint32_t dst_off;    // receiver-local offset of the run's first element
+    uint32_t len_flags;  // low 16 bits: elements (0: padding); high bits: kFlag*
+    uint32_t tile;       // index of the tile (placement record) this descriptor belongs to
     uint32_t seg;        // SegRec index when strided
     uint32_t col0;       // strided: column (within the operation's extent) of the first element
 };
@@ -83,7 +87,7 @@ struct __align__(16) GroupConsts {
 static_assert(sizeof(GroupConsts) == 48, "GroupConsts is read as three uint4");
 
 struct ExtractParams {
-    const TileDesc* tiles;
+    const TileDesc* tiles;       // regular tiles: one descriptor each; packed tiles: kSub each
     const SegRec* segs;
     const float* const* theta;   // device table, n_tensors
     const float* const* m;
@@ -93,7 +97,7 @@ struct ExtractParams {
     uint32_t* stage_offsets;     // staging buffer, stage_capacity entries
     uint16_t* stage_values;
     uint64_t stage_capacity;
-    uint32_t n_tiles;
+    uint32_t n_tiles;            // tiles handled by this launch
     Consts c;                    // single-group calls: constants in the kernel parameters
     Screen s;
     const uint32_t* tensor_group;   // per-group calls: group of each source tensor ...
@@ -143,7 +147,7 @@ dte_status cuda_fail(cudaError_t e, const char* what);
         if (e__ != cudaSuccess) return dte::cuda_fail(e__, #call); \
     } while (0)
 
-dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, int n_ctas, cudaStream_t st);
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, cudaStream_t st);
 dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const uint32_t* offsets,
@@ -160,7 +164,9 @@ struct dte_layout {
     std::vector<uint64_t> shard_numel;
     std::vector<uint8_t> list_has_tiles;
     // device memory owned by the layout
-    dte::TileDesc* d_tiles = nullptr;
+    dte::TileDesc* d_tiles = nullptr;      // n_regular descriptors
+    dte::TileDesc* d_packed = nullptr;     // n_packed * kSub descriptors
+    uint32_t n_regular = 0, n_packed = 0;  // n_tiles = n_regular + n_packed
     dte::SegRec* d_segs = nullptr;
     uint64_t* d_rec = nullptr;             // n_tiles placement records
     uint64_t* d_block_sum = nullptr;       // one word per gather block

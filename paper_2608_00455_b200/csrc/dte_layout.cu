@@ -80,6 +80,7 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
     cudaGetDevice(&prev);
     cudaSetDevice(L->device);
     cudaFree(L->d_tiles);
+    cudaFree(L->d_packed);
     cudaFree(L->d_segs);
     cudaFree(L->d_rec);
     cudaFree(L->d_block_sum);
@@ -192,7 +193,9 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         by_list[op.dst_shard].push_back(pc);
     }
 
-    std::vector<TileDesc> tiles;
+    std::vector<TileDesc> tiles, packed;            // regular: one per tile; packed: kSub per tile
+    uint32_t n_rec = 0;                             // tiles so far, in output order
+    std::vector<uint32_t> list_first_tile(n_shards + 1, 0);
     std::vector<SegRec> segs;
     std::vector<uint8_t> has_tiles(n_shards, 0);
     uint64_t scanned = 0;
@@ -204,20 +207,56 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
                 return fail(DTE_ERR_LAYOUT, "operations " + std::to_string(P[i - 1].op) + " and " +
                                                 std::to_string(P[i].op) + " overlap in shard " + std::to_string(k));
         bool first = true;
+        std::vector<TileDesc> pending;      // pieces (<= kWarpTile slots) waiting to share a CTA
+        auto note_tile = [&](uint32_t tile) {
+            if (first) list_first_tile[k] = tile;
+            first = false;
+        };
+        auto flush_pending = [&]() {
+            if (pending.empty()) return;
+            const uint32_t tile = n_rec++;
+            note_tile(tile);
+            TileDesc empty;
+            std::memset(&empty, 0, sizeof empty);
+            pending.resize(kSub, empty);
+            for (TileDesc& q : pending) q.tile = tile;
+            packed.insert(packed.end(), pending.begin(), pending.end());
+            pending.clear();
+        };
         for (const Piece& pc : P) {
             scanned += pc.len;
+            // a run of <= kTile slots of this piece: a regular tile if full, else warp-level pieces
             auto push = [&](uint64_t src_off, uint64_t dst_off, uint64_t len, uint32_t flags,
                             uint32_t seg, uint32_t col0) {
                 TileDesc t;
                 t.src_off = src_off;
                 t.tensor = pc.tensor;
                 t.dst_off = (uint32_t)dst_off;
-                t.len_flags = (uint32_t)len | flags | (first ? kFlagFirstOfList : 0u);
-                t.list = (uint32_t)k;
+                t.len_flags = (uint32_t)len | flags;
                 t.seg = seg;
                 t.col0 = col0;
-                tiles.push_back(t);
-                first = false;
+                if (len == (uint64_t)kTile) {
+                    flush_pending();
+                    t.tile = n_rec++;
+                    note_tile(t.tile);
+                    tiles.push_back(t);
+                    return;
+                }
+                for (uint64_t c = 0; c < len; c += kWarpTile) {
+                    TileDesc q = t;
+                    const uint64_t n = std::min<uint64_t>(kWarpTile, len - c);
+                    q.dst_off = (uint32_t)(dst_off + c);
+                    q.len_flags = (uint32_t)n | flags;
+                    if (flags & kFlagStrided) {
+                        const uint64_t cc = col0 + c;
+                        q.src_off = src_off + (cc / pc.w) * pc.s;
+                        q.col0 = (uint32_t)(cc % pc.w);
+                    } else {
+                        q.src_off = src_off + c;
+                    }
+                    pending.push_back(q);
+                    if (pending.size() == (size_t)kSub) flush_pending();
+                }
             };
             if (pc.rows == 1) {
                 const bool vec = (pc.src_start % 4 == 0);
@@ -256,10 +295,11 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
                 }
             }
         }
+        flush_pending();
         has_tiles[k] = !first;
     }
-    if (tiles.size() >= kNone) return fail(DTE_ERR_LAYOUT, "too many tiles");
-    if (!tiles.empty()) tiles.back().len_flags |= kFlagLastTile;
+    const size_t n_ctas = n_rec;
+    if (tiles.size() + packed.size() >= kNone) return fail(DTE_ERR_LAYOUT, "too many tiles");
 
     int prev = -1;
     DTE_CUDA(cudaGetDevice(&prev));
@@ -268,7 +308,9 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     L->device = device;
     L->n_tensors = (uint32_t)n_tensors;
     L->n_lists = (uint32_t)n_shards;
-    L->n_tiles = (uint32_t)tiles.size();
+    L->n_tiles = (uint32_t)n_ctas;
+    L->n_regular = (uint32_t)tiles.size();
+    L->n_packed = (uint32_t)(packed.size() / kSub);
     L->n_segs = (uint32_t)segs.size();
     L->scanned = scanned;
     L->tensor_numel = numel;
@@ -279,18 +321,15 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     // first placement record of each list; lists without tiles start where the next list
     // with tiles starts (n_rec if none follows)
     std::vector<uint32_t> first_rec(n_shards, 0);
-    {
-        std::vector<uint32_t> first_tile(n_shards + 1, (uint32_t)tiles.size());
-        for (size_t i = tiles.size(); i-- > 0;)
-            if (tiles[i].len_flags & kFlagFirstOfList) first_tile[tiles[i].list] = (uint32_t)i;
-        for (size_t k = n_shards; k-- > 0;) {
-            if (!has_tiles[k]) first_tile[k] = first_tile[k + 1];
-            first_rec[k] = first_tile[k];
-        }
+    list_first_tile[n_shards] = (uint32_t)n_ctas;
+    for (size_t k = n_shards; k-- > 0;) {
+        if (!has_tiles[k]) list_first_tile[k] = list_first_tile[k + 1];
+        first_rec[k] = list_first_tile[k];
     }
     dte_status st = DTE_OK;
     auto guard = [&](dte_status s) { if (st == DTE_OK) st = s; };
     guard(upload(&L->d_tiles, tiles));
+    guard(upload(&L->d_packed, packed));
     guard(upload(&L->d_segs, segs));
     guard(upload(&L->d_shard_numel, L->shard_numel));
     guard(upload(&L->d_list_first_rec, first_rec));
@@ -305,7 +344,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         guard(upload(&L->d_tensor_group, grp));
     }
     if (st == DTE_OK) {
-        const size_t n_rec = tiles.size();
+        const size_t n_rec = n_ctas;
         const size_t n_blocks = (n_rec + kRecsPerBlock - 1) / kRecsPerBlock;
         cudaError_t e = cudaMalloc((void**)&L->d_rec, std::max<size_t>(1, n_rec) * sizeof(uint64_t));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_block_sum, std::max<size_t>(1, n_blocks) * sizeof(uint64_t));
