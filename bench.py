@@ -35,7 +35,7 @@ UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per scanned element of the extract kernel, from the ncu capture summarised in
 # profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over a 2.3 GB case, per element).
-NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT = 12.134
+NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT = 12.125
 
 
 def log(*a):
