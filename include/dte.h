@@ -182,10 +182,12 @@ DTE_API dte_status dte_extract_delta_groups(const dte_layout* layout, const floa
  * staging buffer live in one fixed array inside the library's device image (about 12.5 MiB;
  * every GPU that loads the library holds it until the process exits), and it calls no
  * cudaMalloc, cudaFree or other device-allocating routine.
- *   Limits: the layout may have at most DTE_STATIC_MAX_TILES tiles (a tile is up to 9216
- * consecutive destination slots of one operation, so up to 603,979,776 scanned elements when
- * the tiles are full) and out->capacity at most DTE_STATIC_MAX_CAPACITY entries.  Larger
- * requests return DTE_ERR_CAPACITY with the numbers in dte_last_error(); nothing is enqueued.
+ *   Limits: the layout may have at most DTE_STATIC_MAX_TILES tiles (a tile is the work of one
+ * CTA: 9216 consecutive destination slots of one operation, or up to eight shorter runs of one
+ * list; a layout of full tiles scans up to 603,979,776 elements, and dte_layout_last_launch
+ * reports the tile count of a layout after any extract) and out->capacity at most
+ * DTE_STATIC_MAX_CAPACITY entries.  Larger requests return DTE_ERR_CAPACITY with the numbers in
+ * dte_last_error(); nothing is enqueued.
  *   The first call on a device looks up the array's address on that device (a host-side
  * query, once per device and process); make that first call before starting a stream capture.
  *   All calls on a device share the array, and it keeps what the last call left.  The call
