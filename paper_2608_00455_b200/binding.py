@@ -42,6 +42,11 @@ class OpDesc(C.Structure):
                 ("dst_base", C.c_uint64), ("dst_ld", C.c_uint64), ("dst_origin", C.c_uint64 * 2)]
 
 
+_OP_DTYPE = np.dtype([("src_tensor", np.uint32), ("dst_shard", np.uint32), ("src_origin", np.uint64, (2,)),
+                      ("extent", np.uint64, (2,)), ("dst_base", np.uint64), ("dst_ld", np.uint64),
+                      ("dst_origin", np.uint64, (2,))])
+
+
 class DeltaStruct(C.Structure):
     _fields_ = [("offsets", C.c_void_p), ("values", C.c_void_p), ("capacity", C.c_uint64),
                 ("list_ptr", C.c_void_p), ("counters", C.c_void_p)]
@@ -186,15 +191,15 @@ class Layout:
             S[k].numel = n
             S[k].receiver = int(shard_receivers[k]) if shard_receivers is not None else 0
         ops = np.asarray(ops, dtype=np.int64).reshape(-1, 10)
-        O = (OpDesc * max(1, ops.shape[0]))()
-        for i, r in enumerate(ops):
-            O[i].src_tensor, O[i].dst_shard = int(r[0]), int(r[1])
-            O[i].src_origin[0], O[i].src_origin[1] = int(r[2]), int(r[3])
-            O[i].extent[0], O[i].extent[1] = int(r[4]), int(r[5])
-            O[i].dst_base, O[i].dst_ld = int(r[6]), int(r[7])
-            O[i].dst_origin[0], O[i].dst_origin[1] = int(r[8]), int(r[9])
+        # dte_op_desc as a numpy record array (same layout as OpDesc): a plan can have millions of rows
+        O = np.zeros(max(1, ops.shape[0]), dtype=_OP_DTYPE)
+        if ops.shape[0]:
+            O["src_tensor"], O["dst_shard"] = ops[:, 0], ops[:, 1]
+            O["src_origin"], O["extent"] = ops[:, 2:4], ops[:, 4:6]
+            O["dst_base"], O["dst_ld"], O["dst_origin"] = ops[:, 6], ops[:, 7], ops[:, 8:10]
+        assert O.dtype.itemsize == C.sizeof(OpDesc)
         h = C.c_void_p()
-        _check(lib().dte_layout_create(T, len(shapes), S, len(self.shard_numels), O, ops.shape[0],
+        _check(lib().dte_layout_create(T, len(shapes), S, len(self.shard_numels), O.ctypes.data, ops.shape[0],
                                        self.device.index or 0, C.byref(h)))
         self._h = h
 
