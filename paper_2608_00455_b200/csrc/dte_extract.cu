@@ -210,6 +210,73 @@ __device__ __forceinline__ void load_chunk(const WarpTile& wt, uint32_t cb, int 
     }
 }
 
+// Phase A of one warp-tile: stream theta / m / v chunk by chunk, screen every element, and
+// append the indices of the undecided ones to the warp's queue in element order.  Returns the
+// queue length.
+template <bool DIV_BC1, bool DIV_DECAY, bool FAST>
+__device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint32_t* queue, const Screen& sc,
+                                            float abs_lr) {
+    float4 a[kItems], b[kItems], g[kItems];
+    uint32_t qn = 0;
+#pragma unroll 1
+    for (uint32_t cb = 0; cb < (FAST ? (uint32_t)kWarpTile : cur.len); cb += kChunk) {
+        if (FAST) {
+            const float4* pt = reinterpret_cast<const float4*>(cur.th + cb) + lane;
+            const float4* pm = reinterpret_cast<const float4*>(cur.mm + cb) + lane;
+            const float4* pv = reinterpret_cast<const float4*>(cur.vv + cb) + lane;
+#pragma unroll
+            for (int i = 0; i < kItems; ++i) {
+                a[i] = __ldg(pt + i * 32);
+                b[i] = __ldg(pm + i * 32);
+                g[i] = __ldg(pv + i * 32);
+            }
+        } else {
+            load_chunk(cur, cb, lane, a, b, g);
+        }
+        uint32_t amb[kItems];
+        uint32_t cnt = 0;
+#pragma unroll
+        for (int i = 0; i < kItems; ++i) {
+            const uint32_t e = cb + i * 128 + lane * 4;
+            amb[i] = 0;
+            if (FAST || e < cur.len) {
+                const float tt[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
+                const float m4[4] = {b[i].x, b[i].y, b[i].z, b[i].w};
+                const float v4[4] = {g[i].x, g[i].y, g[i].z, g[i].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (!surely_unchanged<DIV_BC1, DIV_DECAY>(tt[j], m4[j], v4[j], sc, abs_lr)) amb[i] |= 1u << j;
+                if (!FAST && (cur.len_flags & kFlagScalar))           // ragged tail of a scalar tile
+                    amb[i] &= (1u << min(cur.len - e, 4u)) - 1u;
+            }
+            cnt |= __popc(amb[i]) << (8 * i);
+        }
+        // ordered slots: warp scan of the per-item counts, packed 8 bits each (each <= 128)
+        uint32_t incl = cnt;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= d) incl += up;
+        }
+        const uint32_t excl = incl - cnt;
+        const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
+        uint32_t run = qn;
+#pragma unroll
+        for (int i = 0; i < kItems; ++i) {
+            uint32_t pos = run + ((excl >> (8 * i)) & 0xFFu);
+            uint32_t mk = amb[i];
+            while (mk) {
+                const int j = __ffs(mk) - 1;
+                mk &= mk - 1;
+                queue[pos++] = cb + i * 128 + lane * 4 + j;
+            }
+            run += (tot >> (8 * i)) & 0xFFu;
+        }
+        qn = run;
+    }
+    return qn;
+}
+
 // GROUPS: the constants come from the tile's parameter group instead of the kernel parameters.
 template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED>
 __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const ExtractParams p) {
@@ -226,7 +293,6 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
     const uint32_t lanemask_lt = (1u << lane) - 1u;
     static_assert(kSub == kWarps, "one warp per warp-tile");
 
-    float4 a[kItems], b[kItems], g[kItems];
     WarpTile cur;
     uint32_t tile;
     {
@@ -242,51 +308,13 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
         const float abs_lr = fabsf(c.lr);
 
         // ---- phase A: stream, screen, queue the undecided elements in element order ---------
+        // FAST: a full, contiguous, 16-byte-aligned warp-tile (nearly all of them): no bounds
+        // checks and no per-item address arithmetic (pointer + immediate).
         uint32_t qn = 0;
-#pragma unroll 1
-        for (uint32_t cb = 0; cb < cur.len; cb += kChunk) {
-            load_chunk(cur, cb, lane, a, b, g);
-            uint32_t amb[kItems];
-            uint32_t cnt = 0;
-#pragma unroll
-            for (int i = 0; i < kItems; ++i) {
-                const uint32_t e = cb + i * 128 + lane * 4;
-                amb[i] = 0;
-                if (e < cur.len) {
-                    const float tt[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
-                    const float m4[4] = {b[i].x, b[i].y, b[i].z, b[i].w};
-                    const float v4[4] = {g[i].x, g[i].y, g[i].z, g[i].w};
-#pragma unroll
-                    for (int j = 0; j < 4; ++j)
-                        if (!surely_unchanged<DIV_BC1, DIV_DECAY>(tt[j], m4[j], v4[j], sc, abs_lr)) amb[i] |= 1u << j;
-                    if (cur.len_flags & kFlagScalar)                  // ragged tail of a scalar tile
-                        amb[i] &= (1u << min(cur.len - e, 4u)) - 1u;
-                }
-                cnt |= __popc(amb[i]) << (8 * i);
-            }
-            // ordered slots: warp scan of the per-item counts, packed 4 x 8 bits (each <= 128)
-            uint32_t incl = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                if (lane >= d) incl += up;
-            }
-            const uint32_t excl = incl - cnt;
-            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            uint32_t run = qn;
-#pragma unroll
-            for (int i = 0; i < kItems; ++i) {
-                uint32_t pos = run + ((excl >> (8 * i)) & 0xFFu);
-                uint32_t mk = amb[i];
-                while (mk) {
-                    const int j = __ffs(mk) - 1;
-                    mk &= mk - 1;
-                    queue[pos++] = cb + i * 128 + lane * 4 + j;
-                }
-                run += (tot >> (8 * i)) & 0xFFu;
-            }
-            qn = run;
-        }
+        if (cur.len == (uint32_t)kWarpTile && !(cur.len_flags & (kFlagScalar | kFlagStrided)))
+            qn = phase_a<DIV_BC1, DIV_DECAY, true>(cur, lane, queue, sc, abs_lr);
+        else
+            qn = phase_a<DIV_BC1, DIV_DECAY, false>(cur, lane, queue, sc, abs_lr);
         __syncwarp();
         DTE_STAT(0, qn);
         DTE_STAT(2, (qn + 31) / 32);
