@@ -409,3 +409,14 @@ def mcore_dense_plan(n_layers: int, tp_send: int, tp_recv: int, with_embeddings:
             for piece in restrict_to_flat_range(op, n1, lo, hi):
                 q.ops.append((new_index[op[0], d],) + tuple(piece[1:]))
     return q
+
+
+def canonical_plan(names: Sequence[str], shapes: Sequence[Sequence[int]]) -> Plan:
+    """Identity plan: every source tensor maps onto one destination of its own shape, so the
+    lists are the canonical (index, value) pairs of Eq. 4 - what the storage path publishes
+    before any receiver layout is applied (Section 4.4)."""
+    p = Plan()
+    for name, shape in zip(names, shapes):
+        t = p.add_tensor(name, shape)
+        p.replicated(name, t, 0)
+    return p

@@ -324,3 +324,21 @@ def test_op_counts_match_oracle_including_zero_length_operations():
     assert_lists_equal(d.to_host(), want[:3], plan)
     assert np.array_equal(got, want[3])
     assert (got == 0).sum() > 10 and int(got.sum()) == d.total()
+
+
+def test_identity_plan_yields_the_canonical_pairs_of_eq4():
+    # Section 4.2.1 / 4.4: with an identity plan the lists are I = nonzero(M), V = vec(W_t)[I]
+    # per canonical tensor, checked here against the oracle's Eq. 4 mask tensor by tensor
+    dense = plans.qwen3_dense_plan(1, 1, True, configs.SMALL_DENSE)
+    plan = plans.canonical_plan(dense.tensor_names, dense.tensor_shapes)
+    wl = configs.Workload("canonical", plan, Hyper(step=200, lr=2e-6, wd=0.05), configs._specs(plan), 77)
+    st = wl.materialize("cuda")
+    lay, d = run_extract(plan, st, wl.hp)
+    lp, off, val = d.to_host()
+    c = oracle.derive_constants(*wl.hp.as_args())
+    for p in range(plan.n_tensors):
+        mask, v16 = oracle.changed_mask(st.theta[p].cpu().numpy(), st.m[p].cpu().numpy(), st.v[p].cpu().numpy(), c)
+        idx = np.nonzero(mask)[0]
+        assert np.array_equal(off[int(lp[p]):int(lp[p + 1])], idx.astype(np.uint32)), plan.tensor_names[p]
+        assert np.array_equal(val[int(lp[p]):int(lp[p + 1])], v16[idx])
+    assert int(lp[-1]) > 1000
