@@ -1,7 +1,7 @@
 """ctypes front end of the CPU oracle (test infrastructure, not product code).
 
 Only tests, the smoke check and the benchmark's CPU-baseline leg import this
-package.  It compiles ``dte_oracle.cpp`` with g++ on first use and exposes the
+package.  It compiles ``dte_oracle.cpp`` and ``chunk_oracle.cpp`` with g++ on first use and exposes the
 oracle's functions on numpy arrays.  Nothing here touches the CUDA library.
 """
 from __future__ import annotations
@@ -14,7 +14,7 @@ import threading
 import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-_SRC = os.path.join(_HERE, "dte_oracle.cpp")
+_SRCS = [os.path.join(_HERE, "dte_oracle.cpp"), os.path.join(_HERE, "chunk_oracle.cpp")]
 _LIB = os.path.join(_HERE, "libdte_oracle.so")
 _CXXFLAGS = ["-O2", "-std=c++17", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
 _lock = threading.Lock()
@@ -23,9 +23,9 @@ _lib = None
 
 def build(force: bool = False) -> str:
     """Compile the oracle into ``libdte_oracle.so`` next to its source."""
-    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < max(map(os.path.getmtime, _SRCS)):
         tmp = _LIB + f".tmp{os.getpid()}"
-        subprocess.run(["g++", *_CXXFLAGS, "-o", tmp, _SRC], check=True)
+        subprocess.run(["g++", *_CXXFLAGS, "-o", tmp, *_SRCS], check=True)
         os.replace(tmp, _LIB)
     return _LIB
 
@@ -61,6 +61,14 @@ def lib() -> ctypes.CDLL:
             L.oracle_apply.argtypes = [c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                        c.c_void_p]
             L.oracle_apply.restype = c.c_int
+            L.oracle_adler32.argtypes = [c.c_void_p, c.c_uint64]
+            L.oracle_adler32.restype = c.c_uint32
+            L.oracle_pack_chunks.argtypes = [c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_uint32,
+                                             c.c_uint32, c.c_void_p, c.c_void_p, c.c_void_p]
+            L.oracle_pack_chunks.restype = c.c_uint64
+            L.oracle_unpack_chunks.argtypes = [c.c_void_p, c.c_void_p, c.c_uint64, c.c_uint64,
+                                               c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+            L.oracle_unpack_chunks.restype = c.c_uint64
             _lib = L
     return _lib
 
@@ -168,3 +176,45 @@ def apply(shard_numels, list_ptr, offsets, values, shards) -> None:
                             val.ctypes.data, _ptr_array(shards))
     if rc != 0:
         raise ValueError("receiver index outside its shard")
+
+
+def adler32(data) -> int:
+    """Adler-32 (RFC 1950) of a byte string / uint8 array, by its definition."""
+    b = np.ascontiguousarray(np.frombuffer(bytes(data), dtype=np.uint8))
+    return int(lib().oracle_adler32(b.ctypes.data if b.size else None, b.size))
+
+
+def pack_chunks(list_ptr, offsets, values, chunk_entries, fmt=0):
+    """Serialise lists into the chunk stream of the storage path (Section 4.4).
+
+    Returns (stream uint8[bytes], directory uint64[n_chunks + 1, 3] = {byte offset, list,
+    first_entry}; the last row holds the total size)."""
+    lp = np.ascontiguousarray(list_ptr, dtype=np.uint64)
+    off = np.ascontiguousarray(offsets, dtype=np.uint32)
+    val = np.ascontiguousarray(values, dtype=np.uint16)
+    n_lists = lp.size - 1
+    n_chunks = np.zeros(1, np.uint64)
+    args = (n_lists, lp.ctypes.data, off.ctypes.data, val.ctypes.data, int(chunk_entries), int(fmt))
+    size = lib().oracle_pack_chunks(*args, None, None, n_chunks.ctypes.data)
+    if size == 2 ** 64 - 1:
+        raise ValueError("chunk_entries must be a positive multiple of 8 and fmt 0 or 1")
+    stream = np.zeros(int(size), np.uint8)
+    directory = np.zeros((int(n_chunks[0]) + 1, 3), np.uint64)
+    lib().oracle_pack_chunks(*args, stream.ctypes.data, directory.ctypes.data, n_chunks.ctypes.data)
+    return stream, directory
+
+
+def unpack_chunks(stream, directory, list_ptr):
+    """Inverse of pack_chunks: (offsets uint32[M], values uint16[M], rejected chunks, entries
+    written); entries of rejected chunks stay zero."""
+    st = np.ascontiguousarray(stream, dtype=np.uint8)
+    d = np.ascontiguousarray(directory, dtype=np.uint64).reshape(-1, 3)
+    lp = np.ascontiguousarray(list_ptr, dtype=np.uint64)
+    total = int(lp[-1])
+    off = np.zeros(total, np.uint32)
+    val = np.zeros(total, np.uint16)
+    written = np.zeros(1, np.uint64)
+    rejected = lib().oracle_unpack_chunks(st.ctypes.data, d.ctypes.data, d.shape[0] - 1, lp.size - 1,
+                                          lp.ctypes.data, off.ctypes.data, val.ctypes.data,
+                                          written.ctypes.data)
+    return off, val, int(rejected), int(written[0])
