@@ -61,6 +61,7 @@ typedef enum dte_status {
 #define DTE_DEV_OVERFLOW 1u /* more changed elements than `capacity`; lists not produced   */
 #define DTE_DEV_BOUNDS 2u   /* apply met an offset >= numel of its shard; entry skipped  */
 #define DTE_DEV_TIMEOUT 4u  /* reserved (no kernel of this library waits on another CTA)  */
+#define DTE_DEV_CORRUPT 8u  /* unpack rejected a chunk (header or checksum); lists have holes */
 
 /* Source tensor p of the canonical training-side space: fp32, row-major.  ndim is 1 or 2;
  * for ndim == 1 shape[1] must be 1.  `group` is the tensor's parameter group (< 65536): the
@@ -207,7 +208,8 @@ DTE_API dte_status dte_extract_delta_static(const dte_layout* layout, const floa
  * shard_ptrs: HOST array of n_shards DEVICE pointers (BF16 buffers, numel as declared;
  * shards whose lists are necessarily empty may be NULL).  Reads list sizes on the device,
  * so it can be enqueued right after extract without a host round trip.  Refuses to write
- * anything (and sets DTE_DEV_OVERFLOW again) if `delta` overflowed its capacity. */
+ * anything (and sets DTE_DEV_OVERFLOW again) if `delta` overflowed its capacity, and nothing
+ * if its counters carry DTE_DEV_CORRUPT (lists read from a damaged chunk stream). */
 DTE_API dte_status dte_apply(const dte_layout* layout, const dte_delta* delta,
                      uint16_t* const* shard_ptrs, void* cuda_stream);
 
@@ -221,6 +223,74 @@ DTE_API dte_status dte_op_counts(const dte_layout* layout, const dte_delta* delt
                                  void* cuda_stream);
 /* Number of operations the layout was created with. */
 DTE_API size_t dte_layout_num_ops(const dte_layout* layout);
+
+/* ---- Chunk codec of the storage-mediated path (Section 4.4) ---------------------------------
+ * Across clusters the paper publishes the sparse changes as compressed payload chunks of
+ * changed index-value pairs, every entry an int32 index and a BF16 value, and a manifest with
+ * the payload locations, lengths and checksums; the destination verifies and applies them.
+ * The paper prints no byte layout; this library's is:
+ *   stream  : chunks back to back, each on a 16-byte boundary, lists in order, entries of a
+ *             list in ascending order, at most `chunk_entries` entries of ONE list per chunk,
+ *             no chunk for an empty list.
+ *   chunk   : 32-byte header + payload.  Header = eight little-endian uint32: DTE_CHUNK_MAGIC,
+ *             format, list, first_entry (rank of the chunk's first entry within its list),
+ *             count, payload_bytes, checksum, 0.
+ *   payload : DTE_CHUNK_PLAIN - count x int32 index, count x BF16 value, zeros to a multiple
+ *             of 16 bytes.  DTE_CHUNK_BYTE_PLANES - six planes of P = count rounded up to a
+ *             multiple of 16 bytes: byte 0, 1, 2, 3 of every index, byte 0, 1 of every value,
+ *             each zero-padded; the same entries transposed so that a byte-oriented compressor
+ *             (the paper uses Zstandard, a host library outside this path) finds the slowly
+ *             varying bytes together.
+ *   checksum: Adler-32 (RFC 1950) of header bytes [0, 24) followed by the payload.
+ *   directory (the manifest's locations): one dte_chunk_ref per chunk and a final entry
+ *             {total bytes, 0xFFFFFFFF, 0}.
+ * Lists are whatever the layout's shards are: with an identity plan (every source tensor its
+ * own destination) they are the canonical (index, value) pairs of Eq. 4 that this path ships. */
+#define DTE_CHUNK_MAGIC 0x43455444u /* "DTEC" */
+#define DTE_CHUNK_HEADER_BYTES 32u
+#define DTE_CHUNK_PLAIN 0u
+#define DTE_CHUNK_BYTE_PLANES 1u
+#define DTE_CHUNK_MAX_ENTRIES 1048576u
+
+typedef struct dte_chunk_ref {
+    uint64_t byte_offset; /* of the chunk's header in the stream; multiple of 16 */
+    uint32_t list;
+    uint32_t first_entry;
+} dte_chunk_ref;
+
+/* Upper bounds for sizing: chunks (the directory needs one entry more) and stream bytes for a
+ * delta of at most `entries` entries in `n_lists` lists.  Host only; 0 if chunk_entries is 0. */
+DTE_API uint64_t dte_chunk_count_bound(size_t n_lists, uint64_t entries, uint32_t chunk_entries);
+DTE_API uint64_t dte_chunk_bytes_bound(size_t n_lists, uint64_t entries, uint32_t chunk_entries,
+                                       uint32_t format);
+
+/* Serialises a complete extract result.  All buffers are DEVICE memory owned by the caller:
+ *   stream    : stream_capacity bytes, 16-byte aligned
+ *   directory : directory_capacity + 1 entries
+ *   info      : 4 x uint64 = { chunks, stream bytes, DTE_DEV_* bits, entries }
+ * chunk_entries: a multiple of 8 in [8, DTE_CHUNK_MAX_ENTRIES]; format: DTE_CHUNK_*.
+ * Sizes are found on the device (no host round trip after extract).  If the delta overflowed,
+ * or the chunks do not fit the directory or the stream, DTE_DEV_OVERFLOW is set in info[2] and
+ * nothing is serialised; in the second case info[0] and info[1] hold the exact requirement.
+ * Deterministic: the same lists give the same bytes.  Errors: DTE_ERR_INVALID_ARG, DTE_ERR_CUDA. */
+DTE_API dte_status dte_pack_chunks(const dte_layout* layout, const dte_delta* delta, uint32_t chunk_entries,
+                                   uint32_t format, void* stream, uint64_t stream_capacity,
+                                   dte_chunk_ref* directory, uint64_t directory_capacity, uint64_t* info,
+                                   void* cuda_stream);
+
+/* Reads a stream back into lists.  stream / directory: DEVICE memory (stream 16-byte aligned;
+ * n_chunks + 1 directory entries, as published).  out->list_ptr is an INPUT here: the list
+ * boundaries from the manifest ((num_lists + 1) x uint64, device); out->offsets / values receive
+ * the entries; out->counters = { entries written, chunks accepted, DTE_DEV_* bits, chunks
+ * rejected }.  A chunk is rejected - none of its entries written, DTE_DEV_CORRUPT set - when the
+ * directory places it outside the stream or off a 16-byte boundary, when its header disagrees
+ * with the directory, the lists or its own size, or when its checksum does not match; the
+ * checksum is verified before the first entry of the chunk is written.  dte_apply refuses a
+ * delta whose counters carry DTE_DEV_CORRUPT.  If list_ptr's total exceeds out->capacity every
+ * chunk is rejected and DTE_DEV_OVERFLOW is set as well. */
+DTE_API dte_status dte_unpack_chunks(const dte_layout* layout, const void* stream, uint64_t stream_bytes,
+                                     const dte_chunk_ref* directory, uint64_t n_chunks,
+                                     const dte_delta* out, void* cuda_stream);
 
 /* End-to-end variant for optimizer state that lives in HOST memory (pinned for full
  * copy speed).  Copies theta / m / v (HOST arrays of n_tensors HOST pointers) into

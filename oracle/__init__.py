@@ -66,7 +66,7 @@ def lib() -> ctypes.CDLL:
             L.oracle_pack_chunks.argtypes = [c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_uint32,
                                              c.c_uint32, c.c_void_p, c.c_void_p, c.c_void_p]
             L.oracle_pack_chunks.restype = c.c_uint64
-            L.oracle_unpack_chunks.argtypes = [c.c_void_p, c.c_void_p, c.c_uint64, c.c_uint64,
+            L.oracle_unpack_chunks.argtypes = [c.c_void_p, c.c_uint64, c.c_void_p, c.c_uint64, c.c_uint64,
                                                c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
             L.oracle_unpack_chunks.restype = c.c_uint64
             _lib = L
@@ -214,7 +214,7 @@ def unpack_chunks(stream, directory, list_ptr):
     off = np.zeros(total, np.uint32)
     val = np.zeros(total, np.uint16)
     written = np.zeros(1, np.uint64)
-    rejected = lib().oracle_unpack_chunks(st.ctypes.data, d.ctypes.data, d.shape[0] - 1, lp.size - 1,
+    rejected = lib().oracle_unpack_chunks(st.ctypes.data, st.size, d.ctypes.data, d.shape[0] - 1, lp.size - 1,
                                           lp.ctypes.data, off.ctypes.data, val.ctypes.data,
                                           written.ctypes.data)
     return off, val, int(rejected), int(written[0])

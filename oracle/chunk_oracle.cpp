@@ -141,21 +141,28 @@ uint64_t oracle_pack_chunks(uint64_t n_lists, const uint64_t* list_ptr, const ui
 }
 
 // Reads a stream back into lists laid out by `list_ptr` (from the manifest).  A chunk is
-// rejected, and none of its entries written, when its header is inconsistent (magic, format,
-// list or range outside the lists, payload size, chunk extent in the directory) or when the
+// rejected, and none of its entries written, when the directory places it outside the stream
+// or off a 16-byte boundary, when its header is inconsistent (magic, format, list or range
+// outside the lists, payload size, chunk extent in the directory) or when the
 // chunk's checksum differs from the header's.  Returns the number of rejected chunks;
 // *entries_written counts the accepted entries.
-uint64_t oracle_unpack_chunks(const uint8_t* stream, const uint64_t* dir, uint64_t n_chunks,
-                              uint64_t n_lists, const uint64_t* list_ptr, uint32_t* offsets,
-                              uint16_t* values, uint64_t* entries_written) {
+uint64_t oracle_unpack_chunks(const uint8_t* stream, uint64_t stream_bytes, const uint64_t* dir,
+                              uint64_t n_chunks, uint64_t n_lists, const uint64_t* list_ptr,
+                              uint32_t* offsets, uint16_t* values, uint64_t* entries_written) {
     uint64_t rejected = 0, written = 0;
     for (uint64_t c = 0; c < n_chunks; ++c) {
-        const uint8_t* h = stream + dir[3 * c];
-        const uint64_t extent = dir[3 * (c + 1)] - dir[3 * c];
+        const uint64_t begin = dir[3 * c], end = dir[3 * (c + 1)];
+        // the directory must place the chunk inside the stream, on a 16-byte boundary
+        if (begin % 16 != 0 || end < begin || end - begin < kHeaderBytes || end > stream_bytes) {
+            rejected += 1;
+            continue;
+        }
+        const uint8_t* h = stream + begin;
+        const uint64_t extent = end - begin;
         const uint32_t magic = get_u32(h), format = get_u32(h + 4), list = get_u32(h + 8);
         const uint32_t first = get_u32(h + 12), count = get_u32(h + 16), pb = get_u32(h + 20);
         const uint32_t sum = get_u32(h + 24);
-        bool ok = extent >= kHeaderBytes && magic == kMagic && format <= 1 && list < n_lists &&
+        bool ok = magic == kMagic && format <= 1 && list < n_lists &&
                   count > 0;
         ok = ok && list == dir[3 * c + 1] && first == dir[3 * c + 2];
         ok = ok && (uint64_t)first + count <= list_ptr[list + 1] - list_ptr[list];

@@ -17,14 +17,17 @@ import torch
 from . import build as _build
 
 DTE_OK = 0
-DTE_DEV_OVERFLOW, DTE_DEV_BOUNDS, DTE_DEV_TIMEOUT = 1, 2, 4
+DTE_DEV_OVERFLOW, DTE_DEV_BOUNDS, DTE_DEV_TIMEOUT, DTE_DEV_CORRUPT = 1, 2, 4, 8
+DTE_CHUNK_PLAIN, DTE_CHUNK_BYTE_PLANES = 0, 1
+DTE_CHUNK_MAGIC, DTE_CHUNK_HEADER_BYTES, DTE_CHUNK_MAX_ENTRIES = 0x43455444, 32, 1 << 20
 
 SYMBOLS = [
     "dte_layout_create", "dte_layout_destroy", "dte_layout_num_lists", "dte_layout_num_elements",
     "dte_layout_host_workspace_bytes", "dte_derive_constants", "dte_extract_delta", "dte_apply",
     "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
     "dte_extract_delta_static", "dte_extract_delta_groups", "dte_layout_num_groups",
-    "dte_op_counts", "dte_layout_num_ops",
+    "dte_op_counts", "dte_layout_num_ops", "dte_chunk_count_bound", "dte_chunk_bytes_bound",
+    "dte_pack_chunks", "dte_unpack_chunks",
 ]
 
 
@@ -96,6 +99,14 @@ def lib() -> C.CDLL:
         L.dte_op_counts.restype = C.c_int
         L.dte_layout_num_ops.argtypes = [vp]
         L.dte_layout_num_ops.restype = C.c_size_t
+        L.dte_chunk_count_bound.argtypes = [C.c_size_t, u64, C.c_uint32]
+        L.dte_chunk_count_bound.restype = u64
+        L.dte_chunk_bytes_bound.argtypes = [C.c_size_t, u64, C.c_uint32, C.c_uint32]
+        L.dte_chunk_bytes_bound.restype = u64
+        L.dte_pack_chunks.argtypes = [vp, vp, C.c_uint32, C.c_uint32, vp, u64, vp, u64, vp, vp]
+        L.dte_pack_chunks.restype = C.c_int
+        L.dte_unpack_chunks.argtypes = [vp, vp, u64, vp, u64, vp, vp]
+        L.dte_unpack_chunks.restype = C.c_int
         L.dte_apply.argtypes = [vp, vp, vp, vp]
         L.dte_apply.restype = C.c_int
         L.dte_extract_delta_host.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, u64,
@@ -318,6 +329,55 @@ def dte_op_counts(layout: Layout, delta: Delta, stream=None) -> torch.Tensor:
 def dte_apply(layout: Layout, delta: Delta, shard_table, stream=None) -> None:
     """Enqueue one apply.  `shard_table` = layout.shard_table(shards)."""
     _check(lib().dte_apply(layout._h, C.byref(delta.struct), shard_table, _stream_ptr(stream)))
+
+
+# dte_chunk_ref as a numpy record: {byte_offset u64, list u32, first_entry u32}
+CHUNK_REF_DTYPE = np.dtype([("byte_offset", np.uint64), ("list", np.uint32), ("first_entry", np.uint32)])
+
+
+class ChunkStream:
+    """Caller-owned device buffers of one serialised delta (see dte_pack_chunks in dte.h)."""
+
+    def __init__(self, n_lists: int, entries: int, chunk_entries: int, fmt: int, device):
+        L = lib()
+        dev = torch.device(device)
+        self.chunk_entries, self.format = int(chunk_entries), int(fmt)
+        self.directory_capacity = int(L.dte_chunk_count_bound(n_lists, int(entries), self.chunk_entries))
+        self.stream_capacity = int(L.dte_chunk_bytes_bound(n_lists, int(entries), self.chunk_entries, self.format))
+        self.stream = torch.empty(max(16, self.stream_capacity), dtype=torch.uint8, device=dev)
+        # 16 bytes per directory entry, one entry more than chunks
+        self.directory = torch.zeros(2 * (self.directory_capacity + 1), dtype=torch.int64, device=dev)
+        self.info = torch.zeros(4, dtype=torch.int64, device=dev)
+
+    def to_host(self):
+        """(stream uint8[bytes], directory records[n_chunks + 1], info) - synchronises."""
+        info = self.info.cpu().numpy().astype(np.uint64)
+        if int(info[2]) & DTE_DEV_OVERFLOW:
+            return np.zeros(0, np.uint8), np.zeros(0, CHUNK_REF_DTYPE), info
+        n_chunks, nbytes = int(info[0]), int(info[1])
+        stream = self.stream[:nbytes].cpu().numpy()
+        directory = self.directory[:2 * (n_chunks + 1)].cpu().numpy().view(CHUNK_REF_DTYPE)
+        return stream, directory, info
+
+
+def dte_pack_chunks(layout: Layout, delta: Delta, out: ChunkStream, stream=None) -> None:
+    """Serialise a complete extract result into `out` (sizes are found on the device)."""
+    _check(lib().dte_pack_chunks(layout._h, C.byref(delta.struct), out.chunk_entries, out.format,
+                                 out.stream.data_ptr(), out.stream_capacity, out.directory.data_ptr(),
+                                 out.directory_capacity, out.info.data_ptr(), _stream_ptr(stream)))
+
+
+def dte_unpack_chunks(layout: Layout, stream_bytes: torch.Tensor, directory: torch.Tensor, n_chunks: int,
+                      delta: Delta, stream=None, nbytes: Optional[int] = None) -> None:
+    """Verify and decode a chunk stream into `delta` (delta.list_ptr must hold the manifest's list
+    boundaries).  `stream_bytes`: uint8 device tensor; `directory`: device tensor holding
+    n_chunks + 1 dte_chunk_ref records."""
+    assert stream_bytes.dtype == torch.uint8 and stream_bytes.is_contiguous() and stream_bytes.device == layout.device
+    assert directory.is_contiguous() and directory.device == layout.device
+    assert directory.numel() * directory.element_size() >= 16 * (int(n_chunks) + 1)
+    n = stream_bytes.numel() if nbytes is None else int(nbytes)
+    _check(lib().dte_unpack_chunks(layout._h, stream_bytes.data_ptr(), n, directory.data_ptr(), int(n_chunks),
+                                   C.byref(delta.struct), _stream_ptr(stream)))
 
 
 class HostResult:

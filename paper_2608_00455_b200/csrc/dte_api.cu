@@ -1,5 +1,5 @@
-// C entry points that enqueue the kernels: dte_extract_delta, dte_apply and the
-// host-buffer variant dte_extract_delta_host.
+// C entry points that enqueue the kernels: the extract variants, dte_apply, dte_op_counts,
+// the chunk codec and the host-buffer variant dte_extract_delta_host.
 #include <cmath>
 #include <cstring>
 #include <limits>
@@ -256,6 +256,75 @@ extern "C" dte_status dte_op_counts(const dte_layout* layout, const dte_delta* d
     DeviceGuard g(layout->device);
     return launch_op_counts(layout->d_op_ranges, layout->n_ops, delta->offsets, delta->list_ptr, counts,
                             (cudaStream_t)cuda_stream);
+}
+
+// ---- chunk codec -------------------------------------------------------------------------
+extern "C" uint64_t dte_chunk_count_bound(size_t n_lists, uint64_t entries, uint32_t chunk_entries) {
+    return chunk_entries ? entries / chunk_entries + n_lists : 0;
+}
+
+extern "C" uint64_t dte_chunk_bytes_bound(size_t n_lists, uint64_t entries, uint32_t chunk_entries,
+                                          uint32_t format) {
+    // per chunk: the header and at most 15 (plain) or 6 * 15 (byte planes) bytes of padding
+    const uint64_t pad = format == DTE_CHUNK_PLAIN ? 15 : 90;
+    return 6 * entries + dte_chunk_count_bound(n_lists, entries, chunk_entries) * (DTE_CHUNK_HEADER_BYTES + pad);
+}
+
+extern "C" dte_status dte_pack_chunks(const dte_layout* layout, const dte_delta* delta, uint32_t chunk_entries,
+                                      uint32_t format, void* stream, uint64_t stream_capacity,
+                                      dte_chunk_ref* directory, uint64_t directory_capacity,
+                                      uint64_t* info, void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    dte_status s = check_delta(delta);
+    if (s != DTE_OK) return s;
+    if (chunk_entries < 8 || chunk_entries % 8 != 0 || chunk_entries > DTE_CHUNK_MAX_ENTRIES)
+        return fail(DTE_ERR_INVALID_ARG, "chunk_entries must be a multiple of 8 in [8, DTE_CHUNK_MAX_ENTRIES]");
+    if (format > DTE_CHUNK_BYTE_PLANES) return fail(DTE_ERR_INVALID_ARG, "unknown chunk format");
+    if (!directory || !info) return fail(DTE_ERR_INVALID_ARG, "directory / info is null");
+    if (stream_capacity && !stream) return fail(DTE_ERR_INVALID_ARG, "stream is null with capacity > 0");
+    if ((uintptr_t)stream & 15u) return fail(DTE_ERR_INVALID_ARG, "stream must be 16-byte aligned");
+    DeviceGuard g(layout->device);
+    PackParams p;
+    p.offsets = delta->offsets;
+    p.values = delta->values;
+    p.list_ptr = delta->list_ptr;
+    p.counters = delta->counters;
+    p.capacity = delta->capacity;
+    p.n_lists = layout->n_lists;
+    p.chunk_entries = chunk_entries;
+    p.format = format;
+    p.stream = (uint8_t*)stream;
+    p.stream_capacity = stream_capacity;
+    p.dir = directory;
+    p.dir_capacity = directory_capacity;
+    p.info = info;
+    return launch_pack_chunks(p, layout->device, (cudaStream_t)cuda_stream);
+}
+
+extern "C" dte_status dte_unpack_chunks(const dte_layout* layout, const void* stream, uint64_t stream_bytes,
+                                        const dte_chunk_ref* directory, uint64_t n_chunks,
+                                        const dte_delta* out, void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    dte_status s = check_delta(out);
+    if (s != DTE_OK) return s;
+    if (!directory) return fail(DTE_ERR_INVALID_ARG, "directory is null");
+    if (stream_bytes && !stream) return fail(DTE_ERR_INVALID_ARG, "stream is null with bytes > 0");
+    if ((uintptr_t)stream & 15u) return fail(DTE_ERR_INVALID_ARG, "stream must be 16-byte aligned");
+    DeviceGuard g(layout->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
+    UnpackParams p;
+    p.stream = (const uint8_t*)stream;
+    p.stream_bytes = stream_bytes;
+    p.dir = directory;
+    p.n_chunks = n_chunks;
+    p.n_lists = layout->n_lists;
+    p.list_ptr = out->list_ptr;
+    p.offsets = out->offsets;
+    p.values = out->values;
+    p.capacity = out->capacity;
+    p.counters = out->counters;
+    return launch_unpack_chunks(p, layout->device, st);
 }
 
 extern "C" dte_status dte_extract_delta_host(const dte_layout* layout, const float* const* theta_h,

@@ -21,10 +21,11 @@ __global__ void __launch_bounds__(kApplyThreads) apply_kernel(const ApplyParams 
     __syncthreads();
     const uint64_t* lp = cached ? s_ptr : p.list_ptr;
     const uint64_t total = lp[L];
-    if (total > p.capacity || (p.counters[2] & DTE_DEV_OVERFLOW)) {
+    const uint64_t dev_bits = p.counters[2];
+    if (total > p.capacity || (dev_bits & (DTE_DEV_OVERFLOW | DTE_DEV_CORRUPT))) {
         // the lists are incomplete: writing part of a version would leave the shard in a
         // state that is neither the old nor the new one
-        if (blockIdx.x == 0 && threadIdx.x == 0)
+        if (blockIdx.x == 0 && threadIdx.x == 0 && !(dev_bits & DTE_DEV_CORRUPT))
             atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_OVERFLOW);
         return;
     }

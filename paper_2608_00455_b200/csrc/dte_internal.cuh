@@ -138,6 +138,34 @@ struct OpRange {
     uint64_t begin, end;   // receiver-local flat range [begin, end); begin == end for empty overlaps
 };
 
+// Chunk codec (storage-mediated path).
+struct PackParams {
+    const uint32_t* offsets;
+    const uint16_t* values;
+    const uint64_t* list_ptr;
+    const uint64_t* counters;   // of the delta: an overflowed delta is not packed
+    uint64_t capacity;          // of the delta
+    uint32_t n_lists, chunk_entries, format;
+    uint8_t* stream;
+    uint64_t stream_capacity;
+    dte_chunk_ref* dir;
+    uint64_t dir_capacity;      // chunks the directory can hold (it has one more entry)
+    uint64_t* info;
+};
+
+struct UnpackParams {
+    const uint8_t* stream;
+    uint64_t stream_bytes;
+    const dte_chunk_ref* dir;
+    uint64_t n_chunks;
+    uint32_t n_lists;
+    const uint64_t* list_ptr;
+    uint32_t* offsets;
+    uint16_t* values;
+    uint64_t capacity;
+    uint64_t* counters;   // {entries written, chunks accepted, DTE_DEV_* bits, chunks rejected}
+};
+
 void set_error(const std::string& msg);
 dte_status cuda_fail(cudaError_t e, const char* what);
 
@@ -150,6 +178,8 @@ dte_status cuda_fail(cudaError_t e, const char* what);
 dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, cudaStream_t st);
 dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
+dte_status launch_pack_chunks(const PackParams& p, int device, cudaStream_t st);
+dte_status launch_unpack_chunks(const UnpackParams& p, int device, cudaStream_t st);
 dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const uint32_t* offsets,
                             const uint64_t* list_ptr, uint64_t* counts, cudaStream_t st);
 

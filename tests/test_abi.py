@@ -58,3 +58,20 @@ def test_compute_calls_fail_loudly_without_a_gpu():
         pytest.skip("GPU present")
     with pytest.raises(RuntimeError):
         dte.Layout([(4, 4)], [16], [(0, 0, 0, 0, 4, 4, 0, 4, 0, 0)])
+
+
+@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("chunk_entries", [8, 64, 4096])
+def test_chunk_bounds_cover_what_the_oracle_writes(fmt, chunk_entries):
+    # host-only sizing helpers: never smaller than the stream the oracle serialises
+    rng = np.random.default_rng(chunk_entries + fmt)
+    L = dte.lib()
+    for _ in range(20):
+        lens = rng.integers(0, 3 * chunk_entries + 2, rng.integers(1, 12))
+        lp = np.concatenate([[0], np.cumsum(lens)]).astype(np.uint64)
+        n = int(lp[-1])
+        stream, d = oracle.pack_chunks(lp, np.arange(n, dtype=np.uint32), np.zeros(n, np.uint16),
+                                       chunk_entries, fmt)
+        assert d.shape[0] - 1 <= L.dte_chunk_count_bound(lens.size, n, chunk_entries)
+        assert stream.size <= L.dte_chunk_bytes_bound(lens.size, n, chunk_entries, fmt)
+    assert L.dte_chunk_count_bound(3, 100, 0) == 0

@@ -125,6 +125,10 @@ def test_every_corrupted_payload_byte_and_header_field_is_rejected(fmt):
     bad_dir = d.copy()
     bad_dir[0, 2] = 8                              # directory and header disagree
     assert oracle.unpack_chunks(stream, bad_dir, LP)[2] == 1
+    for row, value in ((1, int(d[1, 0]) + 8), (2, stream.size + 16), (1, 16)):
+        bad_dir = d.copy()                         # chunk off its boundary / past the end / too short
+        bad_dir[row, 0] = value
+        assert oracle.unpack_chunks(stream, bad_dir, LP)[2] >= 1
 
 
 def test_empty_delta_has_no_chunks():
