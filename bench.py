@@ -234,6 +234,40 @@ def run_reference(args, rank):
     print(json.dumps(out), flush=True)
 
 
+def time_chunk_codec(dte, lay, delta, M, device, peak, chunk_entries=16384, reps=5):
+    """Storage-path leg (not part of the step): serialise the step's lists into byte-plane chunks
+    and read them back, timed with CUDA events; algorithmic bytes = lists + stream, each way."""
+    fmt = dte.DTE_CHUNK_BYTE_PLANES
+    cs = dte.ChunkStream(lay.num_lists, M, chunk_entries, fmt, device)
+    back = lay.new_delta(M)
+    back.list_ptr.copy_(delta.list_ptr)
+    stream = torch.cuda.current_stream()
+    dte.dte_pack_chunks(lay, delta, cs)
+    torch.cuda.synchronize()
+    n_chunks, nbytes, bits, _ = (int(x) for x in cs.info.cpu().tolist())
+    if bits:
+        return {"error": f"pack status bits {bits}"}
+    flush = torch.empty(1 << 28, dtype=torch.uint8, device=device)
+    t_pack, t_unpack = [], []
+    for _ in range(reps):
+        e = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        flush.zero_()
+        e[0].record(stream); dte.dte_pack_chunks(lay, delta, cs); e[1].record(stream)
+        flush.zero_()
+        e[2].record(stream); dte.dte_unpack_chunks(lay, cs.stream, cs.directory, n_chunks, back, nbytes=nbytes); e[3].record(stream)
+        torch.cuda.synchronize()
+        t_pack.append(e[0].elapsed_time(e[1])); t_unpack.append(e[2].elapsed_time(e[3]))
+    same = bool(torch.equal(back.offsets[:M], delta.offsets[:M]) and torch.equal(back.values[:M], delta.values[:M]))
+    counters = back.counters.cpu().tolist()
+    moved = 6.0 * M + nbytes
+    pk, un = sum(t_pack) / reps, sum(t_unpack) / reps
+    return {"format": "byte planes", "chunk_entries": chunk_entries, "chunks": n_chunks, "stream_bytes": nbytes,
+            "pack_ms": pk, "unpack_ms": un, "pack_GBps": moved / (pk * 1e-3) / 1e9,
+            "unpack_GBps": moved / (un * 1e-3) / 1e9, "pack_frac_of_peak": moved / (pk * 1e-3) / 1e9 / peak,
+            "unpack_frac_of_peak": moved / (un * 1e-3) / 1e9 / peak, "round_trip_equal": same,
+            "chunks_rejected": int(counters[3]), "gpu_launches": 3 * reps, "l2": "256 MB written before each timed call"}
+
+
 def aggregate_over_ranks(ms_local: float, units_local: float, dist, device):
     """Weak scaling: the job's time is the slowest rank's, its units the sum over ranks."""
     if dist is None:
@@ -260,6 +294,7 @@ def main():
                     help="association of the generator's forward AdamW step (only changes the inputs)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-codec", action="store_true", help="skip the storage path's chunk codec leg")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -373,6 +408,12 @@ def main():
     if NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT is not None:
         traffic = NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT * N
 
+    # ---- storage path: chunk codec on the step's lists (outside the timed step) ------------------
+    codec = None
+    if rank == 0 and not args.no_codec:
+        codec = time_chunk_codec(dte, lay, delta, M, device, peak)
+        log(f"[bench] chunk codec: {codec}")
+
     # ---- end to end through the host-buffer entry point -----------------------------------------
     e2e = None
     if not args.no_e2e:
@@ -418,6 +459,7 @@ def main():
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "peak_source": peak_kind, "kernel": "extract_kernel"},
             "reconstruction_vs_truth": {"false_negatives": fn, "false_positives": fp, "variant": wl.variant},
+            "chunk_codec": codec,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
             "launch": lay.last_launch(),
         }

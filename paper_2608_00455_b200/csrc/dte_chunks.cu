@@ -175,13 +175,27 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_pack_kernel(const PackPar
         if (p.format == DTE_CHUNK_PLAIN) {
             uint32_t* out_o = reinterpret_cast<uint32_t*>(pay);
             uint16_t* out_v = reinterpret_cast<uint16_t*>(pay + 4ull * count);
-            for (uint32_t i = tid; i < count; i += kChunkThreads) {
-                const uint32_t o = src_o[i];
-                const uint32_t v = src_v[i];
-                out_o[i] = o;
-                out_v[i] = (uint16_t)v;
-                add_word(acc, o, pb - 4 * i);
-                add_half(acc, v, pb - (4 * count + 2 * i));
+            // four coalesced entries per thread in flight
+            for (uint32_t i0 = tid; i0 < count; i0 += 4 * kChunkThreads) {
+                uint32_t o[4], v[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t i = i0 + e * kChunkThreads;
+                    if (i < count) {
+                        o[e] = src_o[i];
+                        v[e] = src_v[i];
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t i = i0 + e * kChunkThreads;
+                    if (i < count) {
+                        out_o[i] = o[e];
+                        out_v[i] = (uint16_t)v[e];
+                        add_word(acc, o[e], pb - 4 * i);
+                        add_half(acc, v[e], pb - (4 * count + 2 * i));
+                    }
+                }
             }
             for (uint32_t q = 6 * count + tid; q < pb; q += kChunkThreads) pay[q] = 0;
         } else {
@@ -257,12 +271,23 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_unpack_kernel(const Unpac
         const uint8_t* pay = p.stream + begin + kHeaderBytes;
         if (ok) {   // pass 1: checksum of what is about to be decoded
             Sums acc{0, 0};
-            for (uint32_t q = 16 * tid; q < pb; q += 16 * kChunkThreads) {
-                const uint4 w = *reinterpret_cast<const uint4*>(pay + q);
-                add_word(acc, w.x, pb - q);
-                add_word(acc, w.y, pb - q - 4);
-                add_word(acc, w.z, pb - q - 8);
-                add_word(acc, w.w, pb - q - 12);
+            for (uint32_t q0 = 16 * tid; q0 < pb; q0 += 4 * 16 * kChunkThreads) {
+                uint4 w[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t q = q0 + e * 16 * kChunkThreads;
+                    w[e] = q < pb ? *reinterpret_cast<const uint4*>(pay + q) : make_uint4(0, 0, 0, 0);
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t q = q0 + e * 16 * kChunkThreads;
+                    if (q < pb) {
+                        add_word(acc, w[e].x, pb - q);
+                        add_word(acc, w[e].y, pb - q - 4);
+                        add_word(acc, w[e].z, pb - q - 8);
+                        add_word(acc, w[e].w, pb - q - 12);
+                    }
+                }
             }
             const Sums tot = block_sum(acc, s_red);
             ok = finish_checksum(tot, h, pb) == h[6];
@@ -278,9 +303,25 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_unpack_kernel(const Unpac
         if (format == DTE_CHUNK_PLAIN) {
             const uint32_t* in_o = reinterpret_cast<const uint32_t*>(pay);
             const uint16_t* in_v = reinterpret_cast<const uint16_t*>(pay + 4ull * count);
-            for (uint32_t i = tid; i < count; i += kChunkThreads) {
-                out_o[i] = in_o[i];
-                out_v[i] = in_v[i];
+            for (uint32_t i0 = tid; i0 < count; i0 += 4 * kChunkThreads) {
+                uint32_t o[4];
+                uint16_t v[4];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t i = i0 + e * kChunkThreads;
+                    if (i < count) {
+                        o[e] = in_o[i];
+                        v[e] = in_v[i];
+                    }
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t i = i0 + e * kChunkThreads;
+                    if (i < count) {
+                        out_o[i] = o[e];
+                        out_v[i] = v[e];
+                    }
+                }
             }
         } else {
             const uint32_t P = (uint32_t)round16(count);
