@@ -168,6 +168,28 @@ class Delta:
         self.struct = DeltaStruct(self.offsets.data_ptr(), self.values.data_ptr(), self.capacity,
                                   self.list_ptr.data_ptr(), self.counters.data_ptr())
 
+    @classmethod
+    def wrap(cls, list_ptr, offsets: torch.Tensor, values: torch.Tensor) -> "Delta":
+        """A delta around lists that already exist on the device (received from a peer or decoded
+        from chunks): `list_ptr` host array of n_lists + 1 boundaries, `offsets` int32 / `values`
+        int16 device tensors holding list_ptr[-1] entries.  No copy of the entries."""
+        lp = np.ascontiguousarray(list_ptr, dtype=np.uint64)
+        total = int(lp[-1])
+        assert offsets.dtype == torch.int32 and values.dtype == torch.int16
+        assert offsets.is_contiguous() and values.is_contiguous() and offsets.device == values.device
+        assert offsets.numel() >= total and values.numel() >= total
+        self = cls.__new__(cls)
+        dev = offsets.device
+        self.capacity, self.n_lists = total, lp.size - 1
+        # zero-entry deltas still need valid pointers
+        self.offsets = offsets if total else torch.empty(1, dtype=torch.int32, device=dev)
+        self.values = values if total else torch.empty(1, dtype=torch.int16, device=dev)
+        self.list_ptr = torch.from_numpy(lp.astype(np.int64)).to(dev)
+        self.counters = torch.tensor([total, 0, 0, 0], dtype=torch.int64, device=dev)
+        self.struct = DeltaStruct(self.offsets.data_ptr(), self.values.data_ptr(), self.capacity,
+                                  self.list_ptr.data_ptr(), self.counters.data_ptr())
+        return self
+
     # host views (synchronise)
     def total(self) -> int:
         return int(self.counters[0].item())

@@ -420,3 +420,28 @@ def canonical_plan(names: Sequence[str], shapes: Sequence[Sequence[int]]) -> Pla
         t = p.add_tensor(name, shape)
         p.replicated(name, t, 0)
     return p
+
+
+def tensor_senders(plan: Plan, tp_send: int, dp: int = 1) -> List[int]:
+    """Sender index of every source tensor of a Megatron-Core-native plan, from its name:
+    `.tp{s}` shards belong to TP rank s, `.dp{d}` slices to data-parallel rank d, tensors
+    replicated over TP ranks are taken from TP rank 0.  Sender index = s * dp + d."""
+    import re
+    out = []
+    for name in plan.tensor_names:
+        s = re.search(r"\.tp(\d+)", name)
+        d = re.search(r"\.dp(\d+)", name)
+        s, d = int(s.group(1)) if s else 0, int(d.group(1)) if d else 0
+        assert s < tp_send and d < dp
+        out.append(s * dp + d)
+    return out
+
+
+def sender_subplan(plan: Plan, owners: Sequence[int], sender: int) -> Plan:
+    """The plan as sender `sender` executes it: every tensor and shard keeps its index, only the
+    operations whose source tensor the sender owns remain (in plan order)."""
+    q = Plan(tensor_names=plan.tensor_names, tensor_shapes=plan.tensor_shapes, shard_names=plan.shard_names,
+             shard_receivers=plan.shard_receivers, shard_numels=plan.shard_numels)
+    q.slice_ranges = plan.slice_ranges
+    q.ops = [op for op in plan.ops if owners[op[0]] == sender]
+    return q
