@@ -109,6 +109,9 @@ def build_workload(name: str, device):
         return configs.config2()
     if name == "config4":
         return configs.config4(device)
+    if name.startswith("moe:"):          # moe:<receiver TP>:<EP>[:<layers>]  (config 4's state, other inference layout)
+        f = [int(x) for x in name.split(":")[1:]]
+        return configs.config4(device, n_layers=f[2] if len(f) > 2 else 12, tp=f[0], ep=f[1])
     raise SystemExit(f"unknown workload {name}")
 
 

@@ -105,9 +105,10 @@ def config3_mcore(device, tp_send=2, tp_recv=2, dp=1, n_layers=36, seed=1234, di
 
 
 def config4(device, n_layers=12, seed=1234, dims=P.QWEN3_30B_A3B, target=0.015,
-            tokens=64) -> Workload:
-    """Qwen3-30B-A3B-shaped slice; experts' state scaled by a Zipf routing histogram."""
-    plan = P.qwen3_moe_plan(n_layers, 4, 4, dims)
+            tokens=64, tp=4, ep=4) -> Workload:
+    """Qwen3-30B-A3B-shaped slice; experts' state scaled by a Zipf routing histogram.
+    tp > ep: tensor-parallel experts; tp > 4 (the KV head count): replicated KV heads."""
+    plan = P.qwen3_moe_plan(n_layers, tp, ep, dims)
     w = calibrate_sigma_g(WEIGHT, HP_T500, seed, device, target)
     specs = _specs(plan, w)
     cold = 0
@@ -120,7 +121,7 @@ def config4(device, n_layers=12, seed=1234, dims=P.QWEN3_30B_A3B, target=0.015,
             if name.startswith(f"layers.{l}.experts."):
                 e = int(name.split(".")[3])
                 specs[p] = replace(w, scale=float(c[e] / mean))
-    wl = Workload(f"qwen3-30b-a3b.first{n_layers}.tp4ep4", plan, HP_T500, specs, seed)
+    wl = Workload(f"qwen3-30b-a3b.first{n_layers}.tp{tp}ep{ep}", plan, HP_T500, specs, seed)
     wl.notes.update(sigma_g=w.sigma_g, cold_experts=cold, routing_tokens=tokens)
     return wl
 

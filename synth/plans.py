@@ -98,6 +98,25 @@ class Plan:
             at += nr
         return k
 
+    def fused_qkv(self, name: str, q: int, k: int, v: int, r: int, R: int, hkv: int, hd: int) -> int:
+        """Fused qkv_proj of receiver r split by head.  With R <= hkv every receiver takes
+        hkv/R KV heads (plain row blocks).  With R > hkv (R a multiple of hkv) the KV heads are
+        replicated: receiver r holds KV head r // (R / hkv) whole, next to its own Q heads, so
+        R / hkv receivers emit the same K and V entries."""
+        if hkv % R == 0:
+            return self.fused_rows(name, [q, k, v], r, R)
+        assert R % hkv == 0, "receivers must be a multiple of the KV heads to replicate them"
+        cols = self.tensor_shapes[q][1]
+        q_rows = self.tensor_shapes[q][0]
+        assert q_rows % R == 0 and self.tensor_shapes[k] == (hkv * hd, cols) == self.tensor_shapes[v]
+        nq = q_rows // R
+        j = r // (R // hkv)
+        dst = self.add_shard(f"r{r}.{name}", r, (nq + 2 * hd) * cols)
+        self.add_op(q, dst, (r * nq, 0), (nq, cols), 0, cols, (0, 0))
+        self.add_op(k, dst, (j * hd, 0), (hd, cols), 0, cols, (nq, 0))
+        self.add_op(v, dst, (j * hd, 0), (hd, cols), 0, cols, (nq + hd, 0))
+        return dst
+
     def row_parallel(self, name: str, src: int, r: int, R: int) -> int:
         """Column block [r*I/R, (r+1)*I/R) of the source (o_proj, down_proj)."""
         n0, n1 = self.tensor_shapes[src]
@@ -107,18 +126,30 @@ class Plan:
         self.add_op(src, k, (0, r * w), (n0, w), 0, w, (0, 0))
         return k
 
-    def expert_stack(self, name: str, per_expert_srcs: Sequence[Sequence[int]], r: int) -> int:
-        """Stacked local experts: dst[l] = row-concatenation of per_expert_srcs[l]."""
-        cols = self.tensor_shapes[per_expert_srcs[0][0]][1]
-        rows_per = sum(self.tensor_shapes[s][0] for s in per_expert_srcs[0])
+    def expert_stack(self, name: str, per_expert_srcs: Sequence[Sequence[int]], r: int,
+                     row_part: Tuple[int, int] = (0, 1), col_part: Tuple[int, int] = (0, 1)) -> int:
+        """Stacked local experts: dst[l] = row-concatenation of per_expert_srcs[l].
+
+        With expert tensor parallelism each source contributes only its row block
+        row_part = (i, n) (w13: gate and up split along the intermediate dimension) or its
+        column block col_part = (i, n) (w2: down_proj split along its input dimension)."""
+        (ri, rn), (ci, cn) = row_part, col_part
+        n1_full = self.tensor_shapes[per_expert_srcs[0][0]][1]
+        assert n1_full % cn == 0
+        cols = n1_full // cn
+        rows_per = 0
+        for s in per_expert_srcs[0]:
+            assert self.tensor_shapes[s][0] % rn == 0
+            rows_per += self.tensor_shapes[s][0] // rn
         k = self.add_shard(f"r{r}.{name}", r, len(per_expert_srcs) * rows_per * cols)
         for l, srcs in enumerate(per_expert_srcs):
             at = 0
             for s in srcs:
                 n0, n1 = self.tensor_shapes[s]
-                assert n1 == cols
-                self.add_op(s, k, (0, 0), (n0, n1), l * rows_per * cols, cols, (at, 0))
-                at += n0
+                assert n1 == n1_full
+                nr = n0 // rn
+                self.add_op(s, k, (ri * nr, ci * cols), (nr, cols), l * rows_per * cols, cols, (at, 0))
+                at += nr
             assert at == rows_per
         return k
 
@@ -157,8 +188,8 @@ def _dense_layer_tensors(p: Plan, pre: str, d: dict) -> dict:
     return t
 
 
-def _dense_layer_shards(p: Plan, pre: str, t: dict, r: int, R: int) -> None:
-    p.fused_rows(pre + "qkv_proj", [t["q"], t["k"], t["v"]], r, R)
+def _dense_layer_shards(p: Plan, pre: str, t: dict, r: int, R: int, d: dict) -> None:
+    p.fused_qkv(pre + "qkv_proj", t["q"], t["k"], t["v"], r, R, d["kv_heads"], d["head_dim"])
     p.row_parallel(pre + "o_proj", t["o"], r, R)
     p.fused_rows(pre + "gate_up_proj", [t["gate"], t["up"]], r, R)
     p.row_parallel(pre + "down_proj", t["down"], r, R)
@@ -180,7 +211,7 @@ def qwen3_dense_plan(n_layers: int, tp: int, with_embeddings: bool, dims: dict =
         head = p.add_tensor("lm_head", (dims["vocab"], dims["hidden"]))
     for r in range(tp):
         for l, t in enumerate(layers):
-            _dense_layer_shards(p, f"layers.{l}.", t, r, tp)
+            _dense_layer_shards(p, f"layers.{l}.", t, r, tp, dims)
         if with_embeddings:
             p.fused_rows("embed_tokens", [emb], r, tp)
             p.fused_rows("lm_head", [head], r, tp)
@@ -188,8 +219,13 @@ def qwen3_dense_plan(n_layers: int, tp: int, with_embeddings: bool, dims: dict =
 
 
 def qwen3_moe_plan(n_layers: int, tp: int = 4, ep: int = 4, dims: dict = QWEN3_30B_A3B) -> Plan:
-    """Qwen3-30B-A3B-shaped layers: attention TP, experts EP (stacked w13 / w2)."""
-    assert tp == ep, "one receiver set: receiver r holds TP rank r and EP rank r"
+    """Qwen3-30B-A3B-shaped layers: attention TP, experts EP (stacked w13 / w2).
+
+    One receiver set of `tp` ranks.  With ep < tp the experts are also tensor-parallel: the
+    tp / ep ranks of an expert-parallel group split every local expert (gate and up by rows,
+    down by columns).  With tp above the KV head count the KV heads are replicated."""
+    assert tp % ep == 0, "receiver r holds TP rank r, EP rank r // (tp/ep), expert-TP rank r % (tp/ep)"
+    etp = tp // ep
     p = Plan()
     h, hd, E, F = dims["hidden"], dims["head_dim"], dims["experts"], dims["moe_inter"]
     layers = []
@@ -216,13 +252,14 @@ def qwen3_moe_plan(n_layers: int, tp: int = 4, ep: int = 4, dims: dict = QWEN3_3
     for r in range(tp):
         for l, t in enumerate(layers):
             pre = f"layers.{l}."
-            p.fused_rows(pre + "qkv_proj", [t["q"], t["k"], t["v"]], r, tp)
+            p.fused_qkv(pre + "qkv_proj", t["q"], t["k"], t["v"], r, tp, dims["kv_heads"], hd)
             p.row_parallel(pre + "o_proj", t["o"], r, tp)
             for n in ("router", "q_norm", "k_norm", "ln1", "ln2"):
                 p.replicated(pre + n, t[n], r)
-            mine = t["experts"][r * e_loc:(r + 1) * e_loc]
-            p.expert_stack(pre + "w13", [(g, u) for g, u, _ in mine], r)
-            p.expert_stack(pre + "w2", [(dn,) for _, _, dn in mine], r)
+            g_ep, g_tp = r // etp, r % etp
+            mine = t["experts"][g_ep * e_loc:(g_ep + 1) * e_loc]
+            p.expert_stack(pre + "w13", [(g, u) for g, u, _ in mine], r, row_part=(g_tp, etp))
+            p.expert_stack(pre + "w2", [(dn,) for _, _, dn in mine], r, col_part=(g_tp, etp))
     return p
 
 

@@ -58,12 +58,16 @@ def test_config1_single_matrix_tp2():
     assert stale <= 8
 
 
-@pytest.mark.parametrize("name", ["dense_tp4", "dense_tp2", "moe", "matrix_tp3_ragged"])
+@pytest.mark.parametrize("name", ["dense_tp4", "dense_tp2", "moe", "matrix_tp3_ragged",
+                                  "moe_tp8_ep4_replicated_kv", "dense_tp8_replicated_kv"])
 def test_small_plans_with_ragged_widths(name):
     plan = {
         "dense_tp4": lambda: plans.qwen3_dense_plan(2, 4, True, configs.SMALL_DENSE),
         "dense_tp2": lambda: plans.qwen3_dense_plan(3, 2, True, configs.SMALL_DENSE),
         "moe": lambda: plans.qwen3_moe_plan(2, 4, 4, configs.SMALL_MOE),
+        # receivers above the KV head count (KV heads replicated) and tensor-parallel experts
+        "moe_tp8_ep4_replicated_kv": lambda: plans.qwen3_moe_plan(2, 8, 4, configs.SMALL_MOE),
+        "dense_tp8_replicated_kv": lambda: plans.qwen3_dense_plan(2, 8, True, dict(configs.SMALL_DENSE, vocab=3008)),
         # 4099 x 1027: nothing is a multiple of 4 -> scalar tiles, ragged tails
         "matrix_tp3_ragged": lambda: plans.single_matrix_plan(3 * 1367, 1027, 3),
     }[name]()

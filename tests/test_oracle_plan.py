@@ -33,6 +33,8 @@ SMALL_PLANS = {
     "dense_tp4": lambda: plans.qwen3_dense_plan(2, 4, True, configs.SMALL_DENSE),
     "dense_tp2": lambda: plans.qwen3_dense_plan(1, 2, True, configs.SMALL_DENSE),
     "moe": lambda: plans.qwen3_moe_plan(2, 4, 4, configs.SMALL_MOE),
+    "moe_tp8_ep4_replicated_kv": lambda: plans.qwen3_moe_plan(1, 8, 4, configs.SMALL_MOE),
+    "dense_tp8_replicated_kv": lambda: plans.qwen3_dense_plan(1, 8, False, configs.SMALL_DENSE),
 }
 
 
@@ -130,6 +132,44 @@ def test_moe_plan_equals_stacked_experts():
         assert torch.equal(shards[k2], w2.reshape(-1))
         kr = plan.shard_names.index(f"r{r}.layers.0.router")
         assert torch.equal(shards[kr], dense[name_to_p["layers.0.router"]].reshape(-1))
+
+
+def test_replicated_kv_heads_and_expert_tensor_parallelism_equal_textbook_sharding():
+    # receivers above the KV head count hold one whole KV head each (head r // replicas), and an
+    # expert-parallel group of tp/ep ranks splits its experts: gate/up by rows, down by columns
+    d = configs.SMALL_MOE                               # 8 Q heads, 4 KV heads, 16 experts
+    tp, ep = 8, 4
+    etp, hd, hkv = tp // ep, d["head_dim"], d["kv_heads"]
+    plan = plans.qwen3_moe_plan(1, tp, ep, d)
+    g = torch.Generator().manual_seed(3)
+    dense = [torch.randint(-30000, 30000, s, generator=g, dtype=torch.int16) for s in plan.tensor_shapes]
+    shards = [torch.zeros(n, dtype=torch.int16) for n in plan.shard_numels]
+    plans.scatter_dense(plan, dense, shards)
+    at = {n: dense[i] for i, n in enumerate(plan.tensor_names)}
+    e_loc = d["experts"] // ep
+    for r in range(tp):
+        q = at["layers.0.q_proj"].chunk(tp, 0)[r]
+        j = r // (tp // hkv)
+        k = at["layers.0.k_proj"].view(hkv, hd, -1)[j]
+        v = at["layers.0.v_proj"].view(hkv, hd, -1)[j]
+        got = shards[plan.shard_names.index(f"r{r}.layers.0.qkv_proj")]
+        assert torch.equal(got, torch.cat([q, k, v], 0).reshape(-1))
+        experts = range((r // etp) * e_loc, (r // etp + 1) * e_loc)
+        w13 = torch.stack([torch.cat([at[f"layers.0.experts.{e}.gate_proj"].chunk(etp, 0)[r % etp],
+                                      at[f"layers.0.experts.{e}.up_proj"].chunk(etp, 0)[r % etp]], 0) for e in experts])
+        w2 = torch.stack([at[f"layers.0.experts.{e}.down_proj"].chunk(etp, 1)[r % etp] for e in experts])
+        assert torch.equal(shards[plan.shard_names.index(f"r{r}.layers.0.w13")], w13.reshape(-1))
+        assert torch.equal(shards[plan.shard_names.index(f"r{r}.layers.0.w2")], w2.reshape(-1))
+    # the dense model the same way: Qwen3-8B-like heads at TP 8 with 4 KV heads
+    dd = configs.SMALL_DENSE
+    dp = plans.qwen3_dense_plan(1, 8, False, dd)
+    dense = [torch.randint(-30000, 30000, s, generator=g, dtype=torch.int16) for s in dp.tensor_shapes]
+    shards = [torch.zeros(n, dtype=torch.int16) for n in dp.shard_numels]
+    plans.scatter_dense(dp, dense, shards)
+    for r in range(8):
+        want = torch.cat([dense[0].chunk(8, 0)[r], dense[1].view(4, dd["head_dim"], -1)[r // 2],
+                          dense[2].view(4, dd["head_dim"], -1)[r // 2]], 0)
+        assert torch.equal(shards[dp.shard_names.index(f"r{r}.layers.0.qkv_proj")], want.reshape(-1))
 
 
 def test_plan_counts_match_the_full_size_models():
