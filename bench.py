@@ -194,6 +194,58 @@ def time_oracle(wl, st, chosen):
     return time.perf_counter() - t0, res
 
 
+def time_oracle_threads(wl, st, chosen, threads):
+    """The same single-threaded oracle on `threads` host threads, each with a disjoint share of the
+    chosen tensors (largest first onto the least loaded thread); wall-clock of the slowest."""
+    import threading
+    import oracle
+    plan = wl.plan
+    shares = [[] for _ in range(threads)]
+    load = [0] * threads
+    for p in sorted(chosen, key=lambda q: -plan.numel(q)):
+        i = load.index(min(load))
+        shares[i].append(p)
+        load[i] += plan.numel(p)
+    shares = [sorted(s) for s in shares if s]
+    c = oracle.derive_constants(*wl.hp.as_args())
+    jobs = [oracle_inputs(plan, st, share) for share in shares]
+    changed = [0] * len(jobs)
+
+    def work(i):
+        shapes, ops, host = jobs[i]
+        changed[i] = int(oracle.extract(shapes, plan.shard_numels, ops, *host, c)[0][-1])
+
+    ts = [threading.Thread(target=work, args=(i,)) for i in range(len(jobs))]
+    t0 = time.perf_counter()
+    for t in ts: t.start()
+    for t in ts: t.join()
+    dt = time.perf_counter() - t0
+    scanned = int(sum(int((j[1][:, 4] * j[1][:, 5]).sum()) for j in jobs))
+    return dt, scanned, sum(changed), len(jobs)
+
+
+def read_ceiling(dte, device, nbytes=4 << 30, reps=10):
+    """Read-only streaming bandwidth: one launch over a 4 GiB buffer of its own (CUDA events)."""
+    buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
+    buf.random_(0, 256)
+    out = torch.zeros(1, dtype=torch.int64, device=device)
+    stream = torch.cuda.current_stream()
+    for _ in range(3):
+        dte.dte_read_bandwidth_probe(buf, out)
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(reps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        dte.dte_read_bandwidth_probe(buf, out)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms.append(e0.elapsed_time(e1))
+    avg = sum(ms) / len(ms)
+    return {"GBps": nbytes / (avg * 1e-3) / 1e9, "GBps_best": nbytes / (min(ms) * 1e-3) / 1e9, "bytes": nbytes,
+            "launches": reps, "note": "4 GiB buffer, larger than L2, one launch per pass"}
+
+
 def run_reference(args, rank):
     """The CPU oracle, as it stands, on a bounded sample of the same workload."""
     if rank != 0:
@@ -411,6 +463,12 @@ def main():
     if NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT is not None:
         traffic = NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT * N
 
+    # ---- practical ceiling for a read-only kernel: plain streaming reads of the same tensors --------
+    ceiling = None
+    if rank == 0:
+        ceiling = read_ceiling(dte, device)
+        log(f"[bench] read-only streaming ceiling: {ceiling}")
+
     # ---- storage path: chunk codec on the step's lists (outside the timed step) ------------------
     codec = None
     if rank == 0 and not args.no_codec:
@@ -443,6 +501,12 @@ def main():
         cpu = {"value": (12.0 * scanned + 6.0 * m_cpu) / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"first {len(chosen)} source tensors ({scanned} scanned elements) of {wl.name}, extract only, "
                          f"{dt:.1f} s", "elements_per_s": scanned / dt, "lists_equal_gpu": bool(ok)}
+        # the same oracle on every host core, disjoint tensors per thread
+        k = os.cpu_count() or 1
+        dt_k, scanned_k, m_k, used = time_oracle_threads(wl, st, chosen, k)
+        cpu["all_cores"] = {"value": (12.0 * scanned_k + 6.0 * m_k) / dt_k / 1e9, "unit": UNIT, "cores": used,
+                            "seconds": dt_k, "elements_per_s": scanned_k / dt_k,
+                            "sample": "the same tensors, split over the threads largest first"}
 
     if rank == 0:
         out = {
@@ -460,7 +524,9 @@ def main():
                       "GBps_sector_traffic": 70.0 * M / (app_avg * 1e-3) / 1e9,
                       "frac_of_peak_sector_traffic": 70.0 * M / (app_avg * 1e-3) / 1e9 / peak},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": traffic, "peak_source": peak_kind, "kernel": "extract_kernel"},
+                         "traffic": traffic, "peak_source": peak_kind, "kernel": "extract_kernel",
+                         "read_only_ceiling": ceiling,
+                         "frac_of_read_only_ceiling": achieved / ceiling["GBps"] if ceiling else None},
             "reconstruction_vs_truth": {"false_negatives": fn, "false_positives": fp, "variant": wl.variant},
             "chunk_codec": codec,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,

@@ -306,6 +306,13 @@ DTE_API dte_status dte_extract_delta_host(const dte_layout* layout, const float*
                                   uint32_t* offsets_h, uint16_t* values_h, uint64_t* list_ptr_h,
                                   uint64_t* counters_h, void* cuda_stream);
 
+/* Measurement aid, no counterpart in the paper: one read-only streaming pass over `bytes` bytes
+ * of DEVICE memory at `src` (16-byte aligned; a trailing bytes % 16 is ignored), XOR-folding
+ * what it reads into *xor_out (DEVICE, 8 bytes, not cleared).  Timed by the caller, it gives the
+ * read bandwidth ceiling of `device` for a kernel that, like the extract, only reads. */
+DTE_API dte_status dte_read_bandwidth_probe(const void* src, uint64_t bytes, uint64_t* xor_out, int device,
+                                            void* cuda_stream);
+
 /* Static strings. */
 DTE_API const char* dte_status_string(dte_status s);
 /* Message of the calling thread's most recent failed call ("" if none). */

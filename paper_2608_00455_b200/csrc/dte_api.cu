@@ -258,6 +258,14 @@ extern "C" dte_status dte_op_counts(const dte_layout* layout, const dte_delta* d
                             (cudaStream_t)cuda_stream);
 }
 
+extern "C" dte_status dte_read_bandwidth_probe(const void* src, uint64_t bytes, uint64_t* xor_out, int device,
+                                               void* cuda_stream) {
+    if (!src || !xor_out) return fail(DTE_ERR_INVALID_ARG, "src / xor_out is null");
+    if ((uintptr_t)src & 15u) return fail(DTE_ERR_INVALID_ARG, "src must be 16-byte aligned");
+    DeviceGuard g(device);
+    return launch_read_probe(src, bytes, xor_out, device, (cudaStream_t)cuda_stream);
+}
+
 // ---- chunk codec -------------------------------------------------------------------------
 extern "C" uint64_t dte_chunk_count_bound(size_t n_lists, uint64_t entries, uint32_t chunk_entries) {
     return chunk_entries ? entries / chunk_entries + n_lists : 0;

@@ -180,6 +180,7 @@ dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 dte_status launch_pack_chunks(const PackParams& p, int device, cudaStream_t st);
 dte_status launch_unpack_chunks(const UnpackParams& p, int device, cudaStream_t st);
+dte_status launch_read_probe(const void* src, uint64_t bytes, uint64_t* out, int device, cudaStream_t st);
 dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const uint32_t* offsets,
                             const uint64_t* list_ptr, uint64_t* counts, cudaStream_t st);
 

@@ -482,3 +482,78 @@ def sender_subplan(plan: Plan, owners: Sequence[int], sender: int) -> Plan:
     q.slice_ranges = plan.slice_ranges
     q.ops = [op for op in plan.ops if owners[op[0]] == sender]
     return q
+
+
+def random_plan(seed: int, max_tensors: int = 6) -> Plan:
+    """A seeded plan of arbitrary hyper-rectangles for parity fuzzing: odd shapes, row / column /
+    grid splits, single-row pieces assembled into wider destination rows, stacked destinations
+    with gaps, replication, regions and whole tensors no operation reads.  Every destination
+    region is a contiguous flat range and no two overlap (the layout's rules)."""
+    rng = np.random.default_rng(seed)
+    p = Plan()
+
+    def cuts(n, k):
+        """k random consecutive blocks covering [0, n)."""
+        k = max(1, min(k, n))
+        inner = np.sort(rng.choice(np.arange(1, n), size=k - 1, replace=False)) if k > 1 else np.zeros(0, np.int64)
+        b = [0] + [int(x) for x in inner] + [n]
+        return list(zip(b[:-1], b[1:]))
+
+    n_t = int(rng.integers(1, max_tensors + 1))
+    for t in range(n_t):
+        if rng.random() < 0.25:
+            shape = (int(rng.integers(1, 60000)), 1)
+        else:
+            shape = (int(rng.integers(1, 400)), int(rng.integers(1, 900)))
+        src = p.add_tensor(f"t{t}", shape)
+        n0, n1 = shape
+        kind = rng.choice(["rows", "cols", "grid", "replicate", "row_pieces", "stack", "skip"],
+                          p=[0.2, 0.2, 0.15, 0.1, 0.15, 0.15, 0.05])
+        recv = lambda: int(rng.integers(0, 4))
+        if kind == "skip":
+            continue
+        if kind == "rows":                    # row blocks, each its own destination (some dropped)
+            for lo, hi in cuts(n0, int(rng.integers(1, 5))):
+                if rng.random() < 0.15:
+                    continue
+                k = p.add_shard(f"t{t}.rows{lo}", recv(), (hi - lo) * n1)
+                p.add_op(src, k, (lo, 0), (hi - lo, n1), 0, n1, (0, 0))
+        elif kind == "cols":                  # column blocks: strided sources, whole destination rows
+            for lo, hi in cuts(n1, int(rng.integers(1, 5))):
+                k = p.add_shard(f"t{t}.cols{lo}", recv(), n0 * (hi - lo))
+                p.add_op(src, k, (0, lo), (n0, hi - lo), 0, hi - lo, (0, 0))
+        elif kind == "grid":
+            for r0, r1 in cuts(n0, int(rng.integers(1, 4))):
+                for c0, c1 in cuts(n1, int(rng.integers(1, 4))):
+                    k = p.add_shard(f"t{t}.g{r0}.{c0}", recv(), (r1 - r0) * (c1 - c0))
+                    p.add_op(src, k, (r0, c0), (r1 - r0, c1 - c0), 0, c1 - c0, (0, 0))
+        elif kind == "replicate":
+            for r in range(int(rng.integers(2, 5))):
+                k = p.add_shard(f"t{t}.copy{r}", r, n0 * n1)
+                p.add_op(src, k, (0, 0), (n0, n1), 0, n1, (0, 0))
+        elif kind == "row_pieces":            # destination rows wider than the pieces that fill them
+            rows = min(n0, int(rng.integers(1, 12)))
+            pad_l, pad_r = int(rng.integers(0, 9)), int(rng.integers(0, 9))
+            ld = pad_l + n1 + pad_r
+            k = p.add_shard(f"t{t}.pieces", recv(), rows * ld)
+            for row in range(rows):
+                for c0, c1 in cuts(n1, int(rng.integers(1, 4))):
+                    if rng.random() < 0.1:
+                        continue              # a hole inside the destination row
+                    p.add_op(src, k, (row, c0), (1, c1 - c0), 0, ld, (row, pad_l + c0))
+        else:                                 # stack: row blocks at scattered bases of one destination
+            blocks = cuts(n0, int(rng.integers(1, 5)))
+            order = rng.permutation(len(blocks))
+            gap = int(rng.integers(0, 3)) * int(rng.integers(0, 50))
+            base, places = 0, {}
+            for i in order:
+                lo, hi = blocks[int(i)]
+                places[int(i)] = base
+                base += (hi - lo) * n1 + gap
+            k = p.add_shard(f"t{t}.stack", recv(), base + int(rng.integers(0, 20)))
+            for i, (lo, hi) in enumerate(blocks):
+                p.add_op(src, k, (lo, 0), (hi - lo, n1), places[i], n1, (0, 0))
+    if not p.ops:                             # never hand out an empty plan
+        k = p.add_shard("t0.all", 0, p.numel(0))
+        p.add_op(0, k, (0, 0), p.tensor_shapes[0], 0, p.tensor_shapes[0][1], (0, 0))
+    return p

@@ -56,6 +56,25 @@ def test_coverage_each_slot_once_and_reassembly(name):
     assert np.array_equal(val, want)
 
 
+@pytest.mark.parametrize("seed", range(12))
+def test_random_plans_remap_like_strided_slicing(seed):
+    # arbitrary hyper-rectangles with gaps and replication: with every element changed, list k is
+    # exactly the covered slots of shard k in ascending order, carrying the sliced dense values
+    plan = plans.random_plan(1000 + seed)
+    th, mm, vv, c = _all_changed_state(plan, seed)
+    lp, off, val = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), th, mm, vv, c)
+    marker = -1                                         # 0xFFFF cannot come out of these values
+    shards = [torch.full((n,), marker, dtype=torch.int16) for n in plan.shard_numels]
+    plans.scatter_dense(plan, [_bf16_bits_t(t).reshape(plan.tensor_shapes[i]) for i, t in enumerate(th)], shards)
+    assert int(lp[-1]) == plan.total_scanned_elements()
+    for k, buf in enumerate(shards):
+        b = buf.numpy().view(np.uint16)
+        covered = np.nonzero(b != 0xFFFF)[0]
+        seg = slice(int(lp[k]), int(lp[k + 1]))
+        assert np.array_equal(off[seg], covered.astype(np.uint32)), plan.shard_names[k]
+        assert np.array_equal(val[seg], b[covered])
+
+
 def test_tp1_is_identity_and_row_split_is_an_offset():
     plan = plans.single_matrix_plan(24, 20, 1)
     th, mm, vv, c = _all_changed_state(plan)
