@@ -95,11 +95,13 @@ __device__ __forceinline__ float rsqrt_ftz(float x) {
 
 template <bool DIV_BC1, bool DIV_DECAY>
 __device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s, float abs_lr) {
-    const uint32_t a = __float_as_uint(theta) & 0x7FFFFFFFu;
-    const uint32_t hi = ((a + 0x8000u) & 0xFFFF0000u) | 0x7FFEu;   // boundary above, minus 2 ulp
+    // boundaries from the raw pattern: the sign bit rides along (no carry reaches it below the NaN
+    // range) and is dropped by the |.| operand modifiers, which cost nothing
+    const uint32_t u = __float_as_uint(theta);
+    const uint32_t hi = ((u + 0x8000u) & 0xFFFF0000u) | 0x7FFEu;   // boundary above |theta|, minus 2 ulp
     const uint32_t lo = hi - 0xFFFCu;                               // boundary below, plus 2 ulp
-    const float at = __uint_as_float(a);
-    const float room = min_nan(__uint_as_float(hi) - at, at - __uint_as_float(lo));   // exact differences
+    const float at = fabsf(theta);
+    const float room = min_nan(fabsf(__uint_as_float(hi)) - at, at - fabsf(__uint_as_float(lo)));   // exact differences
     const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
     const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);   // -Inf for v = -0 or a negative subnormal
     float b = __fmul_rn(__fmul_rn(am, w), abs_lr);
@@ -361,13 +363,15 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
         // ---- phase C: one reservation per CTA, coalesced writes in tile order, the record -----
         if (lane == 0) s_count[warp] = n_changed;
         __syncthreads();
-        uint32_t before = 0, total = 0;
+        // exclusive prefix and total of the eight warp counts: lanes 0..7 of every warp scan them
+        uint32_t incl = lane < kWarps ? s_count[lane] : 0u;
 #pragma unroll
-        for (int w = 0; w < kWarps; ++w) {
-            const uint32_t x = s_count[w];
-            if (w < warp) before += x;
-            total += x;
+        for (int d = 1; d < kWarps; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= d) incl += up;
         }
+        const uint32_t total = __shfl_sync(0xFFFFFFFFu, incl, kWarps - 1);
+        const uint32_t before = __shfl_sync(0xFFFFFFFFu, incl, warp) - n_changed;
         if (threadIdx.x == 0) {
             unsigned long long pos0 = 0;
             if (total) pos0 = atomicAdd(p.cursor, (unsigned long long)total);
