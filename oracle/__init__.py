@@ -61,6 +61,9 @@ def lib() -> ctypes.CDLL:
             L.oracle_apply.argtypes = [c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
                                        c.c_void_p]
             L.oracle_apply.restype = c.c_int
+            L.oracle_apply_canonical.argtypes = [c.c_uint64, c.c_void_p, c.c_uint64, c.c_void_p, c.c_uint64,
+                                                 c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p]
+            L.oracle_apply_canonical.restype = c.c_int
             L.oracle_adler32.argtypes = [c.c_void_p, c.c_uint64]
             L.oracle_adler32.restype = c.c_uint32
             L.oracle_pack_chunks.argtypes = [c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_uint32,
@@ -176,6 +179,29 @@ def apply(shard_numels, list_ptr, offsets, values, shards) -> None:
                             val.ctypes.data, _ptr_array(shards))
     if rc != 0:
         raise ValueError("receiver index outside its shard")
+
+
+def apply_canonical(tensor_shapes, shard_numels, ops, list_ptr, indices, values, shards) -> None:
+    """Eq. 5-7 on canonical entries (destination-side mapping of the storage path), in place on
+    ``shards``: a list of contiguous uint16 arrays, or None for shards other receivers hold."""
+    shp = np.ascontiguousarray(tensor_shapes, dtype=np.int64).reshape(-1, 2)
+    num = np.ascontiguousarray(shard_numels, dtype=np.int64).reshape(-1)
+    op = np.ascontiguousarray(ops, dtype=np.int64).reshape(-1, 10)
+    lp = np.ascontiguousarray(list_ptr, dtype=np.uint64)
+    idx = np.ascontiguousarray(indices, dtype=np.uint32)
+    val = np.ascontiguousarray(values, dtype=np.uint16)
+    assert lp.size == shp.shape[0] + 1 and len(shards) == num.size
+    ptrs = (ctypes.c_void_p * max(1, num.size))()
+    for k, s in enumerate(shards):
+        if s is not None:
+            assert s.dtype == np.uint16 and s.flags.c_contiguous and s.size == num[k]
+            ptrs[k] = s.ctypes.data
+    rc = lib().oracle_apply_canonical(shp.shape[0], shp.ctypes.data, num.size, num.ctypes.data, op.shape[0],
+                                      op.ctypes.data, lp.ctypes.data, idx.ctypes.data, val.ctypes.data, ptrs)
+    if rc == 1:
+        raise ValueError("receiver index outside its shard")
+    if rc == 2:
+        raise ValueError("canonical index outside its tensor")
 
 
 def adler32(data) -> int:

@@ -16,13 +16,15 @@
 // cast against a nearest-neighbour formulation in fp64 and a library cast;
 // the changed set against an unfused array-at-a-time evaluation; the remap
 // against coverage / reassembly invariants and dense slicing; apply against
-// idempotence, untouched positions and the end-state identity.
+// idempotence, untouched positions and the end-state identity; the destination-side mapping
+// against dense slicing of the changed positions and against extract-then-apply.
 //
 // Passages followed:
 //   Eq. 2  (AdamW inverse, Section 4.1; derivation Eq. 9-11, Appendix A)
 //   Eq. 4  (BF16 cast, 16-bit pattern compare, nonzero, target values; Section 4.2.1)
 //   Eq. 5-6 and the membership test between them (unravel - remap - ravel; Section 4.2.2)
 //   Eq. 7  (direct sparse apply; Section 4.3)
+//   Section 4.4 (destination-side mapping of canonical entries: Eq. 5-7 per received entry)
 
 #include <algorithm>
 #include <cmath>
@@ -249,3 +251,39 @@ int oracle_apply(uint64_t n_shards, const int64_t* shard_numel, const uint64_t* 
 }
 
 }  // extern "C"
+
+// Destination-side mapping of canonical entries (Section 4.4: the storage-mediated path ships
+// canonical changes and "performs the final inference-layout mapping inside the destination").
+// list p = changed flat indices i of canonical tensor p with their target values.  Literally
+// Eq. 5-7: for every entry, u = unravel(i, n_s); for every operation on tensor p in plan order
+// with a_s <= u < a_s + e: j = ravel(u - a_s + a_r, n_r) and shard[dst][j] <- value.  Operations
+// whose shard pointer is NULL belong to other receivers and are skipped.  Returns 0, 1 if a j
+// lies outside its shard, 2 if an index lies outside its tensor (nothing further is written).
+extern "C" int oracle_apply_canonical(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n_shards,
+                                      const int64_t* shard_numel, uint64_t n_ops, const int64_t* ops,
+                                      const uint64_t* list_ptr, const uint32_t* indices,
+                                      const uint16_t* values, uint16_t* const* shards) {
+    (void)n_shards;
+    for (uint64_t p = 0; p < n_tensors; ++p) {
+        const uint64_t n0 = (uint64_t)tensor_shape[2 * p], n1 = (uint64_t)tensor_shape[2 * p + 1];
+        for (uint64_t q = list_ptr[p]; q < list_ptr[p + 1]; ++q) {
+            const uint64_t i = indices[q];
+            if (i >= n0 * n1) return 2;
+            const uint64_t u0 = i / n1, u1 = i % n1;                       // Eq. 5
+            for (uint64_t o = 0; o < n_ops; ++o) {
+                const int64_t* op = ops + 10 * o;
+                if ((uint64_t)op[0] != p) continue;
+                const uint64_t as0 = (uint64_t)op[2], as1 = (uint64_t)op[3];
+                const uint64_t e0 = (uint64_t)op[4], e1 = (uint64_t)op[5];
+                if (u0 < as0 || u0 >= as0 + e0 || u1 < as1 || u1 >= as1 + e1) continue;
+                uint16_t* dst = shards[(uint64_t)op[1]];
+                if (!dst) continue;
+                const uint64_t j = (uint64_t)op[6] + (u0 - as0 + (uint64_t)op[8]) * (uint64_t)op[7] +
+                                   (u1 - as1 + (uint64_t)op[9]);                // Eq. 6
+                if (j >= (uint64_t)shard_numel[(uint64_t)op[1]]) return 1;
+                dst[j] = values[q];                                          // Eq. 7
+            }
+        }
+    }
+    return 0;
+}

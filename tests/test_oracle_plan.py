@@ -355,3 +355,64 @@ def test_op_counts_keep_every_planned_operation():
         end = begin + e0 * e1          # whole destination rows: a contiguous block
         seg = off[int(lp[dst]):int(lp[dst + 1])].astype(np.int64)
         assert int(((seg >= begin) & (seg < end)).sum()) == int(cnt[o])
+
+
+# ---------------------------------------------------------------- destination-side mapping (Section 4.4)
+
+def _canonical_lists(plan, th, mm, vv, c):
+    ident = plans.canonical_plan(plan.tensor_names, plan.tensor_shapes)
+    return oracle.extract(ident.tensor_shapes, ident.shard_numels, ident.ops_array(), th, mm, vv, c)
+
+
+@pytest.mark.parametrize("name", list(SMALL_PLANS) + [f"random{i}" for i in range(6)])
+def test_canonical_entries_mapped_at_the_destination_equal_dense_slicing(name):
+    plan = plans.random_plan(1000 + int(name[6:])) if name.startswith("random") else SMALL_PLANS[name]()
+    hp = Hyper(step=50, lr=3e-5, wd=0.01)
+    wl = configs.Workload(name, plan, hp, configs._specs(plan), 11)
+    st = wl.materialize("cpu")
+    th, mm, vv = ([t.numpy() for t in x] for x in (st.theta, st.m, st.v))
+    c = oracle.derive_constants(*hp.as_args())
+    lp, idx, val = _canonical_lists(plan, th, mm, vv, c)
+    assert 0 < int(lp[-1]) < plan.total_source_elements()
+    canary = 0x5A5A
+    got = [np.full(n, canary, np.uint16) for n in plan.shard_numels]
+    oracle.apply_canonical(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), lp, idx, val, got)
+    # independent statement: a dense tensor holding the target value at changed positions and a
+    # marker elsewhere, pushed through strided slicing; marker slots keep the canary
+    marker = 0xFFFF
+    dense = []
+    for p in range(plan.n_tensors):
+        d = np.full(plan.numel(p), marker, np.uint16)
+        seg = slice(int(lp[p]), int(lp[p + 1]))
+        d[idx[seg]] = val[seg]
+        assert not np.any(val[seg] == marker)
+        dense.append(torch.from_numpy(d.view(np.int16)).reshape(plan.tensor_shapes[p]))
+    sliced = [torch.full((n,), -1, dtype=torch.int16) for n in plan.shard_numels]
+    plans.scatter_dense(plan, dense, sliced)
+    for k in range(plan.n_shards):
+        want = sliced[k].numpy().view(np.uint16).copy()
+        want[want == marker] = canary
+        assert np.array_equal(got[k], want), plan.shard_names[k]
+    # and it is what extract-with-the-plan followed by apply produces
+    lists = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), th, mm, vv, c)
+    ref = [np.full(n, canary, np.uint16) for n in plan.shard_numels]
+    oracle.apply(plan.shard_numels, *lists, ref)
+    for k in range(plan.n_shards):
+        assert np.array_equal(got[k], ref[k])
+
+
+def test_canonical_mapping_skips_other_receivers_and_reports_bad_entries():
+    plan = plans.qwen3_dense_plan(1, 2, False, configs.SMALL_DENSE)
+    th, mm, vv, c = _all_changed_state(plan)
+    lp, idx, val = _canonical_lists(plan, th, mm, vv, c)
+    mine = [k for k, r in enumerate(plan.shard_receivers) if r == 1]
+    shards = [np.zeros(n, np.uint16) if k in mine else None for k, n in enumerate(plan.shard_numels)]
+    oracle.apply_canonical(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), lp, idx, val, shards)
+    full = [torch.zeros(n, dtype=torch.int16) for n in plan.shard_numels]
+    plans.scatter_dense(plan, [_bf16_bits_t(t) for t in th], full)
+    for k in mine:
+        assert np.array_equal(shards[k], full[k].numpy().view(np.uint16))
+    bad = idx.copy()
+    bad[0] = plan.numel(0)                                   # one past the end of tensor 0
+    with pytest.raises(ValueError):
+        oracle.apply_canonical(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), lp, bad, val, shards)
