@@ -59,7 +59,8 @@ typedef enum dte_status {
 
 /* Device-detected conditions, OR-ed into dte_delta.counters[2]. */
 #define DTE_DEV_OVERFLOW 1u /* more changed elements than `capacity`; lists not produced   */
-#define DTE_DEV_BOUNDS 2u   /* apply met an offset >= numel of its shard; entry skipped  */
+#define DTE_DEV_BOUNDS 2u   /* apply met an offset >= numel of its shard, an entry for a NULL
+                               shard, or a canonical index outside its tensor; entry skipped */
 #define DTE_DEV_TIMEOUT 4u  /* reserved (no kernel of this library waits on another CTA)  */
 #define DTE_DEV_CORRUPT 8u  /* unpack rejected a chunk (header or checksum); lists have holes */
 
@@ -205,13 +206,30 @@ DTE_API dte_status dte_extract_delta_static(const dte_layout* layout, const floa
                                             const dte_delta* out, void* cuda_stream);
 
 /* Eq. 7: shard[k][offsets[e]] = values[e] for every entry e of every list k.
- * shard_ptrs: HOST array of n_shards DEVICE pointers (BF16 buffers, numel as declared;
- * shards whose lists are necessarily empty may be NULL).  Reads list sizes on the device,
+ * shard_ptrs: HOST array of n_shards DEVICE pointers (BF16 buffers, numel as declared; a shard
+ * whose list is empty may be NULL - a receiver passes only the tensors it holds; an entry that
+ * does arrive for a NULL shard is skipped and flagged DTE_DEV_BOUNDS).  Reads list sizes on the device,
  * so it can be enqueued right after extract without a host round trip.  Refuses to write
  * anything (and sets DTE_DEV_OVERFLOW again) if `delta` overflowed its capacity, and nothing
  * if its counters carry DTE_DEV_CORRUPT (lists read from a damaged chunk stream). */
 DTE_API dte_status dte_apply(const dte_layout* layout, const dte_delta* delta,
                      uint16_t* const* shard_ptrs, void* cuda_stream);
+
+/* Section 4.4, destination side of the storage-mediated path: the published entries are
+ * canonical - list p of `canonical` holds the changed flat indices of SOURCE tensor p (ascending)
+ * and their BF16 target values, i.e. Eq. 4's (I, V) per tensor, what an extract over the identity
+ * plan of the same tensors produces; list_ptr has n_tensors + 1 entries - and the mapping into
+ * the inference layout happens here.  For every entry and every operation of the layout on its
+ * tensor, in plan order: u = unravel(i) (Eq. 5), membership src_origin <= u < src_origin + extent,
+ * j by Eq. 6, shard[dst_shard][j] = value (Eq. 7).  An operation whose shard pointer is NULL is
+ * skipped (the tensor lives on another receiver), so one plan serves every receiver.  Refuses, like
+ * dte_apply, a delta that overflowed or carries DTE_DEV_CORRUPT; an index outside its tensor or a
+ * j outside its shard is skipped and flagged DTE_DEV_BOUNDS.  The first call on a layout uploads
+ * its per-tensor operation tables (cudaMalloc, synchronous; 32 bytes per operation).  Cost is
+ * proportional to the operations per source tensor: meant for canonical (HF-shaped) sources.
+ * Errors: DTE_ERR_LAYOUT if a tensor the plan reads has >= 2^32 elements. */
+DTE_API dte_status dte_apply_canonical(const dte_layout* layout, const dte_delta* canonical,
+                                       uint16_t* const* shard_ptrs, void* cuda_stream);
 
 /* Section 4.3, round 1 of the two-round transfer: the entry count c_o = |I_o| of every
  * operation of the plan, in plan order, zero-length operations included (both peers keep

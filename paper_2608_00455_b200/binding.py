@@ -27,7 +27,7 @@ SYMBOLS = [
     "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
     "dte_extract_delta_static", "dte_extract_delta_groups", "dte_layout_num_groups",
     "dte_op_counts", "dte_layout_num_ops", "dte_chunk_count_bound", "dte_chunk_bytes_bound",
-    "dte_pack_chunks", "dte_unpack_chunks", "dte_read_bandwidth_probe",
+    "dte_pack_chunks", "dte_unpack_chunks", "dte_read_bandwidth_probe", "dte_apply_canonical",
 ]
 
 
@@ -109,6 +109,8 @@ def lib() -> C.CDLL:
         L.dte_unpack_chunks.restype = C.c_int
         L.dte_read_bandwidth_probe.argtypes = [vp, u64, vp, C.c_int, vp]
         L.dte_read_bandwidth_probe.restype = C.c_int
+        L.dte_apply_canonical.argtypes = [vp, vp, vp, vp]
+        L.dte_apply_canonical.restype = C.c_int
         L.dte_apply.argtypes = [vp, vp, vp, vp]
         L.dte_apply.restype = C.c_int
         L.dte_extract_delta_host.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, u64,
@@ -409,6 +411,12 @@ def dte_read_bandwidth_probe(tensor: torch.Tensor, xor_out: torch.Tensor, stream
     assert tensor.is_cuda and tensor.is_contiguous() and xor_out.is_cuda and xor_out.dtype == torch.int64
     _check(lib().dte_read_bandwidth_probe(tensor.data_ptr(), tensor.numel() * tensor.element_size(),
                                           xor_out.data_ptr(), tensor.device.index or 0, _stream_ptr(stream)))
+
+
+def dte_apply_canonical(layout: Layout, canonical: Delta, shard_table, stream=None) -> None:
+    """Map canonical entries (one list per SOURCE tensor) into the receiver's shards and store them:
+    the destination side of the storage path.  Shards of other receivers may be None in the table."""
+    _check(lib().dte_apply_canonical(layout._h, C.byref(canonical.struct), shard_table, _stream_ptr(stream)))
 
 
 class HostResult:

@@ -212,6 +212,22 @@ extern "C" dte_status dte_extract_delta_groups(const dte_layout* layout, const f
     return enqueue_extract(L, groups[0].c, out, st, &groups);
 }
 
+namespace {
+// Upload the shard pointer table unless it equals the one already on the device.
+dte_status sync_shard_table(dte_layout* L, uint16_t* const* shard_ptrs, cudaStream_t st) {
+    const size_t n = L->n_lists;
+    std::vector<uint16_t*> tab(shard_ptrs, shard_ptrs + n);
+    for (size_t k = 0; k < n; ++k)
+        if ((uintptr_t)tab[k] & 1u) return fail(DTE_ERR_INVALID_ARG, "shard pointers must be 2-byte aligned");
+    if (L->shards_valid && tab == L->h_shards) return DTE_OK;
+    L->shards_valid = false;
+    DTE_CUDA(cudaMemcpyAsync((void*)L->d_shards, tab.data(), n * sizeof(void*), cudaMemcpyHostToDevice, st));
+    L->h_shards.swap(tab);
+    L->shards_valid = true;
+    return DTE_OK;
+}
+}  // namespace
+
 extern "C" dte_status dte_apply(const dte_layout* layout, const dte_delta* delta,
                                 uint16_t* const* shard_ptrs, void* cuda_stream) {
     if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
@@ -221,20 +237,9 @@ extern "C" dte_status dte_apply(const dte_layout* layout, const dte_delta* delta
     dte_layout* L = const_cast<dte_layout*>(layout);
     DeviceGuard g(L->device);
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    const size_t n = L->n_lists;
-    if (n == 0) return DTE_OK;
-    std::vector<uint16_t*> tab(shard_ptrs, shard_ptrs + n);
-    for (size_t k = 0; k < n; ++k) {
-        if (!tab[k] && L->list_has_tiles[k] && L->shard_numel[k])
-            return fail(DTE_ERR_INVALID_ARG, "null shard pointer for a list that can hold entries");
-        if ((uintptr_t)tab[k] & 1u) return fail(DTE_ERR_INVALID_ARG, "shard pointers must be 2-byte aligned");
-    }
-    if (!(L->shards_valid && tab == L->h_shards)) {
-        L->shards_valid = false;
-        DTE_CUDA(cudaMemcpyAsync((void*)L->d_shards, tab.data(), n * sizeof(void*), cudaMemcpyHostToDevice, st));
-        L->h_shards.swap(tab);
-        L->shards_valid = true;
-    }
+    if (L->n_lists == 0) return DTE_OK;
+    s = sync_shard_table(L, shard_ptrs, st);
+    if (s != DTE_OK) return s;
     ApplyParams p;
     p.offsets = delta->offsets;
     p.values = delta->values;
@@ -245,6 +250,53 @@ extern "C" dte_status dte_apply(const dte_layout* layout, const dte_delta* delta
     p.shard_numel = L->d_shard_numel;
     p.n_lists = L->n_lists;
     return launch_apply(p, L->device, st);
+}
+
+extern "C" dte_status dte_apply_canonical(const dte_layout* layout, const dte_delta* canonical,
+                                          uint16_t* const* shard_ptrs, void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    dte_status s = check_delta(canonical);
+    if (s != DTE_OK) return s;
+    if (layout->n_lists && !shard_ptrs) return fail(DTE_ERR_INVALID_ARG, "shard pointer table is null");
+    dte_layout* L = const_cast<dte_layout*>(layout);
+    if (!L->canonical_ok)
+        return fail(DTE_ERR_LAYOUT, "a source tensor the plan reads has 2^32 or more elements: no uint32 canonical index");
+    DeviceGuard g(L->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    if (L->n_tensors == 0 || L->n_lists == 0) return DTE_OK;
+    if (!L->d_src_ops) {      // first use: the per-source-tensor operation tables go to the device
+        const size_t n_ops = std::max<size_t>(L->h_src_ops.size(), 1), nt = L->n_tensors;
+        DTE_CUDA(cudaMalloc((void**)&L->d_src_op_ptr, (nt + 1) * sizeof(uint32_t)));
+        DTE_CUDA(cudaMalloc((void**)&L->d_tensor_cols, nt * sizeof(uint32_t)));
+        DTE_CUDA(cudaMalloc((void**)&L->d_tensor_numel32, nt * sizeof(uint32_t)));
+        SrcOp* ops = nullptr;
+        DTE_CUDA(cudaMalloc((void**)&ops, n_ops * sizeof(SrcOp)));
+        cudaError_t e = cudaMemcpy(ops, L->h_src_ops.data(), L->h_src_ops.size() * sizeof(SrcOp), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(L->d_src_op_ptr, L->h_src_op_ptr.data(), (nt + 1) * sizeof(uint32_t), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(L->d_tensor_cols, L->h_tensor_cols.data(), nt * sizeof(uint32_t), cudaMemcpyHostToDevice);
+        if (e == cudaSuccess) e = cudaMemcpy(L->d_tensor_numel32, L->h_tensor_numel32.data(), nt * sizeof(uint32_t), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) {
+            cudaFree(ops);
+            return cuda_fail(e, "upload of the destination-side mapping tables");
+        }
+        L->d_src_ops = ops;
+    }
+    s = sync_shard_table(L, shard_ptrs, st);
+    if (s != DTE_OK) return s;
+    CanonParams p;
+    p.indices = canonical->offsets;
+    p.values = canonical->values;
+    p.capacity = canonical->capacity;
+    p.list_ptr = canonical->list_ptr;
+    p.counters = canonical->counters;
+    p.shards = L->d_shards;
+    p.shard_numel = L->d_shard_numel;
+    p.n_tensors = L->n_tensors;
+    p.ops = L->d_src_ops;
+    p.op_ptr = L->d_src_op_ptr;
+    p.tensor_cols = L->d_tensor_cols;
+    p.tensor_numel = L->d_tensor_numel32;
+    return launch_apply_canonical(p, L->device, st);
 }
 
 extern "C" dte_status dte_op_counts(const dte_layout* layout, const dte_delta* delta, uint64_t* counts,

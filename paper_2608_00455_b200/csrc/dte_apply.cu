@@ -59,12 +59,9 @@ __global__ void __launch_bounds__(kApplyThreads) apply_kernel(const ApplyParams 
             const uint64_t e = base + (uint64_t)j * kApplyThreads + threadIdx.x;
             if (e < total) {
                 while (e >= lp[k + 1]) ++k;          // e < total = lp[L] keeps k < L
-                if ((uint64_t)off[j] < __ldg(p.shard_numel + k)) {
-                    uint16_t* dst = reinterpret_cast<uint16_t*>(__ldg(reinterpret_cast<const unsigned long long*>(p.shards + k)));
-                    dst[off[j]] = val[j];
-                } else {
-                    bad = true;
-                }
+                uint16_t* dst = reinterpret_cast<uint16_t*>(__ldg(reinterpret_cast<const unsigned long long*>(p.shards + k)));
+                if (dst && (uint64_t)off[j] < __ldg(p.shard_numel + k)) dst[off[j]] = val[j];
+                else bad = true;          // outside the shard, or an entry for a shard the caller did not give
             }
         }
     }
@@ -79,6 +76,85 @@ dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st) {
     // 2-byte writes are bound by the memory system's sector read-modify-write rate.  Touching
     // the sector first (a load: 8 G/s; an L2 prefetch one chunk ahead: 31 G/s) only hurts.
     apply_kernel<<<sms * 6, kApplyThreads, 0, st>>>(p);
+    DTE_CUDA(cudaGetLastError());
+    return DTE_OK;
+}
+
+// ---- destination-side mapping of canonical entries (Section 4.4) -------------------------------
+// The storage-mediated path ships canonical (index, value) pairs and maps them to the inference
+// layout on the destination.  Per entry: unravel (Eq. 5), test the operations of its source tensor
+// for membership, ravel (Eq. 6) and store (Eq. 7) - the paper's own source-major form, which is the
+// right one here because only the changed entries exist on this side.
+__global__ void __launch_bounds__(kApplyThreads) apply_canonical_kernel(const CanonParams p) {
+    __shared__ uint64_t s_ptr[kApplySmemLists + 1];
+    const uint32_t L = p.n_tensors;
+    const bool cached = L <= (uint32_t)kApplySmemLists;
+    if (cached)
+        for (uint32_t k = threadIdx.x; k <= L; k += blockDim.x) s_ptr[k] = p.list_ptr[k];
+    __syncthreads();
+    const uint64_t* lp = cached ? s_ptr : p.list_ptr;
+    const uint64_t total = lp[L];
+    const uint64_t dev_bits = p.counters[2];
+    if (total > p.capacity || (dev_bits & (DTE_DEV_OVERFLOW | DTE_DEV_CORRUPT))) {
+        if (blockIdx.x == 0 && threadIdx.x == 0 && !(dev_bits & DTE_DEV_CORRUPT))
+            atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_OVERFLOW);
+        return;
+    }
+    bool bad = false;
+    for (uint64_t base = (uint64_t)blockIdx.x * kApplyChunk; base < total; base += (uint64_t)gridDim.x * kApplyChunk) {
+        uint32_t idx[kApplyPerThread];
+        uint16_t val[kApplyPerThread];
+#pragma unroll
+        for (int j = 0; j < kApplyPerThread; ++j) {
+            const uint64_t e = base + (uint64_t)j * kApplyThreads + threadIdx.x;
+            if (e < total) {
+                idx[j] = __ldcs(p.indices + e);
+                val[j] = __ldcs(p.values + e);
+            }
+        }
+        uint32_t k = 0;
+        {
+            const uint64_t e = base + threadIdx.x;
+            uint32_t lo = 0, hi = L;
+            while (hi - lo > 1) {
+                const uint32_t mid = (lo + hi) >> 1;
+                if (lp[mid] <= e) lo = mid; else hi = mid;
+            }
+            k = lo;
+        }
+#pragma unroll
+        for (int j = 0; j < kApplyPerThread; ++j) {
+            const uint64_t e = base + (uint64_t)j * kApplyThreads + threadIdx.x;
+            if (e >= total) continue;
+            while (e >= lp[k + 1]) ++k;
+            const uint32_t i = idx[j];
+            if (i >= __ldg(p.tensor_numel + k)) { bad = true; continue; }
+            const uint32_t n1 = __ldg(p.tensor_cols + k);
+            const uint32_t u0 = i / n1, u1 = i - u0 * n1;                     // Eq. 5
+            const uint32_t o_end = __ldg(p.op_ptr + k + 1);
+            for (uint32_t o = __ldg(p.op_ptr + k); o < o_end; ++o) {
+                const uint4* q = reinterpret_cast<const uint4*>(p.ops + o);
+                const uint4 w0 = __ldg(q);
+                const uint32_t r0 = u0 - w0.x, r1 = u1 - w0.y;                 // wraps when below the origin
+                if (r0 >= w0.z || r1 >= w0.w) continue;                         // a_s <= u < a_s + e
+                const uint4 w1 = __ldg(q + 1);
+                const uint32_t shard = w1.y;
+                uint16_t* dst = reinterpret_cast<uint16_t*>(__ldg(reinterpret_cast<const unsigned long long*>(p.shards + shard)));
+                if (!dst) continue;                                             // another receiver's tensor
+                const uint64_t ld = (uint64_t)w1.z | ((uint64_t)w1.w << 32);
+                const uint64_t jj = (uint64_t)w1.x + (uint64_t)r0 * ld + r1;   // Eq. 6
+                if (jj < __ldg(p.shard_numel + shard)) dst[jj] = val[j];       // Eq. 7
+                else bad = true;
+            }
+        }
+    }
+    if (bad) atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_BOUNDS);
+}
+
+dte_status launch_apply_canonical(const CanonParams& p, int device, cudaStream_t st) {
+    int sms = 0;
+    DTE_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+    apply_canonical_kernel<<<sms * 6, kApplyThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }

@@ -131,6 +131,32 @@ struct ApplyParams {
     uint32_t n_lists;
 };
 
+// One operation as the destination-side mapping needs it (Eq. 5-6 per received canonical entry):
+// membership a <= u < a + e, then j = dst0 + (u0 - a0) * ld + (u1 - a1).  Sorted by source tensor,
+// plan order within a tensor.
+struct __align__(16) SrcOp {
+    uint32_t a0, a1, e0, e1;
+    uint32_t dst0;       // flat receiver index of the region's first element (< 2^32)
+    uint32_t shard;
+    uint64_t ld;
+};
+static_assert(sizeof(SrcOp) == 32, "SrcOp is read as two uint4");
+
+struct CanonParams {
+    const uint32_t* indices;       // canonical flat indices, list p = source tensor p
+    const uint16_t* values;
+    uint64_t capacity;
+    const uint64_t* list_ptr;      // n_tensors + 1
+    uint64_t* counters;
+    uint16_t* const* shards;       // device table, n_shards (NULL: another receiver's)
+    const uint64_t* shard_numel;
+    uint32_t n_tensors;
+    const SrcOp* ops;
+    const uint32_t* op_ptr;        // n_tensors + 1
+    const uint32_t* tensor_cols;   // n_tensors: n_s[1]
+    const uint32_t* tensor_numel;  // n_tensors
+};
+
 // Destination range of one operation, in plan order (for the per-operation counts).
 struct OpRange {
     uint32_t list;
@@ -178,6 +204,7 @@ dte_status cuda_fail(cudaError_t e, const char* what);
 dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, cudaStream_t st);
 dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
+dte_status launch_apply_canonical(const CanonParams& p, int device, cudaStream_t st);
 dte_status launch_pack_chunks(const PackParams& p, int device, cudaStream_t st);
 dte_status launch_unpack_chunks(const UnpackParams& p, int device, cudaStream_t st);
 dte_status launch_read_probe(const void* src, uint64_t bytes, uint64_t* out, int device, cudaStream_t st);
@@ -214,6 +241,15 @@ struct dte_layout {
     uint32_t n_groups = 1;
     dte::OpRange* d_op_ranges = nullptr;   // n_ops, plan order
     uint32_t n_ops = 0;
+    // destination-side mapping tables: built at create on the host, uploaded by the first call
+    // that needs them (dte_apply_canonical)
+    std::vector<dte::SrcOp> h_src_ops;
+    std::vector<uint32_t> h_src_op_ptr, h_tensor_cols, h_tensor_numel32;
+    bool canonical_ok = true;              // every tensor an operation reads has numel < 2^32
+    dte::SrcOp* d_src_ops = nullptr;
+    uint32_t* d_src_op_ptr = nullptr;
+    uint32_t* d_tensor_cols = nullptr;
+    uint32_t* d_tensor_numel32 = nullptr;
     // host mirrors of the pointer tables last uploaded
     std::vector<const float*> h_ptrs;
     std::vector<uint16_t*> h_shards;

@@ -94,6 +94,10 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
     cudaFree(L->d_tensor_group);
     cudaFree(L->d_op_ranges);
     cudaFree(L->d_groups);
+    cudaFree(L->d_src_ops);
+    cudaFree(L->d_src_op_ptr);
+    cudaFree(L->d_tensor_cols);
+    cudaFree(L->d_tensor_numel32);
     if (prev >= 0) cudaSetDevice(prev);
     delete L;
 }
@@ -335,6 +339,34 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     guard(upload(&L->d_list_first_rec, first_rec));
     guard(upload(&L->d_op_ranges, op_ranges));
     L->n_ops = (uint32_t)n_ops;
+    {   // destination-side mapping tables (host only until first used)
+        L->h_src_op_ptr.assign(n_tensors + 1, 0);
+        L->h_tensor_cols.resize(n_tensors);
+        L->h_tensor_numel32.resize(n_tensors);
+        for (size_t p = 0; p < n_tensors; ++p) {
+            const bool fits = numel[p] < (uint64_t(1) << 32);
+            if (used[p] && !fits) L->canonical_ok = false;
+            L->h_tensor_cols[p] = fits ? (uint32_t)tensors[p].shape[1] : 0u;
+            L->h_tensor_numel32[p] = fits ? (uint32_t)numel[p] : 0u;
+        }
+        for (size_t o = 0; o < n_ops; ++o)
+            if (ops[o].extent[0] && ops[o].extent[1]) L->h_src_op_ptr[ops[o].src_tensor + 1] += 1;
+        for (size_t p = 0; p < n_tensors; ++p) L->h_src_op_ptr[p + 1] += L->h_src_op_ptr[p];
+        L->h_src_ops.resize(L->h_src_op_ptr[n_tensors]);
+        std::vector<uint32_t> at(L->h_src_op_ptr.begin(), L->h_src_op_ptr.end() - 1);
+        if (L->canonical_ok)
+            for (size_t o = 0; o < n_ops; ++o) {
+                const dte_op_desc& op = ops[o];
+                if (!op.extent[0] || !op.extent[1]) continue;
+                SrcOp so;
+                so.a0 = (uint32_t)op.src_origin[0]; so.a1 = (uint32_t)op.src_origin[1];
+                so.e0 = (uint32_t)op.extent[0]; so.e1 = (uint32_t)op.extent[1];
+                so.dst0 = (uint32_t)op_ranges[o].begin;
+                so.shard = op.dst_shard;
+                so.ld = op.dst_ld;
+                L->h_src_ops[at[op.src_tensor]++] = so;
+            }
+    }
     {
         std::vector<uint32_t> grp(n_tensors);
         for (size_t p = 0; p < n_tensors; ++p) {
