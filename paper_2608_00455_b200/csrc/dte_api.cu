@@ -75,43 +75,40 @@ Screen make_screen(const Consts& c) {
     return s;
 }
 
-// `groups`: per-parameter-group constants (NULL: `c` applies to every tensor).
-dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out, cudaStream_t st,
-                           const std::vector<GroupConsts>* groups = nullptr) {
-    uint64_t launches = 0;
+// Where one extract call keeps its placement records, block sums, staging cursor and staged
+// entries: the layout's own buffers, or the fixed array of the allocation-free entry point.
+struct Scratch {
+    uint64_t* cursor;
+    uint64_t* rec;
+    uint64_t* block_sum;
+    uint32_t* stage_offsets;
+    uint16_t* stage_values;
+};
+
+// Enqueues the kernels of one extract: both extract launches (regular and packed tiles), then
+// the scan and gather that put the staged entries in order.  `groups`: per-parameter-group
+// constants (NULL: `c` applies to every tensor).  out->counters is cleared here; the cursor is
+// the only scratch word that must start at zero (records and block sums are rewritten in full,
+// staged entries are read only where this call wrote them).
+dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<GroupConsts>* groups,
+                           const Scratch& sc, const dte_delta* out, cudaStream_t st) {
     DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
     if (L->n_tiles == 0) {
         DTE_CUDA(cudaMemsetAsync(out->list_ptr, 0, (L->n_lists + 1) * sizeof(uint64_t), st));
         L->last_launch[0] = 0; L->last_launch[1] = 0; L->last_launch[2] = 0;
         return DTE_OK;
     }
-    // the staging buffer mirrors the caller's capacity; it is (re)allocated only when a call
-    // brings a larger capacity than any before it
-    if (out->capacity > L->stage_capacity) {
-        DTE_CUDA(cudaStreamSynchronize(st));
-        cudaFree(L->d_stage_offsets);
-        cudaFree(L->d_stage_values);
-        L->d_stage_offsets = nullptr;
-        L->d_stage_values = nullptr;
-        L->stage_capacity = 0;
-        DTE_CUDA(cudaMalloc((void**)&L->d_stage_offsets, out->capacity * sizeof(uint32_t)));
-        DTE_CUDA(cudaMalloc((void**)&L->d_stage_values, out->capacity * sizeof(uint16_t)));
-        L->stage_capacity = out->capacity;
-    }
-    const size_t n_rec = (size_t)L->n_tiles;
-    DTE_CUDA(cudaMemsetAsync(L->d_cursor, 0, sizeof(uint64_t), st));
+    DTE_CUDA(cudaMemsetAsync(sc.cursor, 0, sizeof(uint64_t), st));
     ExtractParams p;
-    p.tiles = L->d_tiles;
     p.segs = L->d_segs;
     p.theta = L->d_ptrs;
     p.m = L->d_ptrs + L->n_tensors;
     p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
-    p.cursor = reinterpret_cast<unsigned long long*>(L->d_cursor);
-    p.rec = L->d_rec;
-    p.stage_offsets = L->d_stage_offsets;
-    p.stage_values = L->d_stage_values;
+    p.cursor = reinterpret_cast<unsigned long long*>(sc.cursor);
+    p.rec = sc.rec;
+    p.stage_offsets = sc.stage_offsets;
+    p.stage_values = sc.stage_values;
     p.stage_capacity = out->capacity;
-    p.n_tiles = L->n_tiles;
     p.c = c;
     p.s = make_screen(c);
     p.tensor_group = nullptr;
@@ -130,7 +127,7 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
         }
     }
     // one CTA per tile; full tiles and packed tiles (short runs sharing a CTA) in two launches
-    const int n_ctas = (int)L->n_tiles;
+    p.tiles = L->d_tiles;
     p.n_tiles = L->n_regular;
     dte_status s = launch_extract(p, div_bc1, div_decay, false, st);
     if (s != DTE_OK) return s;
@@ -139,15 +136,15 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
     s = launch_extract(p, div_bc1, div_decay, true, st);
     if (s != DTE_OK) return s;
     GatherParams g;
-    g.rec = L->d_rec;
-    g.block_sum = L->d_block_sum;
-    g.n_rec = (uint32_t)n_rec;
-    g.n_blocks = (uint32_t)((n_rec + kRecsPerBlock - 1) / kRecsPerBlock);
+    g.rec = sc.rec;
+    g.block_sum = sc.block_sum;
+    g.n_rec = L->n_tiles;
+    g.n_blocks = (L->n_tiles + kRecsPerBlock - 1) / kRecsPerBlock;
     g.list_first_rec = L->d_list_first_rec;
     g.n_lists = L->n_lists;
     g.scanned = L->scanned;
-    g.stage_offsets = L->d_stage_offsets;
-    g.stage_values = L->d_stage_values;
+    g.stage_offsets = sc.stage_offsets;
+    g.stage_values = sc.stage_values;
     g.offsets = out->offsets;
     g.values = out->values;
     g.capacity = out->capacity;
@@ -155,11 +152,30 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
     g.counters = out->counters;
     s = launch_gather(g, st);
     if (s != DTE_OK) return s;
-    launches = 3 + (L->n_regular ? 1 : 0) + (L->n_packed ? 1 : 0);
     L->last_launch[0] = L->n_tiles;
-    L->last_launch[1] = (uint64_t)n_ctas;
-    L->last_launch[2] = launches;
+    L->last_launch[1] = L->n_tiles;                         // one CTA per tile
+    L->last_launch[2] = 3 + (L->n_regular ? 1 : 0) + (L->n_packed ? 1 : 0);
     return DTE_OK;
+}
+
+// The ordinary entry points keep their scratch in the layout.  The staging buffer mirrors the
+// caller's capacity; it is (re)allocated only when a call brings a larger capacity than any
+// before it.
+dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out, cudaStream_t st,
+                           const std::vector<GroupConsts>* groups = nullptr) {
+    if (L->n_tiles && out->capacity > L->stage_capacity) {
+        DTE_CUDA(cudaStreamSynchronize(st));
+        cudaFree(L->d_stage_offsets);
+        cudaFree(L->d_stage_values);
+        L->d_stage_offsets = nullptr;
+        L->d_stage_values = nullptr;
+        L->stage_capacity = 0;
+        DTE_CUDA(cudaMalloc((void**)&L->d_stage_offsets, out->capacity * sizeof(uint32_t)));
+        DTE_CUDA(cudaMalloc((void**)&L->d_stage_values, out->capacity * sizeof(uint16_t)));
+        L->stage_capacity = out->capacity;
+    }
+    const Scratch sc{L->d_cursor, L->d_rec, L->d_block_sum, L->d_stage_offsets, L->d_stage_values};
+    return enqueue_kernels(L, c, groups, sc, out, st);
 }
 
 }  // namespace
@@ -517,53 +533,13 @@ extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const f
     if (s != DTE_OK) return s;
     s = sync_source_table(L, theta, m, v, st);
     if (s != DTE_OK) return s;
-    DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
-    if (L->n_tiles == 0) {
-        DTE_CUDA(cudaMemsetAsync(out->list_ptr, 0, (L->n_lists + 1) * sizeof(uint64_t), st));
-        return DTE_OK;
-    }
-    // the array keeps whatever the previous call left: only the cursor has to start at zero
-    // (records and block sums are rewritten in full, staged entries are read only where this
-    // call wrote them)
-    DTE_CUDA(cudaMemsetAsync(base + kStaticCursorOff, 0, sizeof(uint64_t), st));
+    // the array keeps whatever the previous call left; enqueue_kernels clears the one word (the
+    // cursor) that must start at zero and every other part is written before it is read
     const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
-    ExtractParams p;
-    p.tiles = L->d_tiles;
-    p.segs = L->d_segs;
-    p.theta = L->d_ptrs;
-    p.m = L->d_ptrs + L->n_tensors;
-    p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
-    p.cursor = reinterpret_cast<unsigned long long*>(base + kStaticCursorOff);
-    p.rec = reinterpret_cast<uint64_t*>(base + kStaticRecOff);
-    p.stage_offsets = reinterpret_cast<uint32_t*>(base + kStaticStageOffOff);
-    p.stage_values = reinterpret_cast<uint16_t*>(base + kStaticStageValOff);
-    p.stage_capacity = out->capacity;
-    p.n_tiles = L->n_tiles;
-    p.c = c;
-    p.s = make_screen(c);
-    p.tensor_group = nullptr;
-    p.groups = nullptr;
-    p.n_tiles = L->n_regular;
-    s = launch_extract(p, c.bc1 != 1.0f, c.decay != 1.0f, false, st);
-    if (s != DTE_OK) return s;
-    p.tiles = L->d_packed;
-    p.n_tiles = L->n_packed;
-    s = launch_extract(p, c.bc1 != 1.0f, c.decay != 1.0f, true, st);
-    if (s != DTE_OK) return s;
-    GatherParams gp;
-    gp.rec = p.rec;
-    gp.block_sum = reinterpret_cast<uint64_t*>(base + kStaticBlockSumOff);
-    gp.n_rec = L->n_tiles;
-    gp.n_blocks = (L->n_tiles + kRecsPerBlock - 1) / kRecsPerBlock;
-    gp.list_first_rec = L->d_list_first_rec;
-    gp.n_lists = L->n_lists;
-    gp.scanned = L->scanned;
-    gp.stage_offsets = p.stage_offsets;
-    gp.stage_values = p.stage_values;
-    gp.offsets = out->offsets;
-    gp.values = out->values;
-    gp.capacity = out->capacity;
-    gp.list_ptr = out->list_ptr;
-    gp.counters = out->counters;
-    return launch_gather(gp, st);
+    const Scratch sc{reinterpret_cast<uint64_t*>(base + kStaticCursorOff),
+                     reinterpret_cast<uint64_t*>(base + kStaticRecOff),
+                     reinterpret_cast<uint64_t*>(base + kStaticBlockSumOff),
+                     reinterpret_cast<uint32_t*>(base + kStaticStageOffOff),
+                     reinterpret_cast<uint16_t*>(base + kStaticStageValOff)};
+    return enqueue_kernels(L, c, nullptr, sc, out, st);
 }
