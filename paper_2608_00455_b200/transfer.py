@@ -66,6 +66,9 @@ class TwoRoundTransfer:
         assert self.op_dst_shard.shape == self.op_sender.shape
         self.rank_of_sender = [int(r) for r in rank_of_sender]
         self.rank_of_receiver = [int(r) for r in rank_of_receiver]
+        # two routes between the same pair of ranks in one direction would share a message order
+        assert len(set(self.rank_of_sender)) == len(self.rank_of_sender), "one sender role per rank"
+        assert len(set(self.rank_of_receiver)) == len(self.rank_of_receiver), "one receiver role per rank"
         self.n_shards = int(self.shard_receivers.size)
         self.group = group
         # Issue the round-2 calls of a pair even when its total is zero (the paper's matched
