@@ -98,11 +98,56 @@ def test_config3_full_qwen3_8b_state():
     # all 11 tensors of layer 17 (row- and column-split, replicated norms) and embed_tokens
     names = plan.tensor_names
     sample = [p for p, n in enumerate(names) if n.startswith("layers.17.")] + [names.index("embed_tokens")]
-    lists, _ = _sampled_lists_equal(wl, st, d, sample)
+    lists, want = _sampled_lists_equal(wl, st, d, sample)
     assert len(lists) == 18
     assert _apply_end_state(plan, st, lay, d, shards, lists) <= 8
-    del st, shards, d, lay
+    del shards
     _free()
+    _storage_path_at_full_size(wl, st, lay, d, lists, want)
+    del st, d, lay
+    _free()
+
+
+def _storage_path_at_full_size(wl, st, lay, d, lists, want):
+    """Canonical extract -> chunks -> verified read-back -> destination-side mapping, whole state;
+    the sampled receiver tensors must hold exactly the oracle's lists scattered into zeros."""
+    from synth import plans
+    plan = wl.plan
+    ident = plans.canonical_plan(plan.tensor_names, plan.tensor_shapes)
+    lay_c = dte.Layout.from_plan(ident, 0)
+    d_c = lay_c.new_delta(d.capacity)
+    dte.dte_extract_delta(lay_c, lay_c.source_tables(st.theta, st.m, st.v), *wl.hp.as_args(), d_c)
+    torch.cuda.synchronize()
+    assert d_c.status_bits() == 0
+    M = d_c.total()
+    assert abs(M - d.total()) < 100_000          # only the replicated norms differ
+    cs = dte.ChunkStream(lay_c.num_lists, M, 16384, dte.DTE_CHUNK_BYTE_PLANES, lay_c.device)
+    dte.dte_pack_chunks(lay_c, d_c, cs)
+    n_chunks, nbytes, bits, entries = (int(x) for x in cs.info.cpu().tolist())
+    assert bits == 0 and entries == M and n_chunks >= M // 16384
+    # sampled chunks against the oracle's writer: the first chunks of the stream (tensor 0)
+    lp = d_c.list_ptr.cpu().numpy().astype(np.uint64)
+    n0 = int(lp[1])
+    o_stream, o_dir = oracle.pack_chunks(lp[:2], d_c.offsets[:n0].cpu().numpy().view(np.uint32),
+                                         d_c.values[:n0].cpu().numpy().view(np.uint16), 16384, 1)
+    assert np.array_equal(cs.stream[:o_stream.size].cpu().numpy(), o_stream)
+    back = lay_c.new_delta(M)
+    back.list_ptr.copy_(d_c.list_ptr)
+    dte.dte_unpack_chunks(lay_c, cs.stream, cs.directory, n_chunks, back, nbytes=nbytes)
+    torch.cuda.synchronize()
+    assert back.counters.cpu().tolist() == [M, n_chunks, 0, 0]
+    assert torch.equal(back.offsets[:M], d_c.offsets[:M]) and torch.equal(back.values[:M], d_c.values[:M])
+    shards2 = [torch.zeros(n, dtype=torch.int16, device="cuda") if k in lists else None
+               for k, n in enumerate(plan.shard_numels)]
+    dte.dte_apply_canonical(lay, back, lay.shard_table(shards2))
+    torch.cuda.synchronize()
+    assert back.status_bits() == 0
+    w_lp, w_off, w_val = want
+    for k in lists:
+        exp = np.zeros(plan.shard_numels[k], np.uint16)
+        seg = slice(int(w_lp[k]), int(w_lp[k + 1]))
+        exp[w_off[seg]] = w_val[seg]
+        assert np.array_equal(shards2[k].cpu().numpy().view(np.uint16), exp), plan.shard_names[k]
 
 
 def test_config4_qwen3_30b_a3b_slice():
