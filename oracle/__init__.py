@@ -223,7 +223,7 @@ def pack_chunks(list_ptr, offsets, values, chunk_entries, fmt=0):
     args = (n_lists, lp.ctypes.data, off.ctypes.data, val.ctypes.data, int(chunk_entries), int(fmt))
     size = lib().oracle_pack_chunks(*args, None, None, n_chunks.ctypes.data)
     if size == 2 ** 64 - 1:
-        raise ValueError("chunk_entries must be a positive multiple of 8 and fmt 0 or 1")
+        raise ValueError("chunk_entries must be a positive multiple of 8 and fmt 0, 1 or 2")
     stream = np.zeros(int(size), np.uint8)
     directory = np.zeros((int(n_chunks[0]) + 1, 3), np.uint64)
     lib().oracle_pack_chunks(*args, stream.ctypes.data, directory.ctypes.data, n_chunks.ctypes.data)

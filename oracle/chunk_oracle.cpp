@@ -20,6 +20,10 @@
 //             bytes each - byte 0, 1, 2, 3 of every index, then byte 0, 1 of every value - each
 //             zero-padded to P.  Same information, transposed so that a byte-oriented
 //             compressor sees the slowly varying high bytes together.
+//   payload, format 2 (delta byte planes): as format 1, but the index planes hold the gaps
+//             g_0 = index_0, g_i = index_i - index_{i-1} (entries of a list ascend, so gaps are
+//             small and their upper planes are almost all zero); the reader restores the indices
+//             by a running sum modulo 2^32.
 //   checksum = Adler-32 (RFC 1950) of the first 24 header bytes followed by the payload
 //             bytes, padding included (so a damaged count or list is caught as well)
 //   directory entry per chunk = {byte offset in the stream, list, first_entry}; one more entry
@@ -39,6 +43,8 @@ constexpr uint32_t kMagic = 0x43455444u;
 constexpr uint32_t kHeaderBytes = 32;
 
 inline uint64_t round16(uint64_t x) { return (x + 15) / 16 * 16; }
+
+constexpr uint32_t kFormats = 3;
 
 inline uint64_t payload_bytes(uint64_t count, uint32_t format) {
     return format == 0 ? round16(6 * count) : 6 * round16(count);
@@ -82,7 +88,9 @@ void write_payload(uint8_t* pay, const uint32_t* idx, const uint16_t* val, uint6
     } else {
         const uint64_t P = round16(count);
         for (uint64_t i = 0; i < count; ++i) {
-            for (int b = 0; b < 4; ++b) pay[b * P + i] = (uint8_t)((idx[i] >> (8 * b)) & 0xFF);
+            uint32_t x = idx[i];
+            if (format == 2 && i > 0) x = idx[i] - idx[i - 1];   // the gap to the previous entry of the chunk
+            for (int b = 0; b < 4; ++b) pay[b * P + i] = (uint8_t)((x >> (8 * b)) & 0xFF);
             pay[4 * P + i] = (uint8_t)(val[i] & 0xFF);
             pay[5 * P + i] = (uint8_t)(val[i] >> 8);
         }
@@ -101,7 +109,7 @@ uint32_t oracle_adler32(const uint8_t* p, uint64_t n) { return adler32(p, n); }
 uint64_t oracle_pack_chunks(uint64_t n_lists, const uint64_t* list_ptr, const uint32_t* offsets,
                             const uint16_t* values, uint32_t chunk_entries, uint32_t format,
                             uint8_t* out, uint64_t* dir, uint64_t* n_chunks) {
-    if (chunk_entries == 0 || chunk_entries % 8 != 0 || format > 1) return UINT64_MAX;
+    if (chunk_entries == 0 || chunk_entries % 8 != 0 || format >= kFormats) return UINT64_MAX;
     uint64_t bytes = 0, chunks = 0;
     for (uint64_t l = 0; l < n_lists; ++l) {
         const uint64_t n = list_ptr[l + 1] - list_ptr[l];
@@ -162,7 +170,7 @@ uint64_t oracle_unpack_chunks(const uint8_t* stream, uint64_t stream_bytes, cons
         const uint32_t magic = get_u32(h), format = get_u32(h + 4), list = get_u32(h + 8);
         const uint32_t first = get_u32(h + 12), count = get_u32(h + 16), pb = get_u32(h + 20);
         const uint32_t sum = get_u32(h + 24);
-        bool ok = magic == kMagic && format <= 1 && list < n_lists &&
+        bool ok = magic == kMagic && format < kFormats && list < n_lists &&
                   count > 0;
         ok = ok && list == dir[3 * c + 1] && first == dir[3 * c + 2];
         ok = ok && (uint64_t)first + count <= list_ptr[list + 1] - list_ptr[list];
@@ -183,9 +191,12 @@ uint64_t oracle_unpack_chunks(const uint8_t* stream, uint64_t stream_bytes, cons
             }
         } else {
             const uint64_t P = round16(count);
+            uint32_t running = 0;
             for (uint32_t i = 0; i < count; ++i) {
-                o[i] = (uint32_t)pay[i] | ((uint32_t)pay[P + i] << 8) |
-                       ((uint32_t)pay[2 * P + i] << 16) | ((uint32_t)pay[3 * P + i] << 24);
+                const uint32_t x = (uint32_t)pay[i] | ((uint32_t)pay[P + i] << 8) |
+                                   ((uint32_t)pay[2 * P + i] << 16) | ((uint32_t)pay[3 * P + i] << 24);
+                running = format == 2 ? running + x : x;       // gaps add up to the index
+                o[i] = running;
                 v[i] = (uint16_t)(pay[4 * P + i] | (pay[5 * P + i] << 8));
             }
         }

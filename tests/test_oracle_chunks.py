@@ -40,6 +40,16 @@ def _hand_stream_planes():
     return _header(1, 0, 0, 3, p0) + p0 + _header(1, 2, 0, 2, p1) + p1
 
 
+def _hand_stream_delta_planes():
+    # as the byte planes, but the index planes hold 1, 258 - 1 = 257 = 0x101, 70000 - 258 = 69742 = 0x1106E
+    def plane(*b):
+        return bytes(b) + bytes(16 - len(b))
+    p0 = (plane(0x01, 0x01, 0x6E) + plane(0x00, 0x01, 0x10) + plane(0x00, 0x00, 0x01) + plane() +
+          plane(0x00, 0x01, 0x01) + plane(0x3C, 0xBC, 0x00))
+    p1 = (plane(0x07, 0x02) + plane() + plane() + plane() + plane(0x00, 0xC0) + plane(0x80, 0x7F))
+    return _header(2, 0, 0, 3, p0) + p0 + _header(2, 2, 0, 2, p1) + p1
+
+
 def test_adler32_matches_zlib_and_the_published_example():
     assert oracle.adler32(b"Wikipedia") == 0x11E60398
     assert oracle.adler32(b"") == 1
@@ -50,12 +60,13 @@ def test_adler32_matches_zlib_and_the_published_example():
     assert oracle.adler32(b"\xff" * 300000) == zlib.adler32(b"\xff" * 300000)
 
 
-@pytest.mark.parametrize("fmt,hand", [(0, _hand_stream_plain), (1, _hand_stream_planes)])
+@pytest.mark.parametrize("fmt,hand", [(0, _hand_stream_plain), (1, _hand_stream_planes),
+                                      (2, _hand_stream_delta_planes)])
 def test_worked_example_matches_the_hand_typed_stream(fmt, hand):
     stream, directory = oracle.pack_chunks(LP, OFF, VAL, 8, fmt)
     expect = hand()
     assert stream.tobytes() == expect
-    sizes = [64, 48] if fmt == 0 else [128, 128]
+    sizes = [64, 48] if fmt == 0 else [128, 128]      # header + payload of the two chunks
     assert directory.tolist() == [[0, 0, 0], [sizes[0], 2, 0], [sizes[0] + sizes[1], 0xFFFFFFFF, 0]]
     off, val, rejected, written = oracle.unpack_chunks(np.frombuffer(expect, np.uint8), directory, LP)
     assert rejected == 0 and written == 5
@@ -72,7 +83,7 @@ def _random_lists(rng, n_lists, max_len):
     return lp, off, val
 
 
-@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("fmt", [0, 1, 2])
 @pytest.mark.parametrize("chunk_entries", [8, 16, 64, 4096])
 def test_round_trip_and_structure(fmt, chunk_entries):
     rng = np.random.default_rng(100 + chunk_entries + fmt)
@@ -100,15 +111,18 @@ def test_round_trip_and_structure(fmt, chunk_entries):
     assert np.array_equal(off2, off) and np.array_equal(val2, val)
 
 
-def test_both_formats_carry_the_same_entries():
+def test_all_formats_carry_the_same_entries():
     rng = np.random.default_rng(9)
     lp, off, val = _random_lists(rng, 7, 1000)
+    off[-1] = 0xFFFFFFF0                                  # indices above 2^31 keep their bits
     a = oracle.unpack_chunks(*oracle.pack_chunks(lp, off, val, 64, 0), lp)
-    b = oracle.unpack_chunks(*oracle.pack_chunks(lp, off, val, 64, 1), lp)
-    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    for fmt in (1, 2):
+        b = oracle.unpack_chunks(*oracle.pack_chunks(lp, off, val, 64, fmt), lp)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    assert np.array_equal(a[0], off) and np.array_equal(a[1], val)
 
 
-@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("fmt", [0, 1, 2])
 def test_every_corrupted_payload_byte_and_header_field_is_rejected(fmt):
     stream, d = oracle.pack_chunks(LP, OFF, VAL, 8, fmt)
     first_chunk = slice(int(LP[0]), int(LP[1]))
@@ -139,7 +153,7 @@ def test_empty_delta_has_no_chunks():
         oracle.pack_chunks(lp, np.zeros(0, np.uint32), np.zeros(0, np.uint16), 12, 0)
 
 
-def test_byte_planes_compress_better_than_the_plain_layout():
+def test_byte_planes_and_gaps_compress_better_than_the_plain_layout():
     pa = pytest.importorskip("pyarrow")
     rng = np.random.default_rng(3)
     mask = rng.random(4_000_000) < 0.015            # the paper's change density
@@ -148,7 +162,8 @@ def test_byte_planes_compress_better_than_the_plain_layout():
     val = oracle.bf16_rne(w)
     lp = np.array([0, off.size], np.uint64)
     size = {}
-    for fmt in (0, 1):
+    for fmt in (0, 1, 2):
         stream, _ = oracle.pack_chunks(lp, off, val, 65536, fmt)
         size[fmt] = len(pa.compress(stream.tobytes(), codec="zstd", asbytes=True))
     assert size[1] < 0.7 * size[0]
+    assert size[2] < 0.92 * size[1]                       # gaps instead of indices: smaller again
