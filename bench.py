@@ -291,7 +291,7 @@ def run_reference(args, rank):
 
 def time_storage_path(dte, wl, st, shards, hp, capacity, device, peak, chunk_entries=16384, reps=5):
     """Storage-mediated path (Section 4.4), outside the timed step: extract over the identity plan
-    (canonical index / value pairs), serialise into byte-plane chunks, verify + read back, map into
+    (canonical index / value pairs), serialise into chunks (byte planes of index gaps), verify + read back, map into
     the receiver layout and store.  Each leg timed with CUDA events, L2 flushed before each call."""
     plan = wl.plan
     ident = plans.canonical_plan(plan.tensor_names, plan.tensor_shapes)
@@ -308,7 +308,7 @@ def time_storage_path(dte, wl, st, shards, hp, capacity, device, peak, chunk_ent
     if d_c.status_bits():
         return {"error": f"canonical extract status bits {d_c.status_bits()}"}
     M = d_c.total()
-    fmt = dte.DTE_CHUNK_BYTE_PLANES
+    fmt = dte.DTE_CHUNK_DELTA_PLANES
     cs = dte.ChunkStream(lay_c.num_lists, M, chunk_entries, fmt, device)
     back = lay_c.new_delta(M)
     back.list_ptr.copy_(d_c.list_ptr)
@@ -341,8 +341,8 @@ def time_storage_path(dte, wl, st, shards, hp, capacity, device, peak, chunk_ent
     moved = 6.0 * M + nbytes
     n_src = sum(plan.numel(p) for p in used)
     del theta
-    return {"format": "byte planes", "chunk_entries": chunk_entries, "chunks": n_chunks, "stream_bytes": nbytes,
-            "entries": M, "canonical_elements": n_src,
+    return {"format": "byte planes of index gaps", "chunk_entries": chunk_entries, "chunks": n_chunks,
+            "stream_bytes": nbytes, "entries": M, "canonical_elements": n_src,
             "extract_canonical_ms": avg["extract_canonical"],
             "extract_canonical_GBps": (12.0 * lay_c.num_elements + 6.0 * M) / (avg["extract_canonical"] * 1e-3) / 1e9,
             "pack_ms": avg["pack"], "unpack_ms": avg["unpack"], "map_and_store_ms": avg["map_and_store"],

@@ -258,7 +258,10 @@ DTE_API size_t dte_layout_num_ops(const dte_layout* layout);
  *             multiple of 16 bytes: byte 0, 1, 2, 3 of every index, byte 0, 1 of every value,
  *             each zero-padded; the same entries transposed so that a byte-oriented compressor
  *             (the paper uses Zstandard, a host library outside this path) finds the slowly
- *             varying bytes together.
+ *             varying bytes together.  DTE_CHUNK_DELTA_PLANES - as the byte planes, but the index
+ *             planes hold the gaps g_0 = index_0, g_i = index_i - index_{i-1} within the chunk
+ *             (lists ascend, so the upper gap planes are almost all zero); the reader restores
+ *             the indices by a running sum modulo 2^32.  Smallest under a compressor.
  *   checksum: Adler-32 (RFC 1950) of header bytes [0, 24) followed by the payload.
  *   directory (the manifest's locations): one dte_chunk_ref per chunk and a final entry
  *             {total bytes, 0xFFFFFFFF, 0}.
@@ -268,6 +271,7 @@ DTE_API size_t dte_layout_num_ops(const dte_layout* layout);
 #define DTE_CHUNK_HEADER_BYTES 32u
 #define DTE_CHUNK_PLAIN 0u
 #define DTE_CHUNK_BYTE_PLANES 1u
+#define DTE_CHUNK_DELTA_PLANES 2u
 #define DTE_CHUNK_MAX_ENTRIES 1048576u
 
 typedef struct dte_chunk_ref {

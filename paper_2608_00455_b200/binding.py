@@ -18,7 +18,7 @@ from . import build as _build
 
 DTE_OK = 0
 DTE_DEV_OVERFLOW, DTE_DEV_BOUNDS, DTE_DEV_TIMEOUT, DTE_DEV_CORRUPT = 1, 2, 4, 8
-DTE_CHUNK_PLAIN, DTE_CHUNK_BYTE_PLANES = 0, 1
+DTE_CHUNK_PLAIN, DTE_CHUNK_BYTE_PLANES, DTE_CHUNK_DELTA_PLANES = 0, 1, 2
 DTE_CHUNK_MAGIC, DTE_CHUNK_HEADER_BYTES, DTE_CHUNK_MAX_ENTRIES = 0x43455444, 32, 1 << 20
 
 SYMBOLS = [

@@ -355,7 +355,7 @@ extern "C" dte_status dte_pack_chunks(const dte_layout* layout, const dte_delta*
     if (s != DTE_OK) return s;
     if (chunk_entries < 8 || chunk_entries % 8 != 0 || chunk_entries > DTE_CHUNK_MAX_ENTRIES)
         return fail(DTE_ERR_INVALID_ARG, "chunk_entries must be a multiple of 8 in [8, DTE_CHUNK_MAX_ENTRIES]");
-    if (format > DTE_CHUNK_BYTE_PLANES) return fail(DTE_ERR_INVALID_ARG, "unknown chunk format");
+    if (format > DTE_CHUNK_DELTA_PLANES) return fail(DTE_ERR_INVALID_ARG, "unknown chunk format");
     if (!directory || !info) return fail(DTE_ERR_INVALID_ARG, "directory / info is null");
     if (stream_capacity && !stream) return fail(DTE_ERR_INVALID_ARG, "stream is null with capacity > 0");
     if ((uintptr_t)stream & 15u) return fail(DTE_ERR_INVALID_ARG, "stream must be 16-byte aligned");

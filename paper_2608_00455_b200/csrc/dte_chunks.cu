@@ -209,6 +209,13 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_pack_kernel(const PackPar
                     o[e] = in ? src_o[i + e] : 0u;
                     v[e] = in ? (uint32_t)src_v[i + e] : 0u;
                 }
+                if (p.format == DTE_CHUNK_DELTA_PLANES) {   // gaps to the previous entry of the chunk
+                    const uint32_t before = (i > 0 && i < count) ? src_o[i - 1] : 0u;
+#pragma unroll
+                    for (int e = 3; e > 0; --e)
+                        if (i + e < count) o[e] -= o[e - 1];
+                    o[0] -= before;
+                }
                 const uint32_t lo01 = __byte_perm(o[0], o[1], 0x5140), lo23 = __byte_perm(o[2], o[3], 0x5140);
                 const uint32_t hi01 = __byte_perm(o[0], o[1], 0x7362), hi23 = __byte_perm(o[2], o[3], 0x7362);
                 const uint32_t v01 = v[0] | (v[1] << 16), v23 = v[2] | (v[3] << 16);
@@ -241,6 +248,9 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_pack_kernel(const PackPar
 // ---- unpack ----------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kChunkThreads) chunk_unpack_kernel(const UnpackParams p) {
     __shared__ uint64_t s_red[2 * (kChunkThreads / 32)];
+    __shared__ uint32_t s_scan[kChunkThreads / 32];
+    __shared__ __align__(16) uint32_t s_o[4 * kChunkThreads];   // one decode step of the plane layouts
+    __shared__ __align__(16) uint16_t s_v[4 * kChunkThreads];
     const uint32_t tid = threadIdx.x;
     const uint64_t total = p.list_ptr[p.n_lists];
     uint64_t accepted = 0, rejected = 0, written = 0;   // meaningful in thread 0
@@ -259,7 +269,7 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_unpack_kernel(const Unpac
             h[4] = b.x; h[5] = b.y; h[6] = b.z; h[7] = b.w;
         }
         const uint32_t format = h[1], list = h[2], first = h[3], count = h[4], pb = h[5];
-        ok = ok && h[0] == DTE_CHUNK_MAGIC && format <= DTE_CHUNK_BYTE_PLANES && list < p.n_lists &&
+        ok = ok && h[0] == DTE_CHUNK_MAGIC && format <= DTE_CHUNK_DELTA_PLANES && list < p.n_lists &&
              count > 0 && list == ref.list && first == ref.first_entry;
         uint64_t lbeg = 0;
         if (ok) {
@@ -325,10 +335,16 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_unpack_kernel(const Unpac
             }
         } else {
             const uint32_t P = (uint32_t)round16(count);
-            for (uint32_t i = 4 * tid; i < count; i += 4 * kChunkThreads) {
-                uint32_t plane[6];
+            const bool gaps = format == DTE_CHUNK_DELTA_PLANES;
+            uint32_t carry = 0;                       // gaps: sum of all gaps before this step's entries
+            // uniform trip count: every thread takes part in the scan of every step
+            for (uint32_t i0 = 0; i0 < count; i0 += 4 * kChunkThreads) {
+                const uint32_t i = i0 + 4 * tid;
+                uint32_t plane[6] = {0, 0, 0, 0, 0, 0};
+                if (i < count) {
 #pragma unroll
-                for (int b = 0; b < 6; ++b) plane[b] = *reinterpret_cast<const uint32_t*>(pay + b * P + i);
+                    for (int b = 0; b < 6; ++b) plane[b] = *reinterpret_cast<const uint32_t*>(pay + b * P + i);
+                }
                 const uint32_t lo01 = __byte_perm(plane[0], plane[1], 0x5140);   // e0: b0 b1, e1: b0 b1
                 const uint32_t lo23 = __byte_perm(plane[0], plane[1], 0x7362);
                 const uint32_t hi01 = __byte_perm(plane[2], plane[3], 0x5140);
@@ -341,12 +357,44 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_unpack_kernel(const Unpac
                 const uint32_t v01 = __byte_perm(plane[4], plane[5], 0x5140);
                 const uint32_t v23 = __byte_perm(plane[4], plane[5], 0x7362);
                 v[0] = v01 & 0xFFFF; v[1] = v01 >> 16; v[2] = v23 & 0xFFFF; v[3] = v23 >> 16;
+                if (gaps) {   // index = running sum of the gaps (mod 2^32): thread, warp, CTA, carry
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (i + e < count) {
-                        out_o[i + e] = o[e];
-                        out_v[i + e] = (uint16_t)v[e];
+                    for (int e = 1; e < 4; ++e)
+                        if (i + e < count) o[e] += o[e - 1]; else o[e] = o[e - 1];
+                    const int lane = tid & 31, warp = tid >> 5;
+                    uint32_t incl = o[3];
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                        if (lane >= d) incl += up;
                     }
+                    __syncthreads();                  // s_scan may still be read from the previous step
+                    if (lane == 31) s_scan[warp] = incl;
+                    __syncthreads();
+                    uint32_t before = carry + incl - o[3], step_total = 0;
+#pragma unroll
+                    for (int w = 0; w < kChunkThreads / 32; ++w) {
+                        const uint32_t t = s_scan[w];
+                        if (w < warp) before += t;
+                        step_total += t;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) o[e] += before;
+                    carry += step_total;
+                }
+                // through shared memory, so that the global stores are consecutive across lanes
+                __syncthreads();                      // the previous step's entries have been written out
+                *reinterpret_cast<uint4*>(s_o + 4 * tid) = make_uint4(o[0], o[1], o[2], o[3]);
+                *reinterpret_cast<uint2*>(s_v + 4 * tid) = make_uint2(v[0] | (v[1] << 16), v[2] | (v[3] << 16));
+                __syncthreads();
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const uint32_t r = e * kChunkThreads + tid;
+                    if (i0 + r < count) {
+                        out_o[i0 + r] = s_o[r];
+                        out_v[i0 + r] = s_v[r];
+                    }
+                }
             }
         }
     }

@@ -60,7 +60,7 @@ def test_compute_calls_fail_loudly_without_a_gpu():
         dte.Layout([(4, 4)], [16], [(0, 0, 0, 0, 4, 4, 0, 4, 0, 0)])
 
 
-@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("fmt", [0, 1, 2])
 @pytest.mark.parametrize("chunk_entries", [8, 64, 4096])
 def test_chunk_bounds_cover_what_the_oracle_writes(fmt, chunk_entries):
     # host-only sizing helpers: never smaller than the stream the oracle serialises

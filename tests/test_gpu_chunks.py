@@ -71,7 +71,7 @@ def _unpack(lay, stream, rows, lp, prefill=0):
             d.counters.cpu().numpy().astype(np.uint64), d)
 
 
-@pytest.mark.parametrize("fmt", [dte.DTE_CHUNK_PLAIN, dte.DTE_CHUNK_BYTE_PLANES])
+@pytest.mark.parametrize("fmt", [dte.DTE_CHUNK_PLAIN, dte.DTE_CHUNK_BYTE_PLANES, dte.DTE_CHUNK_DELTA_PLANES])
 @pytest.mark.parametrize("chunk_entries", [8, 64, 4096])
 def test_pack_of_an_extract_result_is_byte_identical(fmt, chunk_entries):
     dense = plans.qwen3_dense_plan(1, 1, True, configs.SMALL_DENSE)
@@ -100,7 +100,7 @@ def test_pack_of_an_extract_result_is_byte_identical(fmt, chunk_entries):
         assert np.array_equal(shards[k].cpu().numpy().view(np.uint16), want[k])
 
 
-@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("fmt", [0, 1, 2])
 def test_full_chunks_ragged_tails_and_empty_lists(fmt):
     lens = [200_003, 0, 65_536, 1, 0, 131_079, 7]
     lp, off, val = _synthetic_lists(11, lens)
@@ -126,7 +126,7 @@ def test_many_lists_cross_the_planner_block():
     lp, off, val = _synthetic_lists(12, lens, numel=1 << 16)
     lay = _layout(len(lens), numel=1 << 16)
     d = _delta_from_lists(lay, lp, off, val)
-    for fmt in (0, 1):
+    for fmt in (0, 1, 2):
         stream, directory, info = _pack(lay, d, 16, fmt).to_host()
         want_stream, want_dir = oracle.pack_chunks(lp, off, val, 16, fmt)
         assert np.array_equal(_dir_rows(directory), want_dir)
@@ -160,7 +160,7 @@ def test_empty_delta_and_overflow_reports():
 def test_bad_arguments_are_rejected_on_the_host():
     lay = _layout(2)
     d = lay.new_delta(16)
-    for chunk_entries, fmt in ((12, 0), (0, 0), (1 << 21, 0), (64, 2)):
+    for chunk_entries, fmt in ((12, 0), (0, 0), (1 << 21, 0), (64, 3)):
         cs = dte.ChunkStream(2, 16, 64, 0, lay.device)
         cs.chunk_entries, cs.format = chunk_entries, fmt
         with pytest.raises(dte.DteError) as e:
@@ -168,7 +168,7 @@ def test_bad_arguments_are_rejected_on_the_host():
         assert e.value.status == 1
 
 
-@pytest.mark.parametrize("fmt", [0, 1])
+@pytest.mark.parametrize("fmt", [0, 1, 2])
 def test_damaged_streams_are_rejected_where_the_oracle_rejects_them(fmt):
     lens = [150, 0, 70, 33]
     numel = 1 << 20

@@ -113,7 +113,7 @@ def test_entries_for_a_missing_shard_are_flagged_by_apply():
     assert d.status_bits() == dte.DTE_DEV_BOUNDS and bool(shards[0].any())
 
 
-@pytest.mark.parametrize("fmt", [dte.DTE_CHUNK_PLAIN, dte.DTE_CHUNK_BYTE_PLANES])
+@pytest.mark.parametrize("fmt", [dte.DTE_CHUNK_PLAIN, dte.DTE_CHUNK_BYTE_PLANES, dte.DTE_CHUNK_DELTA_PLANES])
 def test_whole_storage_path_extract_pack_unpack_map_store(fmt):
     plan = plans.qwen3_moe_plan(1, 4, 4, configs.SMALL_MOE)
     hp = Hyper(step=300, lr=1e-5, wd=0.01)
