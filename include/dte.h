@@ -29,6 +29,10 @@
  *     scanned elements, and a staging buffer of `capacity` (offset, value) pairs.  The
  *     staging buffer is allocated by the first extract call and re-allocated (with a stream
  *     synchronisation) only when a later call passes a larger capacity.
+ *   - Stream capture: a call whose pointer tables equal those of the previous call on the layout
+ *     and whose capacity does not exceed an earlier one only enqueues memsets and kernels, so
+ *     dte_extract_delta + dte_apply can be captured into a CUDA graph after one ordinary call
+ *     and replayed on new contents of the same buffers.
  *   - There is no CPU fallback: every entry point needs a CUDA device.
  */
 #ifndef DTE_H_
