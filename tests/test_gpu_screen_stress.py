@@ -107,3 +107,56 @@ def test_random_bit_patterns_match_oracle(hp):
     lp, off, val = d.to_host()
     assert np.array_equal(lp, want[0]) and np.array_equal(off, want[1]) and np.array_equal(val, want[2])
     assert 0.3 < int(lp[-1]) / n <= 1.0
+
+
+def _wide_exponent_threshold_state(n, hp: Hyper, seed):
+    """Like the near-boundary state, but over EVERY binade of theta and of the second moment:
+    theta a few ulps off a BF16 tie point with any exponent (subnormals included), v with any
+    exponent, m solved (in double) so that the update is 1/8 .. 8 times the distance to the tie -
+    where that needs an m, m-hat or u beyond fp32's range it overflows or underflows, on purpose."""
+    rng = np.random.default_rng(seed)
+    upper = rng.integers(0x0000, 0x7F80, size=n, dtype=np.uint32)
+    sign = rng.integers(0, 2, size=n, dtype=np.uint32) << 31
+    delta = rng.integers(-40, 41, size=n).astype(np.int64)
+    bits = np.clip((upper.astype(np.int64) << 16) + 0x8000 + delta, 0, 0x7F7FFFFF).astype(np.uint32) | sign
+    theta = bits.view(np.float32).copy()
+    vexp = rng.integers(1, 255, size=n, dtype=np.uint32)
+    v = ((vexp << 23) | rng.integers(0, 1 << 23, size=n, dtype=np.uint32)).view(np.float32).copy()
+    with np.errstate(all="ignore"):
+        dist = np.abs(delta).astype(np.float64) * np.spacing(np.abs(theta)).astype(np.float64)
+        dist = np.where(dist == 0, np.spacing(np.abs(theta)).astype(np.float64), dist)
+        factor = 2.0 ** rng.uniform(-3, 3, size=n)
+        c = oracle.derive_constants(*hp.as_args()).astype(np.float64)
+        lr = c[3] if c[3] != 0 else 1.0
+        m64 = dist * factor / abs(lr) * (np.sqrt(v.astype(np.float64) / c[1]) + c[4]) * c[0]
+        m = (m64 * rng.choice([-1.0, 1.0], size=n)).astype(np.float32)
+    return theta, m, v
+
+
+@pytest.mark.parametrize("hp", [
+    Hyper(step=500, lr=1e-6, wd=0.01),
+    Hyper(step=3, lr=1e-3, wd=0.2),
+    Hyper(step=100, lr=1e-6, wd=0.01),
+    Hyper(step=500, lr=1e-4, wd=0.1),
+    Hyper(step=7, lr=1e-3, wd=0.0, eps=0.0),
+    Hyper(step=20, lr=-1e-3, wd=0.5),
+    Hyper(step=2, lr=1e-2, wd=0.01, beta1=0.0, beta2=0.5, eps=1e-30),
+    Hyper(step=40, lr=1e-12, wd=0.0, eps=1e-20),       # tiny lr: huge m-hat and u for a visible step
+    Hyper(step=40, lr=30.0, wd=0.0, eps=1e-3),         # large lr: tiny m-hat and u
+], ids=lambda h: f"t{h.step}-lr{h.lr:g}-wd{h.wd:g}-eps{h.eps:g}")
+def test_threshold_cases_in_every_binade_match_oracle(hp):
+    rows, cols = 2048, 4096
+    n = rows * cols
+    theta, m, v = _wide_exponent_threshold_state(n, hp, seed=1000 + hp.step)
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    c = oracle.derive_constants(*hp.as_args())
+    with np.errstate(all="ignore"):
+        want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), [theta], [m], [v], c)
+    lay = dte.Layout.from_plan(plan, 0)
+    d = lay.new_delta(n)
+    t, mm, vv = (torch.from_numpy(a.copy()).cuda() for a in (theta, m, v))
+    dte.dte_extract_delta(lay, lay.source_tables([t], [mm], [vv]), *hp.as_args(), d)
+    torch.cuda.synchronize()
+    lp, off, val = d.to_host()
+    assert np.array_equal(lp, want[0]) and np.array_equal(off, want[1]) and np.array_equal(val, want[2])
+    assert 0.02 < int(lp[-1]) / n < 0.98
