@@ -126,14 +126,16 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
             div_decay |= g.c.decay != 1.0f;
         }
     }
-    // one CTA per tile; full tiles and packed tiles (short runs sharing a CTA) in two launches
-    p.tiles = L->d_tiles;
-    p.n_tiles = L->n_regular;
-    dte_status s = launch_extract(p, div_bc1, div_decay, false, st);
-    if (s != DTE_OK) return s;
+    // one CTA per tile; packed tiles (short runs sharing a CTA; few) first, then the full tiles,
+    // which may start while the packed launch is still running: the two share nothing but the
+    // staging cursor (atomic) and write different placement records
     p.tiles = L->d_packed;
     p.n_tiles = L->n_packed;
-    s = launch_extract(p, div_bc1, div_decay, true, st);
+    dte_status s = launch_extract(p, div_bc1, div_decay, true, false, st);
+    if (s != DTE_OK) return s;
+    p.tiles = L->d_tiles;
+    p.n_tiles = L->n_regular;
+    s = launch_extract(p, div_bc1, div_decay, false, L->n_packed != 0, st);
     if (s != DTE_OK) return s;
     GatherParams g;
     g.rec = sc.rec;

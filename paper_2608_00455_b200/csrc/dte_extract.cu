@@ -284,6 +284,10 @@ template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED>
 __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const ExtractParams p) {
     // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
     // (dynamic shared memory: kWarps * kWarpTile words, may exceed the 48 KB static limit)
+    // The two launches of one extract (packed tiles, then regular tiles) are independent: let the
+    // second one start while this one still runs (programmatic dependent launch; a no-op when the
+    // next launch in the stream did not ask for it).
+    asm volatile("griddepcontrol.launch_dependents;");
     extern __shared__ __align__(16) uint32_t s_queue[];
     __shared__ uint32_t s_count[kWarps];
     __shared__ unsigned long long s_pos;
@@ -393,8 +397,10 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
 
 constexpr size_t kQueueBytes = (size_t)kWarps * kWarpTile * sizeof(uint32_t);
 
+// `overlap`: the launch may begin before the previous kernel in the stream has finished (it must
+// not depend on that kernel's results).
 template <bool A, bool B, bool G, bool P>
-static dte_status launch_t(const ExtractParams& p, cudaStream_t st) {
+static dte_status launch_t(const ExtractParams& p, bool overlap, cudaStream_t st) {
     static bool configured[64] = {false};     // per device: allow more than 48 KB of dynamic shared memory
     int dev = 0;
     DTE_CUDA(cudaGetDevice(&dev));
@@ -403,14 +409,23 @@ static dte_status launch_t(const ExtractParams& p, cudaStream_t st) {
                                       (int)kQueueBytes));
         configured[dev] = true;
     }
-    extract_kernel<A, B, G, P><<<p.n_tiles, kThreads, kQueueBytes, st>>>(p);
-    DTE_CUDA(cudaGetLastError());
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(p.n_tiles);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = kQueueBytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    DTE_CUDA(cudaLaunchKernelEx(&cfg, extract_kernel<A, B, G, P>, p));
     return DTE_OK;
 }
 
 template <bool A, bool B, bool G>
-static dte_status launch_p(const ExtractParams& p, bool packed, cudaStream_t st) {
-    return packed ? launch_t<A, B, G, true>(p, st) : launch_t<A, B, G, false>(p, st);
+static dte_status launch_p(const ExtractParams& p, bool packed, bool overlap, cudaStream_t st) {
+    return packed ? launch_t<A, B, G, true>(p, overlap, st) : launch_t<A, B, G, false>(p, overlap, st);
 }
 
 #ifdef DTE_STATS
@@ -422,19 +437,20 @@ extern "C" __attribute__((visibility("default"))) void dte_debug_stats(unsigned 
 
 // div_bc1 / div_decay: whether any group in the call has a divisor different from 1.0f.
 // One launch covers p.n_tiles tiles of one kind (p.tiles = their descriptors).
-dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, cudaStream_t st) {
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, bool overlap,
+                          cudaStream_t st) {
     if (p.n_tiles == 0) return DTE_OK;
     const bool a = div_bc1, b = div_decay;
     if (p.groups) {
-        if (a && b) return launch_p<true, true, true>(p, packed, st);
-        if (a) return launch_p<true, false, true>(p, packed, st);
-        if (b) return launch_p<false, true, true>(p, packed, st);
-        return launch_p<false, false, true>(p, packed, st);
+        if (a && b) return launch_p<true, true, true>(p, packed, overlap, st);
+        if (a) return launch_p<true, false, true>(p, packed, overlap, st);
+        if (b) return launch_p<false, true, true>(p, packed, overlap, st);
+        return launch_p<false, false, true>(p, packed, overlap, st);
     }
-    if (a && b) return launch_p<true, true, false>(p, packed, st);
-    if (a) return launch_p<true, false, false>(p, packed, st);
-    if (b) return launch_p<false, true, false>(p, packed, st);
-    return launch_p<false, false, false>(p, packed, st);
+    if (a && b) return launch_p<true, true, false>(p, packed, overlap, st);
+    if (a) return launch_p<true, false, false>(p, packed, overlap, st);
+    if (b) return launch_p<false, true, false>(p, packed, overlap, st);
+    return launch_p<false, false, false>(p, packed, overlap, st);
 }
 
 }  // namespace dte

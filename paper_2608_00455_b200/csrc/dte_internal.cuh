@@ -201,7 +201,8 @@ dte_status cuda_fail(cudaError_t e, const char* what);
         if (e__ != cudaSuccess) return dte::cuda_fail(e__, #call); \
     } while (0)
 
-dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, cudaStream_t st);
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, bool overlap,
+                          cudaStream_t st);
 dte_status launch_gather(const GatherParams& p, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 dte_status launch_apply_canonical(const CanonParams& p, int device, cudaStream_t st);
