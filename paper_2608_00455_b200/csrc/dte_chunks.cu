@@ -274,9 +274,10 @@ __global__ void __launch_bounds__(kChunkThreads) chunk_unpack_kernel(const Unpac
         uint64_t lbeg = 0;
         if (ok) {
             lbeg = p.list_ptr[list];
-            const uint64_t llen = p.list_ptr[list + 1] - lbeg;
-            ok = (uint64_t)first + count <= llen && (uint64_t)pb == payload_bytes(count, format) &&
-                 end - begin == kHeaderBytes + (uint64_t)pb;
+            const uint64_t lend = p.list_ptr[list + 1];
+            // the list boundaries come from a manifest too: they must nest inside the buffers
+            ok = lbeg <= lend && lend <= total && (uint64_t)first + count <= lend - lbeg &&
+                 (uint64_t)pb == payload_bytes(count, format) && end - begin == kHeaderBytes + (uint64_t)pb;
         }
         const uint8_t* pay = p.stream + begin + kHeaderBytes;
         if (ok) {   // pass 1: checksum of what is about to be decoded

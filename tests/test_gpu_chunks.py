@@ -207,3 +207,14 @@ def test_damaged_streams_are_rejected_where_the_oracle_rejects_them(fmt):
             torch.cuda.synchronize()
             assert bool((shard == 7).all())
     assert seen_rejections >= len(cases) - 8              # reserved header bytes may be flipped unnoticed
+
+
+def test_list_boundaries_that_do_not_nest_are_rejected():
+    lens = [100, 50]
+    lp, off, val = _synthetic_lists(21, lens, 1 << 20)
+    lay = _layout(2, 1 << 20)
+    stream, rows = oracle.pack_chunks(lp, off, val, 64, 1)
+    bad_lp = lp.copy()
+    bad_lp[1] = 1 << 40                                   # list 0 "ends" far outside the buffers
+    o2, v2, counters, _ = _unpack(lay, stream, rows, bad_lp)
+    assert counters[0] == 0 and counters[3] == rows.shape[0] - 1 and counters[2] & dte.DTE_DEV_CORRUPT
