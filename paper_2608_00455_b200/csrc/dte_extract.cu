@@ -222,10 +222,26 @@ __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint3
     uint32_t qn = 0;
 #pragma unroll 1
     for (uint32_t cb = 0; cb < (FAST ? (uint32_t)kWarpTile : cur.len); cb += kChunk) {
-        if (FAST) {
-            const float4* pt = reinterpret_cast<const float4*>(cur.th + cb) + lane;
-            const float4* pm = reinterpret_cast<const float4*>(cur.mm + cb) + lane;
-            const float4* pv = reinterpret_cast<const float4*>(cur.vv + cb) + lane;
+        // chunk_fast: the whole chunk is inside the warp-tile and contiguous in the source (for a
+        // column-split operation: inside one source row), so its loads need no bounds checks and
+        // one address computation (warp-uniform decision)
+        bool chunk_fast = FAST;
+        uint64_t chunk_off = cb;
+        if (!FAST && !(cur.len_flags & kFlagScalar) && cb + kChunk <= cur.len) {
+            if (cur.len_flags & kFlagStrided) {
+                const uint32_t w = cur.geom->w, cc = cur.col0 + cb;
+                const uint32_t row = (w == 1) ? cc : __umulhi(cc, cur.geom->magic);
+                const uint32_t col = cc - row * w;
+                chunk_fast = col + kChunk <= w;
+                chunk_off = (uint64_t)row * cur.geom->s + col;
+            } else {
+                chunk_fast = true;
+            }
+        }
+        if (chunk_fast) {
+            const float4* pt = reinterpret_cast<const float4*>(cur.th + chunk_off) + lane;
+            const float4* pm = reinterpret_cast<const float4*>(cur.mm + chunk_off) + lane;
+            const float4* pv = reinterpret_cast<const float4*>(cur.vv + chunk_off) + lane;
 #pragma unroll
             for (int i = 0; i < kItems; ++i) {
                 a[i] = __ldg(pt + i * 32);
@@ -241,7 +257,7 @@ __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint3
         for (int i = 0; i < kItems; ++i) {
             const uint32_t e = cb + i * 128 + lane * 4;
             amb[i] = 0;
-            if (FAST || e < cur.len) {
+            if (chunk_fast || e < cur.len) {
                 const float tt[4] = {a[i].x, a[i].y, a[i].z, a[i].w};
                 const float m4[4] = {b[i].x, b[i].y, b[i].z, b[i].w};
                 const float v4[4] = {g[i].x, g[i].y, g[i].z, g[i].w};
