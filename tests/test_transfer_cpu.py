@@ -139,3 +139,16 @@ def test_schedule_is_static_and_symmetric():
         assert all(owners[plan.ops[o][0]] == s and plan.shard_receivers[plan.ops[o][1]] == r for o in rt.ops)
         assert rt.contiguous and np.array_equal(x.sender_ops[s][rt.local_ops], rt.ops)
     assert np.all(covered == 1)                                          # every operation travels exactly once
+
+
+def test_counts_that_disagree_with_the_lists_stop_the_sender():
+    # announced counts and payload length must match before round 2, or a peer would wait forever
+    from paper_2608_00455_b200.transfer import TwoRoundTransfer
+    x = TwoRoundTransfer([0, 0], [0, 1], [0, 0], [0], [0])            # one sender, one receiver, same rank
+    lp = np.array([0, 3, 5], np.uint64)
+    off = torch.arange(5, dtype=torch.int32)
+    val = torch.arange(5, dtype=torch.int16)
+    got = x.exchange(0, 0, 0, lp, off, val, torch.tensor([3, 2]))
+    assert got[0].list_ptr.tolist() == [0, 3, 5] and torch.equal(got[0].offsets, off)
+    with pytest.raises(RuntimeError):
+        x.exchange(0, 0, 0, lp, off, val, torch.tensor([3, 1]))
