@@ -94,19 +94,39 @@ __device__ __forceinline__ float rsqrt_ftz(float x) {
 }
 
 template <bool DIV_BC1, bool DIV_DECAY>
-__device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s, float abs_lr) {
+__device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s, float lr) {
     // boundaries from the raw pattern: the sign bit rides along (no carry reaches it below the NaN
     // range) and is dropped by the |.| operand modifiers, which cost nothing
     const uint32_t u = __float_as_uint(theta);
-    const uint32_t hi = ((u + 0x8000u) & 0xFFFF0000u) | 0x7FFEu;   // boundary above |theta|, minus 2 ulp
-    const uint32_t lo = hi - 0xFFFCu;                               // boundary below, plus 2 ulp
     const float at = fabsf(theta);
-    const float room = min_nan(fabsf(__uint_as_float(hi)) - at, at - fabsf(__uint_as_float(lo)));   // exact differences
+    float room;
+    if (DIV_DECAY) {
+        // the division by decay moves |theta| one way and the step possibly the other: both sides
+        const uint32_t hi = ((u + 0x8000u) & 0xFFFF0000u) | 0x7FFEu;   // boundary above |theta|, minus 2 ulp
+        const uint32_t lo = hi - 0xFFFCu;                               // boundary below, plus 2 ulp
+        room = min_nan(fabsf(__uint_as_float(hi)) - at, at - fabsf(__uint_as_float(lo)));   // exact differences
+    } else {
+        // Without it the reconstruction is RN(theta + lr * u) and u has the sign of m (den >= +0 or
+        // NaN), so the direction is known: |theta| grows when theta and lr * m agree in sign and
+        // shrinks otherwise, and only the boundary on that side matters.  This halves the elements
+        // that reach the exact path (a step larger than the distance to the boundary BEHIND it
+        // cannot change the pattern).  A theta exactly on a tie point belongs to the cell above or
+        // below it depending on parity; each direction takes the cell that has the tie as its
+        // boundary on that side, so a tie never passes.
+        const uint32_t x = u ^ __float_as_uint(m) ^ __float_as_uint(lr);   // sign bit set: shrinks
+        const bool down = (int32_t)x < 0;
+        const uint32_t cell = (u + (down ? 0x8000u : 0x7FFFu)) & 0xFFFF0000u;
+        const uint32_t bnd = down ? cell - 0x7FFEu : cell + 0x7FFEu;       // 2 ulp inside the boundary
+        const float d = fabsf(__uint_as_float(bnd)) - at;                  // exact; negative on the lower side
+        room = __uint_as_float(__float_as_uint(d) ^ (x & 0x80000000u));    // distance to that boundary (or NaN)
+    }
     const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
     const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);   // -Inf for v = -0 or a negative subnormal
-    float b = __fmul_rn(__fmul_rn(am, w), abs_lr);
+    float b = __fmul_rn(__fmul_rn(am, w), fabsf(lr));
     if (DIV_DECAY) b = __fmaf_rn(at, s.kappa, b);
-    return fabsf(b) <= room;            // |b|: a negative v (w = -Inf or NaN) must not pass
+    // |b|: a negative v (w = -Inf or NaN) must not pass.  Strict: theta = +-Inf has room = +Inf on
+    // its lower side, and an infinite bound (the step may be -Inf, the sum NaN) must not pass it.
+    return fabsf(b) < room;
 }
 
 __device__ __forceinline__ const float* ldg_ptr(const float* const* slot) {
@@ -217,7 +237,7 @@ __device__ __forceinline__ void load_chunk(const WarpTile& wt, uint32_t cb, int 
 // queue length.
 template <bool DIV_BC1, bool DIV_DECAY, bool FAST>
 __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint32_t* queue, const Screen& sc,
-                                            float abs_lr) {
+                                            float lr) {
     float4 a[kItems], b[kItems], g[kItems];
     uint32_t qn = 0;
 #pragma unroll 1
@@ -263,7 +283,7 @@ __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint3
                 const float v4[4] = {g[i].x, g[i].y, g[i].z, g[i].w};
 #pragma unroll
                 for (int j = 0; j < 4; ++j)
-                    if (!surely_unchanged<DIV_BC1, DIV_DECAY>(tt[j], m4[j], v4[j], sc, abs_lr)) amb[i] |= 1u << j;
+                    if (!surely_unchanged<DIV_BC1, DIV_DECAY>(tt[j], m4[j], v4[j], sc, lr)) amb[i] |= 1u << j;
                 if (!FAST && (cur.len_flags & kFlagScalar))           // ragged tail of a scalar tile
                     amb[i] &= (1u << min(cur.len - e, 4u)) - 1u;
             }
@@ -327,16 +347,16 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
             sc.ka = __uint_as_float(g1.y); sc.kb = __uint_as_float(g1.z); sc.kc = __uint_as_float(g1.w);
             sc.kappa = __uint_as_float(g2.x);
         }
-        const float abs_lr = fabsf(c.lr);
+        const float lr = c.lr;
 
         // ---- phase A: stream, screen, queue the undecided elements in element order ---------
         // FAST: a full, contiguous, 16-byte-aligned warp-tile (nearly all of them): no bounds
         // checks and no per-item address arithmetic (pointer + immediate).
         uint32_t qn = 0;
         if (cur.len == (uint32_t)kWarpTile && !(cur.len_flags & (kFlagScalar | kFlagStrided)))
-            qn = phase_a<DIV_BC1, DIV_DECAY, true>(cur, lane, queue, sc, abs_lr);
+            qn = phase_a<DIV_BC1, DIV_DECAY, true>(cur, lane, queue, sc, lr);
         else
-            qn = phase_a<DIV_BC1, DIV_DECAY, false>(cur, lane, queue, sc, abs_lr);
+            qn = phase_a<DIV_BC1, DIV_DECAY, false>(cur, lane, queue, sc, lr);
         __syncwarp();
         DTE_STAT(0, qn);
         DTE_STAT(2, (qn + 31) / 32);
