@@ -31,18 +31,19 @@ struct Sums {
     uint64_t s1, s2;
 };
 
-// Adds the four bytes of a little-endian word whose byte 0 has weight `wt` (bytes 1..3: wt-1 ..).
+// Adds the four bytes of a little-endian word whose byte 0 has weight `wt` (bytes 1..3: wt-1 ..):
+// two byte-wise dot products give the plain and the position-weighted byte sums.
 __device__ __forceinline__ void add_word(Sums& a, uint32_t w, uint32_t wt) {
-    const uint32_t b0 = w & 0xFF, b1 = (w >> 8) & 0xFF, b2 = (w >> 16) & 0xFF, b3 = w >> 24;
-    const uint32_t sum = b0 + b1 + b2 + b3;
+    const uint32_t sum = __dp4a(w, 0x01010101u, 0u);       // b0 + b1 + b2 + b3
+    const uint32_t skew = __dp4a(w, 0x03020100u, 0u);      // b1 + 2 b2 + 3 b3
     a.s1 += sum;
-    a.s2 += (uint64_t)wt * sum - (b1 + 2 * b2 + 3 * b3);
+    a.s2 += (uint64_t)wt * sum - skew;
 }
 
 __device__ __forceinline__ void add_half(Sums& a, uint32_t h, uint32_t wt) {
-    const uint32_t b0 = h & 0xFF, b1 = (h >> 8) & 0xFF;
-    a.s1 += b0 + b1;
-    a.s2 += (uint64_t)wt * (b0 + b1) - b1;
+    const uint32_t sum = __dp4a(h, 0x00000101u, 0u);
+    a.s1 += sum;
+    a.s2 += (uint64_t)wt * sum - (h >> 8);
 }
 
 // Sum over the CTA; every thread gets the result.  s_red: 2 * warps words of shared memory.
