@@ -8,7 +8,7 @@ import torch
 
 import oracle
 import paper_2608_00455_b200 as dte
-from gpu_util import run_extract
+from gpu_util import assert_lists_equal, oracle_extract, run_extract
 from synth import configs, plans
 from synth.tensors import Hyper
 
@@ -79,7 +79,9 @@ def test_pack_of_an_extract_result_is_byte_identical(fmt, chunk_entries):
     wl = configs.Workload("canonical", plan, Hyper(step=200, lr=2e-6, wd=0.05), configs._specs(plan), 77)
     st = wl.materialize("cuda")
     lay, d = run_extract(plan, st, wl.hp)
-    lp, off, val = d.to_host()
+    # the oracle's writer is fed the oracle's own lists (which the GPU's must equal), never GPU output
+    lp, off, val = oracle_extract(plan, st, wl.hp)
+    assert_lists_equal(d.to_host(), (lp, off, val), plan)
     assert int(lp[-1]) > 1000
     cs = _pack(lay, d, chunk_entries, fmt)
     stream, directory, info = cs.to_host()

@@ -121,15 +121,19 @@ def _storage_path_at_full_size(wl, st, lay, d, lists, want):
     assert d_c.status_bits() == 0
     M = d_c.total()
     assert abs(M - d.total()) < 100_000          # only the replicated norms differ
-    cs = dte.ChunkStream(lay_c.num_lists, M, 16384, dte.DTE_CHUNK_BYTE_PLANES, lay_c.device)
+    fmt = dte.DTE_CHUNK_DELTA_PLANES
+    cs = dte.ChunkStream(lay_c.num_lists, M, 16384, fmt, lay_c.device)
     dte.dte_pack_chunks(lay_c, d_c, cs)
     n_chunks, nbytes, bits, entries = (int(x) for x in cs.info.cpu().tolist())
     assert bits == 0 and entries == M and n_chunks >= M // 16384
-    # sampled chunks against the oracle's writer: the first chunks of the stream (tensor 0)
-    lp = d_c.list_ptr.cpu().numpy().astype(np.uint64)
-    n0 = int(lp[1])
-    o_stream, o_dir = oracle.pack_chunks(lp[:2], d_c.offsets[:n0].cpu().numpy().view(np.uint32),
-                                         d_c.values[:n0].cpu().numpy().view(np.uint16), 16384, 1)
+    # sampled chunks against the oracle's writer: the first chunks of the stream (tensor 0), from
+    # the oracle's own canonical list of that tensor
+    shapes, ops0, host = bench.oracle_inputs(ident, st, [0])
+    c = oracle.derive_constants(*wl.hp.as_args())
+    o_lp, o_off, o_val = oracle.extract(shapes, ident.shard_numels, ops0, *host, c)
+    n0 = int(o_lp[1])
+    assert n0 == int(d_c.list_ptr[1].item()) and n0 > 100_000
+    o_stream, o_dir = oracle.pack_chunks(o_lp[:2], o_off[:n0], o_val[:n0], 16384, fmt)
     assert np.array_equal(cs.stream[:o_stream.size].cpu().numpy(), o_stream)
     back = lay_c.new_delta(M)
     back.list_ptr.copy_(d_c.list_ptr)

@@ -8,7 +8,7 @@ import torch
 
 import oracle
 import paper_2608_00455_b200 as dte
-from gpu_util import run_extract
+from gpu_util import assert_lists_equal, oracle_extract, run_extract
 from synth import configs, plans
 from synth.tensors import Hyper, Spec
 
@@ -35,7 +35,9 @@ def test_canonical_entries_mapped_on_the_destination(name):
     st = wl.materialize("cuda")
     ident = plans.canonical_plan(plan.tensor_names, plan.tensor_shapes)
     lay_c, d_c = run_extract(ident, st, hp)                       # sender: canonical (index, value) pairs
-    lp, idx, val = d_c.to_host()
+    # the oracle works on its own canonical lists (which the GPU's must equal), never on GPU output
+    lp, idx, val = oracle_extract(ident, st, hp)
+    assert_lists_equal(d_c.to_host(), (lp, idx, val), ident)
     assert int(lp[-1]) > 0
 
     lay = dte.Layout.from_plan(plan, 0)                           # destination: its plan, its shards
@@ -65,7 +67,8 @@ def test_one_receiver_passes_only_its_own_shards():
     st = wl.materialize("cuda")
     ident = plans.canonical_plan(plan.tensor_names, plan.tensor_shapes)
     _, d_c = run_extract(ident, st, hp)
-    lp, idx, val = d_c.to_host()
+    lp, idx, val = oracle_extract(ident, st, hp)
+    assert_lists_equal(d_c.to_host(), (lp, idx, val), ident)
     lay = dte.Layout.from_plan(plan, 0)
     for r in (0, 3):
         mine = [k for k, rr in enumerate(plan.shard_receivers) if rr == r]
