@@ -185,7 +185,7 @@ DTE_API dte_status dte_extract_delta_groups(const dte_layout* layout, const floa
  * latency-critical loop that cannot afford the implicit synchronisation of cudaMalloc /
  * cudaFree.  dte_extract_delta grows a per-layout staging buffer when a call brings a larger
  * `capacity`; this entry point never does.  Its placement records, block sums, cursor and
- * staging buffer live in one fixed array inside the library's device image (about 12.5 MiB;
+ * staging buffer live in one fixed array inside the library's device image (about 8.5 MiB;
  * every GPU that loads the library holds it until the process exits), and it calls no
  * cudaMalloc, cudaFree or other device-allocating routine.
  *   Limits: the layout may have at most DTE_STATIC_MAX_TILES tiles (a tile is the work of one

@@ -81,8 +81,7 @@ struct Scratch {
     uint64_t* cursor;
     uint64_t* rec;
     uint64_t* block_sum;
-    uint32_t* stage_offsets;
-    uint16_t* stage_values;
+    uint32_t* stage;
 };
 
 // Enqueues the kernels of one extract: both extract launches (regular and packed tiles), then
@@ -106,8 +105,7 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
     p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
     p.cursor = reinterpret_cast<unsigned long long*>(sc.cursor);
     p.rec = sc.rec;
-    p.stage_offsets = sc.stage_offsets;
-    p.stage_values = sc.stage_values;
+    p.stage = sc.stage;
     p.stage_capacity = out->capacity;
     p.c = c;
     p.s = make_screen(c);
@@ -145,8 +143,9 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
     g.list_first_rec = L->d_list_first_rec;
     g.n_lists = L->n_lists;
     g.scanned = L->scanned;
-    g.stage_offsets = sc.stage_offsets;
-    g.stage_values = sc.stage_values;
+    g.stage = sc.stage;
+    g.rec_base = L->d_rec_base;
+    g.packed = L->d_packed;
     g.offsets = out->offsets;
     g.values = out->values;
     g.capacity = out->capacity;
@@ -167,16 +166,13 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
                            const std::vector<GroupConsts>* groups = nullptr) {
     if (L->n_tiles && out->capacity > L->stage_capacity) {
         DTE_CUDA(cudaStreamSynchronize(st));
-        cudaFree(L->d_stage_offsets);
-        cudaFree(L->d_stage_values);
-        L->d_stage_offsets = nullptr;
-        L->d_stage_values = nullptr;
+        cudaFree(L->d_stage);
+        L->d_stage = nullptr;
         L->stage_capacity = 0;
-        DTE_CUDA(cudaMalloc((void**)&L->d_stage_offsets, out->capacity * sizeof(uint32_t)));
-        DTE_CUDA(cudaMalloc((void**)&L->d_stage_values, out->capacity * sizeof(uint16_t)));
+        DTE_CUDA(cudaMalloc((void**)&L->d_stage, out->capacity * sizeof(uint32_t)));
         L->stage_capacity = out->capacity;
     }
-    const Scratch sc{L->d_cursor, L->d_rec, L->d_block_sum, L->d_stage_offsets, L->d_stage_values};
+    const Scratch sc{L->d_cursor, L->d_rec, L->d_block_sum, L->d_stage};
     return enqueue_kernels(L, c, groups, sc, out, st);
 }
 
@@ -474,12 +470,10 @@ constexpr uint64_t kStaticMaxCapacity = DTE_STATIC_MAX_CAPACITY;
 constexpr uint64_t kStaticCursorOff = 0;                                       // 256 bytes reserved
 constexpr uint64_t kStaticRecOff = 256;
 constexpr uint64_t kStaticBlockSumOff = kStaticRecOff + kStaticMaxTiles * 8;
-constexpr uint64_t kStaticStageOffOff =
+constexpr uint64_t kStaticStageOff =
     kStaticBlockSumOff + ((kStaticMaxTiles + kRecsPerBlock - 1) / kRecsPerBlock) * 8;
-constexpr uint64_t kStaticStageValOff = kStaticStageOffOff + kStaticMaxCapacity * 4;
-constexpr uint64_t kStaticScratchBytes = (kStaticStageValOff + kStaticMaxCapacity * 2 + 255) / 256 * 256;
-static_assert(kStaticBlockSumOff % 8 == 0 && kStaticStageOffOff % 8 == 0 && kStaticStageValOff % 4 == 0,
-              "sub-buffers must keep their natural alignment");
+constexpr uint64_t kStaticScratchBytes = (kStaticStageOff + kStaticMaxCapacity * 4 + 255) / 256 * 256;
+static_assert(kStaticBlockSumOff % 8 == 0 && kStaticStageOff % 8 == 0, "sub-buffers must keep their natural alignment");
 
 // In host code this name is only a handle for the runtime's symbol table, never a device
 // address: the address each device gave the array comes from cudaGetSymbolAddress below.
@@ -541,7 +535,6 @@ extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const f
     const Scratch sc{reinterpret_cast<uint64_t*>(base + kStaticCursorOff),
                      reinterpret_cast<uint64_t*>(base + kStaticRecOff),
                      reinterpret_cast<uint64_t*>(base + kStaticBlockSumOff),
-                     reinterpret_cast<uint32_t*>(base + kStaticStageOffOff),
-                     reinterpret_cast<uint16_t*>(base + kStaticStageValOff)};
+                     reinterpret_cast<uint32_t*>(base + kStaticStageOff)};
     return enqueue_kernels(L, c, nullptr, sc, out, st);
 }

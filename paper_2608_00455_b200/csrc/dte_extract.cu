@@ -420,14 +420,10 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
         }
         __syncthreads();
         const unsigned long long pos = s_pos + before;
-        const uint32_t dst0 = cur.dst0;
-        for (uint32_t q = lane; q < n_changed; q += 32) {
-            const uint32_t entry = queue[q];
-            if (pos + q < p.stage_capacity) {         // beyond it the call overflows anyway
-                p.stage_offsets[pos + q] = dst0 + (entry & 0xFFFFu);
-                p.stage_values[pos + q] = (uint16_t)(entry >> 16);
-            }
-        }
+        const uint32_t rel = (uint32_t)warp * kWarpTile;        // tile-relative index: < kTile < 2^16, no carry
+        for (uint32_t q = lane; q < n_changed; q += 32)
+            if (pos + q < p.stage_capacity)               // beyond it the call overflows anyway
+                p.stage[pos + q] = queue[q] + rel;
     }
 }
 

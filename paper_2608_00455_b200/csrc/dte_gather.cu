@@ -136,33 +136,49 @@ __global__ void __launch_bounds__(kGatherThreads) gather_move_kernel(const Gathe
     // warp w moves records 8w .. 8w+7; the eight copies are interleaved so that eight
     // independent loads per lane are in flight (a record holds ~125 entries: few rounds)
     (void)block_total;
-    uint32_t cnt8[kRecsPerWarp];
-    uint64_t src8[kRecsPerWarp], dst8[kRecsPerWarp];
-    uint32_t longest = 0;
+    uint32_t cnt8[kRecsPerWarp], base8[kRecsPerWarp];
+    const uint32_t* src8[kRecsPerWarp];
+    uint32_t* off8[kRecsPerWarp];
+    uint16_t* val8[kRecsPerWarp];
+    uint32_t longest = 0, packed_recs = 0;
 #pragma unroll
     for (int r = 0; r < kRecsPerWarp; ++r) {
         const uint32_t j = warp * kRecsPerWarp + r;
         const uint32_t first = s_prefix[j];
         cnt8[r] = s_prefix[j + 1] - first;
-        src8[r] = s_pos[j];
-        dst8[r] = out_base + first;
+        src8[r] = p.stage + s_pos[j];
+        off8[r] = p.offsets + (out_base + first);
+        val8[r] = p.values + (out_base + first);
+        const uint64_t b = cnt8[r] ? p.rec_base[base_rec + j] : 0ull;
+        base8[r] = (uint32_t)b;
+        if (b & kRecBasePacked) packed_recs |= 1u << r;
         longest = max(longest, cnt8[r]);
     }
     for (uint32_t q = lane; q < longest; q += 32) {
-        uint32_t o[kRecsPerWarp];
-        uint16_t v[kRecsPerWarp];
+        uint32_t w[kRecsPerWarp];
+#pragma unroll
+        for (int r = 0; r < kRecsPerWarp; ++r)
+            if (q < cnt8[r]) w[r] = src8[r][q];
 #pragma unroll
         for (int r = 0; r < kRecsPerWarp; ++r)
             if (q < cnt8[r]) {
-                o[r] = p.stage_offsets[src8[r] + q];
-                v[r] = p.stage_values[src8[r] + q];
+                // a regular tile is one destination run: base + (warp * kWarpTile + index); the
+                // offsets of packed tiles are put right below
+                off8[r][q] = base8[r] + (w[r] & 0xFFFFu);
+                val8[r][q] = (uint16_t)(w[r] >> 16);
             }
+    }
+    // packed tiles (few): every piece has a destination base of its own
+    if (packed_recs == 0) return;
 #pragma unroll
-        for (int r = 0; r < kRecsPerWarp; ++r)
-            if (q < cnt8[r]) {
-                p.offsets[dst8[r] + q] = o[r];
-                p.values[dst8[r] + q] = v[r];
-            }
+    for (int r = 0; r < kRecsPerWarp; ++r) {
+        if (!(packed_recs & (1u << r))) continue;
+        const TileDesc* d = p.packed + (size_t)base8[r] * kSub;
+        for (uint32_t q = lane; q < cnt8[r]; q += 32) {
+            const uint32_t idx = src8[r][q] & 0xFFFFu;
+            const uint32_t piece = idx / kWarpTile;
+            off8[r][q] = __ldg(&d[piece].dst_off) + (idx - piece * kWarpTile);
+        }
     }
 }
 

@@ -68,6 +68,12 @@ struct SegRec {
 constexpr int kRecCountBits = 14;                      // count <= kTile
 constexpr uint64_t kRecCountMask = (1ull << kRecCountBits) - 1;
 constexpr int kRecsPerBlock = 64;                      // records one gather CTA handles
+// A staged entry is one 32-bit word: (warp * kWarpTile + element index in the warp-tile) in the low
+// 16 bits, the BF16 value in the high 16.  The gather turns it into (offset, value) with the tile's
+// destination base: rec_base[r] = dst_off of a regular tile, or kRecBasePacked | index of a packed
+// tile, whose eight pieces have a dst_off each.  (Writing full offsets and values into two staging
+// arrays cost a third more write traffic in the middle of the read stream.)
+constexpr uint64_t kRecBasePacked = 1ull << 63;
 
 struct Consts {
     float bc1, bc2, decay, lr, eps;
@@ -94,8 +100,7 @@ struct ExtractParams {
     const float* const* v;
     unsigned long long* cursor;  // zeroed before launch: entries appended to the staging buffer
     uint64_t* rec;               // n_tiles placement records (written in full)
-    uint32_t* stage_offsets;     // staging buffer, stage_capacity entries
-    uint16_t* stage_values;
+    uint32_t* stage;             // staging buffer, stage_capacity words: tile-relative index | value << 16
     uint64_t stage_capacity;
     uint32_t n_tiles;            // tiles handled by this launch
     Consts c;                    // single-group calls: constants in the kernel parameters
@@ -111,8 +116,9 @@ struct GatherParams {
     const uint32_t* list_first_rec;  // n_lists: first record of each list (n_rec if none follows)
     uint32_t n_lists;
     uint64_t scanned;
-    const uint32_t* stage_offsets;
-    const uint16_t* stage_values;
+    const uint32_t* stage;           // staged words (see ExtractParams)
+    const uint64_t* rec_base;        // n_rec: destination base of each tile (see kRecBasePacked)
+    const TileDesc* packed;          // packed descriptors, kSub per packed tile
     uint32_t* offsets;
     uint16_t* values;
     uint64_t capacity;
@@ -230,8 +236,8 @@ struct dte_layout {
     uint64_t* d_rec = nullptr;             // n_tiles placement records
     uint64_t* d_block_sum = nullptr;       // one word per gather block
     uint64_t* d_cursor = nullptr;          // staging cursor
-    uint32_t* d_stage_offsets = nullptr;   // staging buffer, grown on demand to the caller's capacity
-    uint16_t* d_stage_values = nullptr;
+    uint32_t* d_stage = nullptr;           // staging buffer, grown on demand to the caller's capacity
+    uint64_t* d_rec_base = nullptr;        // n_tiles: destination base per placement record
     uint64_t stage_capacity = 0;
     const float** d_ptrs = nullptr;        // 3 * n_tensors source pointers
     uint16_t** d_shards = nullptr;         // n_lists

@@ -85,8 +85,8 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
     cudaFree(L->d_rec);
     cudaFree(L->d_block_sum);
     cudaFree(L->d_cursor);
-    cudaFree(L->d_stage_offsets);
-    cudaFree(L->d_stage_values);
+    cudaFree(L->d_stage);
+    cudaFree(L->d_rec_base);
     cudaFree((void*)L->d_ptrs);
     cudaFree((void*)L->d_shards);
     cudaFree(L->d_shard_numel);
@@ -332,6 +332,12 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
     }
     dte_status st = DTE_OK;
     auto guard = [&](dte_status s) { if (st == DTE_OK) st = s; };
+    {   // destination base of every placement record, for the gather
+        std::vector<uint64_t> rec_base(n_ctas, 0);
+        for (const TileDesc& t : tiles) rec_base[t.tile] = t.dst_off;
+        for (size_t i = 0; i < packed.size(); i += kSub) rec_base[packed[i].tile] = kRecBasePacked | (uint64_t)(i / kSub);
+        guard(upload(&L->d_rec_base, rec_base));
+    }
     guard(upload(&L->d_tiles, tiles));
     guard(upload(&L->d_packed, packed));
     guard(upload(&L->d_segs, segs));
