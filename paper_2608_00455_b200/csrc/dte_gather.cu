@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(kScanThreads) gather_scan_kernel(const GatherP
 }
 
 // ---- 3. per block: local scan, list starts, gather ---------------------------------------------
-__global__ void __launch_bounds__(kGatherThreads) gather_move_kernel(const GatherParams p) {
+__global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const GatherParams p) {
     __shared__ uint32_t s_prefix[kRecsPerBlock + 1];   // exclusive prefix of counts within the block
     __shared__ uint64_t s_pos[kRecsPerBlock];          // staging position of each record
     __shared__ uint32_t s_warp[kGatherThreads / 32];
