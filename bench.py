@@ -33,9 +33,10 @@ from synth import configs, plans  # noqa: E402
 METRIC = "delta_extract_scanned_GBps"
 UNIT = "GB/s"
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per scanned element of the extract kernel, from the ncu capture summarised in
-# profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over a 2.3 GB case, per element).
-NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT = 12.125
+# Measured DRAM traffic of the extract kernel (ncu: dram__bytes_read.sum + dram__bytes_write.sum
+# of one launch over a one-layer case, and the elements that launch scanned), kept as data next
+# to the capture's summary; `roofline.traffic` scales it to the workload's element count.
+EXTRACT_TRAFFIC_JSON = os.path.join(ROOT, "profiles", "extract_kernel.qwen3-8b-one-layer.traffic.json")
 
 
 def log(*a):
@@ -224,20 +225,107 @@ def time_oracle_threads(wl, st, chosen, threads):
     return dt, scanned, sum(changed), len(jobs)
 
 
-def read_ceiling(dte, device, nbytes=4 << 30, reps=10):
+def extract_traffic(n_elements):
+    """DRAM bytes one extract call moves for `n_elements` scanned elements, scaled from the
+    committed ncu capture (traffic grows in proportion to the elements scanned)."""
+    try:
+        with open(EXTRACT_TRAFFIC_JSON) as f:
+            t = json.load(f)
+        per_el = (float(t["dram_bytes_read"]) + float(t["dram_bytes_write"])) / float(t["elements_scanned"])
+        return per_el * n_elements, {"bytes_per_element": per_el, "capture": os.path.basename(EXTRACT_TRAFFIC_JSON),
+                                     "scaled_from_elements": int(t["elements_scanned"])}
+    except Exception as e:      # no capture committed: say so instead of inventing a number
+        return None, {"error": f"{type(e).__name__}: {e}"}
+
+
+def time_leg(dte, wl, device, steps, warmup, peak, capacity_frac=0.03, with_clocks=True):
+    """One more workload through the same timed loop as the headline: resident state, `warmup`
+    untimed steps, `steps` timed steps of extract + apply (CUDA events per step), L2 flushed
+    between steps when the state could sit in it.  Returns the leg's numbers; frees its memory."""
+    plan = wl.plan
+    st, shards = materialize_resident(wl, device, dte)
+    lay = dte.Layout.from_plan(plan, device.index or 0)
+    N = lay.num_elements
+    delta = lay.new_delta(int(N * capacity_frac) + 1024)
+    tabs = lay.source_tables(st.theta, st.m, st.v)
+    shard_tab = lay.shard_table(shards)
+    hp = wl.hp.as_args()
+    stream = torch.cuda.current_stream()
+    dte.dte_extract_delta(lay, tabs, *hp, delta)
+    torch.cuda.synchronize()
+    if delta.status_bits() & dte.DTE_DEV_OVERFLOW:       # dense sweep points: size discovery, then grow
+        delta = lay.new_delta(delta.total() + 1024)
+        dte.dte_extract_delta(lay, tabs, *hp, delta)
+        torch.cuda.synchronize()
+    if delta.status_bits():
+        return {"workload": wl.name, "error": f"device status bits {delta.status_bits()}"}
+    M = delta.total()
+    flush = torch.empty(1 << 28, dtype=torch.uint8, device=device) if 12 * N < 2e9 else None
+
+    def step(ev=None):
+        if ev: ev[0].record(stream)
+        dte.dte_extract_delta(lay, tabs, *hp, delta)
+        if ev: ev[1].record(stream)
+        dte.dte_apply(lay, delta, shard_tab)
+        if ev: ev[2].record(stream)
+
+    for _ in range(max(warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    sampler = ClockSampler(device.index or 0)
+    if with_clocks:
+        sampler.start()
+        time.sleep(0.25)
+    w0 = time.time()
+    for i in range(steps):
+        if flush is not None:
+            flush.zero_()
+        step(evs[i])
+    torch.cuda.synchronize()
+    w1 = time.time()
+    clocks = sampler.stop(w0, w1) if with_clocks else None
+    ext = [e[0].elapsed_time(e[1]) for e in evs]
+    app = [e[1].elapsed_time(e[2]) for e in evs]
+    ext_avg, app_avg = sum(ext) / len(ext), sum(app) / len(app)
+    gbps = (12.0 * N + 6.0 * M) / (ext_avg * 1e-3) / 1e9
+    out = {"workload": wl.name, "elements_scanned": N, "changed": M, "changed_frac": M / N,
+           "lists": lay.num_lists, "operations": len(plan.ops), "steps": steps,
+           "hyper": {"step": wl.hp.step, "lr": wl.hp.lr, "wd": wl.hp.wd},
+           "extract_ms": ext_avg, "extract_ms_min": min(ext), "extract_GBps": gbps, "frac_of_peak": gbps / peak,
+           "apply_ms": app_avg, "apply_Mchanged_per_s": M / (app_avg * 1e-3) / 1e6 if M else None,
+           "l2": "inputs larger than L2" if flush is None else "256 MB written between timed steps",
+           "gpu_launches": (lay.last_launch()["kernels"] + 1) * steps, "launch": lay.last_launch(), "clocks": clocks,
+           **{k: v for k, v in wl.notes.items() if k in ("cold_experts", "sigma_g")}}
+    del st, shards, delta, lay, tabs, shard_tab, flush
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return out
+
+
+def density_sweep_points():
+    """(lr, step, wd, sigma_g) of the density / edge configuration that the benchmark times: the
+    five learning rates at t = 100, wd = 0.01, and the two dense points at lr = 1e-4."""
+    return [(lr, 100, 0.01, 1e-3) for lr in (1e-8, 1e-7, 1e-6, 1e-5, 1e-4)] + [(1e-4, 100, 0.01, 3e-3),
+                                                                                (1e-4, 100, 0.01, 1e-2)]
+
+
+def read_ceiling(device, nbytes=4 << 30, reps=10):
     """Read-only streaming bandwidth: one launch over a 4 GiB buffer of its own (CUDA events)."""
+    from paper_2608_00455_b200 import probes
     buf = torch.empty(nbytes, dtype=torch.uint8, device=device)
     buf.random_(0, 256)
     out = torch.zeros(1, dtype=torch.int64, device=device)
     stream = torch.cuda.current_stream()
     for _ in range(3):
-        dte.dte_read_bandwidth_probe(buf, out)
+        probes.read_bandwidth(buf, out)
     torch.cuda.synchronize()
     ms = []
     for _ in range(reps):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record(stream)
-        dte.dte_read_bandwidth_probe(buf, out)
+        probes.read_bandwidth(buf, out)
         e1.record(stream)
         torch.cuda.synchronize()
         ms.append(e0.elapsed_time(e1))
@@ -381,6 +469,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-codec", action="store_true", help="skip the storage-mediated path's legs")
+    ap.add_argument("--no-extra-workloads", action="store_true",
+                    help="skip the config 4 / config 1 / density-sweep legs that follow the headline workload")
     args = ap.parse_args()
 
     rank = int(os.environ.get("RANK", "0"))
@@ -481,7 +571,9 @@ def main():
         total_ms = sum(e[0].elapsed_time(e[2]) for e in evs)
     ext_ms = [e[0].elapsed_time(e[1]) for e in evs]
     app_ms = [e[1].elapsed_time(e[2]) for e in evs]
-    launches = (lay.last_launch()["kernels"] + 1) * args.steps     # extract call + apply, per step
+    n_lists = lay.num_lists
+    launch_info = lay.last_launch()
+    launches = (launch_info["kernels"] + 1) * args.steps     # extract call + apply, per step
     bytes_per_step = 12.0 * N + 6.0 * M
     total_ms, bytes_all = aggregate_over_ranks(total_ms, bytes_per_step, dist, device)
     ms_per_step = total_ms / args.steps
@@ -490,14 +582,12 @@ def main():
     app_avg = sum(app_ms) / len(app_ms)
     peak, peak_kind = measured_peak()
     achieved = bytes_per_step / (ext_avg * 1e-3) / 1e9
-    traffic = None
-    if NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT is not None:
-        traffic = NCU_EXTRACT_DRAM_BYTES_PER_ELEMENT * N
+    traffic, traffic_src = extract_traffic(N)
 
     # ---- practical ceiling for a read-only kernel: plain streaming reads of the same tensors --------
     ceiling = None
     if rank == 0:
-        ceiling = read_ceiling(dte, device)
+        ceiling = read_ceiling(device)
         log(f"[bench] read-only streaming ceiling: {ceiling}")
 
     # ---- storage path: chunk codec on the step's lists (outside the timed step) ------------------
@@ -539,13 +629,34 @@ def main():
                             "seconds": dt_k, "elements_per_s": scanned_k / dt_k,
                             "sample": "the same tensors, split over the threads largest first"}
 
+    # ---- the other quoted workloads, one after the other on the freed GPU -------------------------
+    extra = {}
+    if rank == 0 and world == 1 and args.workload == "full" and not args.no_extra_workloads:
+        import gc
+        del st, shards, delta, tabs, shard_tab, lay
+        gc.collect()
+        torch.cuda.empty_cache()
+        legs = max(10, min(args.steps, 30))
+        t0 = time.time()
+        extra["config4"] = time_leg(dte, configs.config4(device), device, legs, args.warmup, peak, 0.04)
+        log(f"[bench] config 4: {extra['config4']} ({time.time() - t0:.0f} s)")
+        extra["config1"] = time_leg(dte, configs.config1(), device, 50, args.warmup, peak)
+        log(f"[bench] config 1: {extra['config1']}")
+        sweep = []
+        for (lr, step_t, wd, sg) in density_sweep_points():
+            r = time_leg(dte, configs.config5(lr, step_t, wd, sg), device, 20, args.warmup, peak, 0.03, with_clocks=False)
+            r["sigma_g"] = sg
+            sweep.append(r)
+            log(f"[bench] sweep lr={lr:g} sigma_g={sg:g}: rho={r.get('changed_frac')} extract {r.get('extract_GBps')} GB/s")
+        extra["density_sweep"] = sweep
+
     if rank == 0:
         out = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": wl.name, "elements_scanned": N, "changed": M, "changed_frac": M / N,
-                       "lists": lay.num_lists, "l2": "inputs larger than L2 (no flush needed)" if flush is None else "256 MB written between timed steps to flush L2",
+                       "lists": n_lists, "l2": "inputs larger than L2 (no flush needed)" if flush is None else "256 MB written between timed steps to flush L2",
                        "hyper": {"step": wl.hp.step, "lr": wl.hp.lr, "wd": wl.hp.wd}, **wl.notes},
             "extract": {"ms": ext_avg, "ms_min": min(ext_ms), "GBps": achieved, "elements_per_s": N / (ext_avg * 1e-3),
                         "frac_of_8TBps": achieved / 8000.0},
@@ -555,13 +666,14 @@ def main():
                       "GBps_sector_traffic": 70.0 * M / (app_avg * 1e-3) / 1e9,
                       "frac_of_peak_sector_traffic": 70.0 * M / (app_avg * 1e-3) / 1e9 / peak},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                         "traffic": traffic, "peak_source": peak_kind, "kernel": "extract_kernel",
+                         "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_kind,
+                         "kernel": "extract call (extract_kernel launches + scan + gather)",
                          "read_only_ceiling": ceiling,
                          "frac_of_read_only_ceiling": achieved / ceiling["GBps"] if ceiling else None},
             "reconstruction_vs_truth": {"false_negatives": fn, "false_positives": fp, "variant": wl.variant},
             "storage_path": codec,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
-            "launch": lay.last_launch(),
+            "launch": launch_info, **extra,
         }
         print(json.dumps(out), flush=True)
     if dist:

@@ -117,7 +117,8 @@ typedef struct dte_layout dte_layout;
  *   counters : 4 x uint64 = { total changed, elements scanned, DTE_DEV_* bits, 0 }
  * If the total exceeds `capacity`, DTE_DEV_OVERFLOW is set, offsets / values hold nothing
  * usable, and list_ptr / counters[0] still hold the exact sizes, so the caller can grow
- * the buffers and call again (the paper's "size discovery before data movement"). */
+ * the buffers and call again (Section 3: sizes are learnt in a step of their own, before
+ * any payload moves). */
 typedef struct dte_delta {
     uint32_t* offsets;
     uint16_t* values;
@@ -238,18 +239,21 @@ DTE_API dte_status dte_apply_canonical(const dte_layout* layout, const dte_delta
 /* Section 4.3, round 1 of the two-round transfer: the entry count c_o = |I_o| of every
  * operation of the plan, in plan order, zero-length operations included (both peers keep
  * the position of an empty operation, so the schedule stays aligned).  `counts`: DEVICE array
- * of dte_layout_num_ops(layout) uint64.  `delta` must be a complete extract result (no
- * overflow); entries of operation o are those of list dst_shard(o) whose offset lies in the
- * operation's destination range, a contiguous run of that list. */
+ * of dte_layout_num_ops(layout) uint64.  Entries of operation o are those of list dst_shard(o)
+ * whose offset lies in the operation's destination range, a contiguous run of that list.  Like
+ * dte_apply it may be enqueued right after the extract: if `delta` turns out incomplete (its
+ * counters carry DTE_DEV_OVERFLOW or DTE_DEV_CORRUPT, or its total exceeds its capacity) every
+ * count is written as zero, DTE_DEV_OVERFLOW is set and no entry is read. */
 DTE_API dte_status dte_op_counts(const dte_layout* layout, const dte_delta* delta, uint64_t* counts,
                                  void* cuda_stream);
 /* Number of operations the layout was created with. */
 DTE_API size_t dte_layout_num_ops(const dte_layout* layout);
 
 /* ---- Chunk codec of the storage-mediated path (Section 4.4) ---------------------------------
- * Across clusters the paper publishes the sparse changes as compressed payload chunks of
- * changed index-value pairs, every entry an int32 index and a BF16 value, and a manifest with
- * the payload locations, lengths and checksums; the destination verifies and applies them.
+ * Between clusters the changes travel through object storage (Section 4.4): what changed is
+ * written out in chunks, four bytes of index and two bytes of BF16 value per element, next to a
+ * manifest that says where each chunk lies, how long it is and what it must hash to; the
+ * destination checks the chunks before it applies them.
  * The paper prints no byte layout; this library's is:
  *   stream  : chunks back to back, each on a 16-byte boundary, lists in order, entries of a
  *             list in ascending order, at most `chunk_entries` entries of ONE list per chunk,
@@ -331,13 +335,6 @@ DTE_API dte_status dte_extract_delta_host(const dte_layout* layout, const float*
                                   void* workspace, uint64_t workspace_bytes, const dte_delta* out,
                                   uint32_t* offsets_h, uint16_t* values_h, uint64_t* list_ptr_h,
                                   uint64_t* counters_h, void* cuda_stream);
-
-/* Measurement aid, no counterpart in the paper: one read-only streaming pass over `bytes` bytes
- * of DEVICE memory at `src` (16-byte aligned; a trailing bytes % 16 is ignored), XOR-folding
- * what it reads into *xor_out (DEVICE, 8 bytes, not cleared).  Timed by the caller, it gives the
- * read bandwidth ceiling of `device` for a kernel that, like the extract, only reads. */
-DTE_API dte_status dte_read_bandwidth_probe(const void* src, uint64_t bytes, uint64_t* xor_out, int device,
-                                            void* cuda_stream);
 
 /* Static strings. */
 DTE_API const char* dte_status_string(dte_status s);

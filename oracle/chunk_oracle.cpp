@@ -3,10 +3,10 @@
 // THIS IS TEST INFRASTRUCTURE, NOT PRODUCT CODE (see dte_oracle.cpp): a plain sequential
 // writer and reader of the chunk stream, byte by byte, sharing nothing with the CUDA library.
 //
-// What the paper fixes (Section 4.4 and the evaluation's data-volume paragraph): only changed
-// index-value pairs are serialised, into payload chunks; every entry stores an int32 index and
-// a BF16 value; the manifest records payload locations, lengths and checksums.  The paper
-// prints no byte layout, so the layout below is this build's reading of it:
+// What the paper fixes (Section 4.4 and the evaluation's data-volume paragraph): nothing but
+// the changed elements is written out, in chunks, four bytes of index and two bytes of BF16
+// value per element, and a manifest says where each chunk lies, how long it is and what it must
+// hash to.  The paper prints no byte layout, so the layout below is this build's reading of it:
 //
 //   stream  = chunks back to back, each starting on a 16-byte boundary
 //   chunk   = 32-byte header + payload, covering at most C consecutive entries of ONE list

@@ -142,7 +142,7 @@ uint64_t oracle_changed_mask(const float* theta, const float* m, const float* v,
 // index in ascending order that changed, for each operation on that tensor in
 // plan order: unravel, test membership, ravel in receiver coordinates, append
 // (j, value) to the operation's receiver list.  Each list is then put in
-// ascending j (the "ordered sparse payload"); a repeated j within one list is
+// ascending j (Section 4.2.2: a payload keeps its entries in order); a repeated j within one list is
 // a plan error.  Lists are concatenated in shard order; empty lists keep
 // their slot (list_ptr[k] == list_ptr[k+1]).
 // `consts` holds 5 scalars per source tensor (n_tensors x 5): eta_t and lambda of Eq. 2 belong

@@ -27,7 +27,7 @@ SYMBOLS = [
     "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
     "dte_extract_delta_static", "dte_extract_delta_groups", "dte_layout_num_groups",
     "dte_op_counts", "dte_layout_num_ops", "dte_chunk_count_bound", "dte_chunk_bytes_bound",
-    "dte_pack_chunks", "dte_unpack_chunks", "dte_read_bandwidth_probe", "dte_apply_canonical",
+    "dte_pack_chunks", "dte_unpack_chunks", "dte_apply_canonical",
 ]
 
 
@@ -107,8 +107,6 @@ def lib() -> C.CDLL:
         L.dte_pack_chunks.restype = C.c_int
         L.dte_unpack_chunks.argtypes = [vp, vp, u64, vp, u64, vp, vp]
         L.dte_unpack_chunks.restype = C.c_int
-        L.dte_read_bandwidth_probe.argtypes = [vp, u64, vp, C.c_int, vp]
-        L.dte_read_bandwidth_probe.restype = C.c_int
         L.dte_apply_canonical.argtypes = [vp, vp, vp, vp]
         L.dte_apply_canonical.restype = C.c_int
         L.dte_apply.argtypes = [vp, vp, vp, vp]
@@ -404,13 +402,6 @@ def dte_unpack_chunks(layout: Layout, stream_bytes: torch.Tensor, directory: tor
     n = stream_bytes.numel() if nbytes is None else int(nbytes)
     _check(lib().dte_unpack_chunks(layout._h, stream_bytes.data_ptr(), n, directory.data_ptr(), int(n_chunks),
                                    C.byref(delta.struct), _stream_ptr(stream)))
-
-
-def dte_read_bandwidth_probe(tensor: torch.Tensor, xor_out: torch.Tensor, stream=None) -> None:
-    """Enqueue one read-only pass over `tensor` (measurement aid; see dte.h)."""
-    assert tensor.is_cuda and tensor.is_contiguous() and xor_out.is_cuda and xor_out.dtype == torch.int64
-    _check(lib().dte_read_bandwidth_probe(tensor.data_ptr(), tensor.numel() * tensor.element_size(),
-                                          xor_out.data_ptr(), tensor.device.index or 0, _stream_ptr(stream)))
 
 
 def dte_apply_canonical(layout: Layout, canonical: Delta, shard_table, stream=None) -> None:

@@ -1,5 +1,6 @@
 // C entry points that enqueue the kernels: the extract variants, dte_apply, dte_op_counts,
 // the chunk codec and the host-buffer variant dte_extract_delta_host.
+#include <atomic>
 #include <cmath>
 #include <cstring>
 #include <limits>
@@ -320,16 +321,8 @@ extern "C" dte_status dte_op_counts(const dte_layout* layout, const dte_delta* d
     if (s != DTE_OK) return s;
     if (layout->n_ops && !counts) return fail(DTE_ERR_INVALID_ARG, "counts is null");
     DeviceGuard g(layout->device);
-    return launch_op_counts(layout->d_op_ranges, layout->n_ops, delta->offsets, delta->list_ptr, counts,
+    return launch_op_counts(layout->d_op_ranges, layout->n_ops, *delta, layout->n_lists, counts,
                             (cudaStream_t)cuda_stream);
-}
-
-extern "C" dte_status dte_read_bandwidth_probe(const void* src, uint64_t bytes, uint64_t* xor_out, int device,
-                                               void* cuda_stream) {
-    if (!src || !xor_out) return fail(DTE_ERR_INVALID_ARG, "src / xor_out is null");
-    if ((uintptr_t)src & 15u) return fail(DTE_ERR_INVALID_ARG, "src must be 16-byte aligned");
-    DeviceGuard g(device);
-    return launch_read_probe(src, bytes, xor_out, device, (cudaStream_t)cuda_stream);
 }
 
 // ---- chunk codec -------------------------------------------------------------------------
@@ -479,19 +472,22 @@ static_assert(kStaticBlockSumOff % 8 == 0 && kStaticStageOff % 8 == 0, "sub-buff
 // address: the address each device gave the array comes from cudaGetSymbolAddress below.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
-unsigned char* g_static_addr[kMaxDevices] = {nullptr};
+// One slot per device ordinal; atomic because two host threads may make their first call on a
+// device at the same time (both then ask the runtime and store the same address).
+std::atomic<unsigned char*> g_static_addr[kMaxDevices];
 
 // First use on a device (that device current): ask the runtime where the array lives there.
 dte_status static_scratch_address(int device, unsigned char** out) {
     if (device < 0 || device >= kMaxDevices) return fail(DTE_ERR_INVALID_ARG, "device ordinal out of range");
-    if (!g_static_addr[device]) {
+    unsigned char* addr = g_static_addr[device].load(std::memory_order_acquire);
+    if (!addr) {
         void* ptr = nullptr;
         DTE_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
         if (!ptr) return fail(DTE_ERR_CUDA, "cudaGetSymbolAddress returned a null address");
-        g_static_addr[device] = static_cast<unsigned char*>(ptr);
+        addr = static_cast<unsigned char*>(ptr);
+        g_static_addr[device].store(addr, std::memory_order_release);
     }
-    *out = g_static_addr[device];
+    *out = addr;
     return DTE_OK;
 }
 

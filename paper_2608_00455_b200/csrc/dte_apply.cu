@@ -161,10 +161,20 @@ dte_status launch_apply_canonical(const CanonParams& p, int device, cudaStream_t
 
 // ---- per-operation counts (Section 4.3, round 1) ---------------------------------------------
 // c_o = number of entries of the operation's list whose offset lies in the operation's
-// destination range: two binary searches in the (ascending) list.
+// destination range: two binary searches in the (ascending) list.  An incomplete delta (its
+// extract overflowed, or it was read from a damaged chunk stream) has list boundaries beyond the
+// entry arrays: it gets zero counts and the overflow bit, and no entry is read.
 __global__ void op_counts_kernel(const OpRange* __restrict__ ranges, uint32_t n_ops,
                                  const uint32_t* __restrict__ offsets, const uint64_t* __restrict__ list_ptr,
+                                 uint32_t n_lists, uint64_t capacity, uint64_t* counters,
                                  uint64_t* __restrict__ counts) {
+    const uint64_t dev_bits = counters[2];
+    if (list_ptr[n_lists] > capacity || (dev_bits & (DTE_DEV_OVERFLOW | DTE_DEV_CORRUPT))) {
+        for (uint32_t o = blockIdx.x * blockDim.x + threadIdx.x; o < n_ops; o += gridDim.x * blockDim.x) counts[o] = 0;
+        if (blockIdx.x == 0 && threadIdx.x == 0 && !(dev_bits & DTE_DEV_CORRUPT))
+            atomicOr((unsigned long long*)(counters + 2), (unsigned long long)DTE_DEV_OVERFLOW);
+        return;
+    }
     for (uint32_t o = blockIdx.x * blockDim.x + threadIdx.x; o < n_ops; o += gridDim.x * blockDim.x) {
         const OpRange r = ranges[o];
         const uint64_t a = list_ptr[r.list], b = list_ptr[r.list + 1];
@@ -183,11 +193,12 @@ __global__ void op_counts_kernel(const OpRange* __restrict__ ranges, uint32_t n_
     }
 }
 
-dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const uint32_t* offsets,
-                            const uint64_t* list_ptr, uint64_t* counts, cudaStream_t st) {
+dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const dte_delta& d, uint32_t n_lists,
+                            uint64_t* counts, cudaStream_t st) {
     if (n_ops == 0) return DTE_OK;
     const int threads = 128, blocks = (int)std::min<uint32_t>((n_ops + threads - 1) / threads, 4096u);
-    op_counts_kernel<<<blocks, threads, 0, st>>>(ranges, n_ops, offsets, list_ptr, counts);
+    op_counts_kernel<<<blocks, threads, 0, st>>>(ranges, n_ops, d.offsets, d.list_ptr, n_lists, d.capacity,
+                                                 d.counters, counts);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }

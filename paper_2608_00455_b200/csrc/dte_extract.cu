@@ -17,21 +17,13 @@
 // Build flags that matter for bit-exactness: -fmad=false -ftz=false -prec-div=true
 // -prec-sqrt=true.  The exact path additionally spells every operation as a
 // round-to-nearest intrinsic so that no flag can silently change it.
+#include <atomic>
+
 #include "dte_internal.cuh"
 
 namespace dte {
 
-#ifndef DTE_MIN_CTAS
-#define DTE_MIN_CTAS 4
-#endif
-
-#ifdef DTE_STATS
-// Development-only counters (never compiled into the shipped library).
-__device__ unsigned long long g_stats[8];
-#define DTE_STAT(i, x) do { if (lane == 0) atomicAdd(&g_stats[i], (unsigned long long)(x)); } while (0)
-#else
-#define DTE_STAT(i, x) do { } while (0)
-#endif
+constexpr int kMinCtasPerSm = 4;
 
 // ---- exact arithmetic ------------------------------------------------------------
 
@@ -317,7 +309,7 @@ __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint3
 
 // GROUPS: the constants come from the tile's parameter group instead of the kernel parameters.
 template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED>
-__global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const ExtractParams p) {
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const ExtractParams p) {
     // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
     // (dynamic shared memory: kWarps * kWarpTile words, may exceed the 48 KB static limit)
     // The two launches of one extract (packed tiles, then regular tiles) are independent: let the
@@ -358,8 +350,6 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
         else
             qn = phase_a<DIV_BC1, DIV_DECAY, false>(cur, lane, queue, sc, lr);
         __syncwarp();
-        DTE_STAT(0, qn);
-        DTE_STAT(2, (qn + 31) / 32);
 
         // ---- phase B: exact evaluation of the queue, 32 entries per round; the changed
         //      entries are compacted to the front of the queue as (index | value << 16) -----
@@ -425,6 +415,11 @@ __global__ void __launch_bounds__(kThreads, DTE_MIN_CTAS) extract_kernel(const E
             if (pos + q < p.stage_capacity)               // beyond it the call overflows anyway
                 p.stage[pos + q] = queue[q] + rel;
     }
+    // The launch of the regular tiles may have begun before the launch of the packed tiles ended.
+    // What follows in the stream (the gather) is ordered after THIS grid only, so this grid must
+    // not complete before the one it overlapped: wait for it here, where nothing is left to do.
+    // A no-op for a launch that did not overlap anything.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 constexpr size_t kQueueBytes = (size_t)kWarps * kWarpTile * sizeof(uint32_t);
@@ -433,13 +428,16 @@ constexpr size_t kQueueBytes = (size_t)kWarps * kWarpTile * sizeof(uint32_t);
 // not depend on that kernel's results).
 template <bool A, bool B, bool G, bool P>
 static dte_status launch_t(const ExtractParams& p, bool overlap, cudaStream_t st) {
-    static bool configured[64] = {false};     // per device: allow more than 48 KB of dynamic shared memory
+    // per device, once: allow more than 48 KB of dynamic shared memory.  Host threads may race
+    // here (two layouts on two threads); setting the attribute twice is harmless, so an atomic
+    // flag per device is enough.
+    static std::atomic<bool> configured[kMaxDevices];
     int dev = 0;
     DTE_CUDA(cudaGetDevice(&dev));
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
         DTE_CUDA(cudaFuncSetAttribute(extract_kernel<A, B, G, P>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                       (int)kQueueBytes));
-        configured[dev] = true;
+        if (dev >= 0 && dev < kMaxDevices) configured[dev].store(true, std::memory_order_release);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(p.n_tiles);
@@ -459,13 +457,6 @@ template <bool A, bool B, bool G>
 static dte_status launch_p(const ExtractParams& p, bool packed, bool overlap, cudaStream_t st) {
     return packed ? launch_t<A, B, G, true>(p, overlap, st) : launch_t<A, B, G, false>(p, overlap, st);
 }
-
-#ifdef DTE_STATS
-extern "C" __attribute__((visibility("default"))) void dte_debug_stats(unsigned long long* out8, int reset) {
-    cudaMemcpyFromSymbol(out8, g_stats, sizeof(g_stats));
-    if (reset) { unsigned long long z[8] = {0}; cudaMemcpyToSymbol(g_stats, z, sizeof(z)); }
-}
-#endif
 
 // div_bc1 / div_decay: whether any group in the call has a divisor different from 1.0f.
 // One launch covers p.n_tiles tiles of one kind (p.tiles = their descriptors).

@@ -36,6 +36,7 @@ constexpr int kSub = 8;                                // warp-tiles per tile
 constexpr int kTile = kSub * kWarpTile;                // 9216 elements
 static_assert(kTile < 16384, "a tile's changed count must fit kRecCountBits");
 constexpr uint32_t kNone = 0xFFFFFFFFu;
+constexpr int kMaxDevices = 64;                        // device ordinals with per-device host state
 
 constexpr uint32_t kLenMask = 0xFFFFu;
 constexpr uint32_t kFlagScalar = 1u << 18;             // not 16-byte alignable: scalar loads
@@ -214,9 +215,8 @@ dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 dte_status launch_apply_canonical(const CanonParams& p, int device, cudaStream_t st);
 dte_status launch_pack_chunks(const PackParams& p, int device, cudaStream_t st);
 dte_status launch_unpack_chunks(const UnpackParams& p, int device, cudaStream_t st);
-dte_status launch_read_probe(const void* src, uint64_t bytes, uint64_t* out, int device, cudaStream_t st);
-dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const uint32_t* offsets,
-                            const uint64_t* list_ptr, uint64_t* counts, cudaStream_t st);
+dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const dte_delta& d, uint32_t n_lists,
+                            uint64_t* counts, cudaStream_t st);
 
 }  // namespace dte
 

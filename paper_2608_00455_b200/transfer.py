@@ -75,7 +75,7 @@ class TwoRoundTransfer:
         # zero-count calls).  Off by default: after round 1 both sides know the total, so both
         # skip the same calls and the schedule stays aligned either way.
         self.zero_count_calls = bool(zero_count_calls)
-        self.check_counts = True   # sender-side consistency check before round 2 (one small host read per route)
+        self.check_counts = True   # sender-side consistency check before round 1 (one small host read per route)
         self.routes: Dict[Tuple[int, int], Route] = {}
         op_receiver = self.shard_receivers[self.op_dst_shard] if self.op_dst_shard.size else self.op_dst_shard
         # operations of each sender in plan order: the order of a sender's own plan and of its counts
@@ -142,10 +142,31 @@ class TwoRoundTransfer:
             list_ptr = np.asarray(list_ptr, dtype=np.uint64)
         got: Dict[int, Received] = {}
 
+        # Before anything is sent: the counts a sender is about to announce must add up to the lists
+        # it holds.  After round 1 the receivers post their receives for the announced totals; a
+        # sender that found a mismatch only then, and left, would keep them waiting for bytes that
+        # never come - and one that left before round 1 would keep them waiting for the counts.  So
+        # a sender whose lists are inconsistent stays in the schedule: it announces -1 for every
+        # operation of every route (round 1 keeps its shape), sends no payload, and raises once both
+        # rounds are over; a receiver that reads -1 posts no receive for that route and raises at
+        # the same point.  Every rank returns or raises; none blocks.
+        payloads, problems = {}, []
+        for rt in out_routes:
+            payloads[rt.receiver] = self._payload(rt, list_ptr, offsets, values)
+            if self.check_counts:
+                announced = int(op_counts[torch.as_tensor(rt.local_ops, device=op_counts.device)].sum().item())
+                held = payloads[rt.receiver][0].numel()
+                if announced != held:
+                    problems.append(f"route {rt.sender}->{rt.receiver}: counts announce {announced} entries, "
+                                    f"lists hold {held}")
+        poisoned = bool(problems)
+
         # round 1: c_o for every operation of every pair, plan order, zeros included
         p2p, keep, count_bufs = [], [], {}
         for rt in out_routes:
             counts = op_counts[torch.as_tensor(rt.local_ops, device=op_counts.device)].to(torch.int64).contiguous()
+            if poisoned:
+                counts = torch.full_like(counts, -1)
             peer = self.rank_of_receiver[rt.receiver]
             if peer == rank:
                 count_bufs[rt.sender] = counts
@@ -163,6 +184,9 @@ class TwoRoundTransfer:
         p2p, keep = [], []
         for rt in in_routes:
             counts = count_bufs[rt.sender].cpu().numpy().astype(np.int64)
+            if counts.size and counts.min() < 0:
+                problems.append(f"sender {rt.sender} reported inconsistent lists; nothing received from it")
+                continue
             total = int(counts.sum())
             rec = Received(rt.sender, counts, self._list_ptr(rt, counts),
                            torch.empty(total, dtype=torch.int32, device=device),
@@ -175,13 +199,10 @@ class TwoRoundTransfer:
 
         # round 2: I_o and V_o, same order
         for rt in out_routes:
-            off, val = self._payload(rt, list_ptr, offsets, values)
+            if poisoned:
+                break
+            off, val = payloads[rt.receiver]
             peer = self.rank_of_receiver[rt.receiver]
-            if self.check_counts:
-                announced = int(op_counts[torch.as_tensor(rt.local_ops, device=op_counts.device)].sum().item())
-                if announced != off.numel():      # a mismatch would leave the peer waiting for bytes that never come
-                    raise RuntimeError(f"route {rt.sender}->{rt.receiver}: counts announce {announced} entries, "
-                                       f"lists hold {off.numel()}")
             if peer == rank:
                 got[rt.sender].offsets.copy_(off)
                 got[rt.sender].values.copy_(val)
@@ -191,4 +212,6 @@ class TwoRoundTransfer:
                 p2p.append(dist.P2POp(dist.isend, off, peer, self.group))
                 p2p.append(dist.P2POp(dist.isend, val, peer, self.group))
         self._run(p2p)
+        if problems:
+            raise RuntimeError("; ".join(problems))
         return got

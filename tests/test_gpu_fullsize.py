@@ -1,6 +1,8 @@
 """Full-size parity in the launch configuration bench.py times: the whole Qwen3-8B-shaped state
-(config 3, 98 GB) and the Qwen3-30B-A3B slice (config 4, 90 GB) resident on one GPU.  The oracle
-checks complete lists of sampled tensors; properties that hold at any size cover the rest."""
+(config 3, 98 GB), the Qwen3-30B-A3B slice (config 4, 90 GB) and the density / edge grid on one
+full-dimension layer (config 5), resident on one GPU.  The oracle checks EVERY list and every
+receiver tensor after apply: the state is streamed to the host group by group and spread over the
+host threads (see gpu_util.full_oracle_parity); nothing is sampled."""
 import gc
 
 import numpy as np
@@ -11,7 +13,7 @@ import bench
 import oracle
 import paper_2608_00455_b200 as dte
 from synth import configs
-from gpu_util import assert_lists_equal
+from gpu_util import assert_lists_equal, full_oracle_parity
 
 pytestmark = pytest.mark.gpu
 
@@ -95,9 +97,19 @@ def test_config3_full_qwen3_8b_state():
     torch.cuda.synchronize()
     lp = _global_properties(plan, lay, d)
     assert 0.01 < lp[-1] / N < 0.02
-    # all 11 tensors of layer 17 (row- and column-split, replicated norms) and embed_tokens
+    # every one of the 580 lists (lm_head, the last tensor with the highest tile indices and
+    # source offsets, and all 36 layers included) and every receiver tensor after apply
+    after = [s.clone() for s in shards]
+    dte.dte_apply(lay, d, lay.shard_table(after))
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    n_lists, n_entries = full_oracle_parity(wl, st, d, shards, after)
+    assert n_lists == 580 and n_entries == int(lp[-1])
+    del after
+    _free()
+    # the storage-path leg below also needs complete oracle lists of a few tensors
     names = plan.tensor_names
-    sample = [p for p, n in enumerate(names) if n.startswith("layers.17.")] + [names.index("embed_tokens")]
+    sample = [p for p, n in enumerate(names) if n.startswith("layers.35.")] + [names.index("lm_head")]
     lists, want = _sampled_lists_equal(wl, st, d, sample)
     assert len(lists) == 18
     assert _apply_end_state(plan, st, lay, d, shards, lists) <= 8
@@ -167,15 +179,61 @@ def test_config4_qwen3_30b_a3b_slice():
     torch.cuda.synchronize()
     _global_properties(plan, lay, d)
     assert wl.notes["cold_experts"] > 0
-    # layer 5 completely: attention, router, norms and all 128 experts (cold ones included)
-    sample = [p for p, n in enumerate(plan.tensor_names) if n.startswith("layers.5.")]
-    lists, want = _sampled_lists_equal(wl, st, d, sample)
-    assert len(lists) == 36
+    # every one of the 432 lists (all 12 layers: attention, router, norms, 128 experts each, cold
+    # ones included) and every receiver tensor after apply
+    after = [s.clone() for s in shards]
+    dte.dte_apply(lay, d, lay.shard_table(after))
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    n_lists, n_entries = full_oracle_parity(wl, st, d, shards, after)
+    assert n_lists == 432 and n_entries == d.total()
     # cold experts (zero state) contribute nothing
-    cold = [p for p in sample if "experts" in plan.tensor_names[p] and wl.specs[p].scale == 0.0]
+    cold = [p for p, n in enumerate(plan.tensor_names) if "experts" in n and wl.specs[p].scale == 0.0]
     assert cold
     for p in cold[:6]:
         assert float(st.m[p].abs().max()) == 0.0 and float(st.v[p].abs().max()) == 0.0
-    assert _apply_end_state(plan, st, lay, d, shards, lists) <= 8
-    del st, shards, d, lay
+    stale = sum(int((a != b).sum().item()) for a, b in zip(after, _expected(plan, st)))
+    assert stale <= 16
+    del st, shards, after, d, lay
+    _free()
+
+
+def _expected(plan, st):
+    """Remapped BF16(theta_t) of every receiver tensor, one at a time (generator)."""
+    ops_by_shard = {}
+    for o in plan.ops:
+        ops_by_shard.setdefault(o[1], []).append(o)
+    for k, n in enumerate(plan.shard_numels):
+        exp = torch.zeros(n, dtype=torch.int16, device="cuda")
+        for (src, _, a0, a1, e0, e1, base, ld, r0, r1) in ops_by_shard.get(k, []):
+            s2 = st.theta[src].reshape(plan.tensor_shapes[src])[a0:a0 + e0, a1:a1 + e1]
+            exp.as_strided((e0, e1), (ld, 1), base + r0 * ld + r1).copy_(s2.to(torch.bfloat16).view(torch.int16))
+        yield exp
+
+
+@pytest.mark.parametrize("point", configs.config5_points(), ids=lambda p: f"lr{p[0]:g}-t{p[1]}-wd{p[2]:g}-sg{p[3]:g}")
+def test_config5_density_and_edge_grid_full_dimensions(point):
+    """The whole grid lr x t x wd (plus the sigma_g = 1e-2 point) on the full-dimension Qwen3-8B
+    layer with planted ties, zeros, extremes and subnormals: every list and every receiver tensor
+    against the oracle."""
+    _need(12)
+    lr, step, wd, sigma_g = point
+    wl = configs.config5(lr, step, wd, sigma_g)
+    plan = wl.plan
+    st = wl.materialize("cuda")
+    lay = dte.Layout.from_plan(plan, 0)
+    assert lay.num_elements == 192971776
+    d = lay.new_delta(lay.num_elements // 2 + 4096)
+    dte.dte_extract_delta(lay, lay.source_tables(st.theta, st.m, st.v), *wl.hp.as_args(), d)
+    torch.cuda.synchronize()
+    _global_properties(plan, lay, d)
+    from gpu_util import initial_shards
+    before = initial_shards(plan, st)
+    after = [s.clone() for s in before]
+    dte.dte_apply(lay, d, lay.shard_table(after))
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    n_lists, n_entries = full_oracle_parity(wl, st, d, before, after)
+    assert n_lists == 32 and n_entries == d.total()
+    del st, before, after, d, lay
     _free()

@@ -161,6 +161,32 @@ def test_capacity_overflow_reports_exact_sizes_and_apply_refuses():
     assert int(canary.sum().item()) == 16 * 0x5A5A
 
 
+def test_op_counts_right_after_an_overflowing_extract_reads_no_entry():
+    # dte_op_counts is meant to be enqueued straight after the extract; when that extract
+    # overflowed, list_ptr holds the exact sizes, which point beyond the entry arrays
+    wl = configs.config2(dims=configs.SMALL_DENSE, hp=Hyper(step=100, lr=1e-4, wd=0.01))
+    st = wl.materialize("cuda")
+    lay = dte.Layout.from_plan(wl.plan, 0)
+    pool = torch.full((4096 + 64,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    d = lay.new_delta(64)
+    # entry arrays carved out of a canary pool: nothing past the 64 entries may be touched
+    d.offsets = pool[2048:2048 + 64]
+    d.struct.offsets = d.offsets.data_ptr()
+    tabs = lay.source_tables(st.theta, st.m, st.v)
+    dte.dte_extract_delta(lay, tabs, *wl.hp.as_args(), d)
+    counts = dte.dte_op_counts(lay, d)
+    torch.cuda.synchronize()
+    assert d.status_bits() & dte.DTE_DEV_OVERFLOW and d.total() > 64
+    assert int(counts.abs().sum().item()) == 0
+    assert bool((pool[:2048] == 0x5A5A5A5A).all()) and bool((pool[2048 + 64:] == 0x5A5A5A5A).all())
+    # a complete delta on the same layout gives the real counts again
+    d2 = lay.new_delta(d.total())
+    dte.dte_extract_delta(lay, tabs, *wl.hp.as_args(), d2)
+    counts = dte.dte_op_counts(lay, d2)
+    torch.cuda.synchronize()
+    assert d2.status_bits() == 0 and int(counts.sum().item()) == d2.total()
+
+
 def test_apply_flags_out_of_range_offsets():
     plan = plans.single_matrix_plan(64, 64, 2)
     wl = configs.Workload("b", plan, Hyper(step=1, lr=0.5, wd=0.0), configs._specs(plan, Spec(sigma_g=1.0)), 3)

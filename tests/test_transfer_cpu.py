@@ -25,6 +25,10 @@ def _lists_of(plan, st, hp, oracle):
                           with_op_counts=True)
 
 
+def scenario_bad_rank(scenario):
+    return scenario[6] if len(scenario) > 6 else None
+
+
 def _worker(rank, world, port, out, scenario):
     os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
     sys.path.insert(0, ROOT)
@@ -35,7 +39,7 @@ def _worker(rank, world, port, out, scenario):
         from synth import configs, plans
         from synth.tensors import Hyper
 
-        tp_send, tp_recv, rank_of_sender, rank_of_receiver, lr, zero_calls = scenario
+        tp_send, tp_recv, rank_of_sender, rank_of_receiver, lr, zero_calls = scenario[:6]
         plan = plans.mcore_dense_plan(1, tp_send, tp_recv, True, configs.SMALL_DENSE)
         owners = plans.tensor_senders(plan, tp_send)
         hp = Hyper(step=200, lr=lr, wd=0.05)
@@ -53,6 +57,17 @@ def _worker(rank, world, port, out, scenario):
             args = dict(list_ptr=lp, offsets=torch.from_numpy(off.view(np.int32).copy()),
                         values=torch.from_numpy(val.view(np.int16).copy()),
                         op_counts=torch.from_numpy(counts.astype(np.int64)))
+        if scenario_bad_rank(scenario) == rank:     # this sender announces one entry too many
+            args["op_counts"] = args["op_counts"].clone()
+            args["op_counts"][0] += 1
+        if scenario_bad_rank(scenario) is not None:
+            try:
+                xfer.exchange(rank, sender, receiver, **args)
+                out.put({"rank": rank, "raised": None})
+            except RuntimeError as e:
+                out.put({"rank": rank, "raised": str(e)})
+            dist.barrier()
+            return
         got = xfer.exchange(rank, sender, receiver, **args)
         report = {"rank": rank, "senders": sorted(got), "entries": {s: int(g.offsets.numel()) for s, g in got.items()}}
         if receiver is not None:
@@ -125,6 +140,16 @@ def test_nothing_changed_keeps_the_schedule_aligned(zero_calls):
         assert r["zero_count_ops"] > 0 and sum(r["entries"].values()) == 0
 
 
+def test_inconsistent_counts_on_one_sender_block_no_rank():
+    # rank 1's counts do not add up to its lists: it stays in the schedule, announces the failure in
+    # round 1 and raises after round 2; its peers raise too (nothing usable arrived from it), and
+    # every process reaches the final barrier - a rank that left early would hang the others
+    res = _run(3, (2, 2, [0, 1], [1, 2], 2e-6, False, 1), 37000)
+    assert "counts announce" in res[1]["raised"]
+    assert "sender 1 reported inconsistent lists" in res[2]["raised"]
+    assert res[0]["raised"] is None          # a sender with consistent lists is not affected
+
+
 def test_schedule_is_static_and_symmetric():
     from paper_2608_00455_b200.transfer import TwoRoundTransfer
     from synth import configs, plans
@@ -142,7 +167,7 @@ def test_schedule_is_static_and_symmetric():
 
 
 def test_counts_that_disagree_with_the_lists_stop_the_sender():
-    # announced counts and payload length must match before round 2, or a peer would wait forever
+    # announced counts and payload length must match before anything is sent
     from paper_2608_00455_b200.transfer import TwoRoundTransfer
     x = TwoRoundTransfer([0, 0], [0, 1], [0, 0], [0], [0])            # one sender, one receiver, same rank
     lp = np.array([0, 3, 5], np.uint64)
@@ -150,5 +175,6 @@ def test_counts_that_disagree_with_the_lists_stop_the_sender():
     val = torch.arange(5, dtype=torch.int16)
     got = x.exchange(0, 0, 0, lp, off, val, torch.tensor([3, 2]))
     assert got[0].list_ptr.tolist() == [0, 3, 5] and torch.equal(got[0].offsets, off)
-    with pytest.raises(RuntimeError):
+    # the local route reports both sides of the failure
+    with pytest.raises(RuntimeError, match="counts announce 4 entries, lists hold 5; sender 0 reported"):
         x.exchange(0, 0, 0, lp, off, val, torch.tensor([3, 1]))

@@ -15,6 +15,7 @@ import torch
 import paper_2608_00455_b200 as dte
 from synth import configs
 from synth.tensors import Hyper
+from gpu_util import assert_lists_equal, oracle_extract
 
 pytestmark = pytest.mark.gpu
 
@@ -55,6 +56,42 @@ def test_static_scratch_extract_matches_the_allocating_one_twice_in_a_row():
     ref2, got2 = _both(lay, st2, wl2.hp, cap)
     _assert_same(ref2, got2)
     assert ref2.total() < ref1.total()
+    # and not only equal to the other entry point: equal to the oracle, both times
+    assert_lists_equal(got1.to_host(), oracle_extract(wl1.plan, st1, wl1.hp), wl1.plan)
+    assert_lists_equal(got2.to_host(), oracle_extract(wl2.plan, st2, wl2.hp), wl2.plan)
+
+
+def test_static_scratch_extract_overflow_and_empty_plan():
+    # capacity below the number of changed elements: exact sizes reported, nothing written past
+    # the caller's arrays (they sit inside a canary pool), same answer as the allocating call
+    wl = configs.config2(dims=configs.SMALL_DENSE, hp=Hyper(step=1, lr=1e-4, wd=0.1), seed=13)
+    lay = dte.Layout.from_plan(wl.plan, 0)
+    st = wl.materialize("cuda")
+    tabs = lay.source_tables(st.theta, st.m, st.v)
+    ref = lay.new_delta(lay.num_elements)
+    dte.dte_extract_delta(lay, tabs, *wl.hp.as_args(), ref)
+    cap = 100
+    pool32 = torch.full((4096,), 0x5A5A5A5A, dtype=torch.int32, device="cuda")
+    pool16 = torch.full((4096,), 0x5A5A, dtype=torch.int16, device="cuda")
+    got = lay.new_delta(cap)
+    got.offsets, got.values = pool32[1024:1024 + cap], pool16[1024:1024 + cap]
+    got.struct.offsets, got.struct.values = got.offsets.data_ptr(), got.values.data_ptr()
+    dte.dte_extract_delta_static(lay, tabs, *wl.hp.as_args(), got)
+    torch.cuda.synchronize()
+    assert ref.status_bits() == 0 and ref.total() > cap
+    assert got.status_bits() & dte.DTE_DEV_OVERFLOW
+    assert got.total() == ref.total() and torch.equal(got.list_ptr, ref.list_ptr)
+    assert bool((pool32[:1024] == 0x5A5A5A5A).all()) and bool((pool32[1024 + cap:] == 0x5A5A5A5A).all())
+    assert bool((pool16[:1024] == 0x5A5A).all()) and bool((pool16[1024 + cap:] == 0x5A5A).all())
+    # a plan without operations: every list empty, counters cleared
+    empty = dte.Layout([(8, 8)], [64, 0, 5], [])
+    d = empty.new_delta(4)
+    d.list_ptr.fill_(7)
+    d.counters.fill_(9)
+    t = torch.ones(64, dtype=torch.float32, device="cuda")
+    dte.dte_extract_delta_static(empty, empty.source_tables([t], [t], [t]), 1, 1e-3, 0.9, 0.999, 1e-8, 0.0, d)
+    torch.cuda.synchronize()
+    assert d.total() == 0 and d.status_bits() == 0 and int(d.list_ptr.abs().sum()) == 0
 
 
 def test_static_scratch_extract_rejects_what_does_not_fit():
