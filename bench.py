@@ -113,6 +113,9 @@ def build_workload(name: str, device):
     if name.startswith("moe:"):          # moe:<receiver TP>:<EP>[:<layers>]  (config 4's state, other inference layout)
         f = [int(x) for x in name.split(":")[1:]]
         return configs.config4(device, n_layers=f[2] if len(f) > 2 else 12, tp=f[0], ep=f[1])
+    if name.startswith("sweep:"):        # sweep:<lr>:<sigma_g>  (one point of the density sweep, t=100, wd=0.01)
+        f = name.split(":")[1:]
+        return configs.config5(float(f[0]), 100, 0.01, float(f[1]))
     raise SystemExit(f"unknown workload {name}")
 
 
@@ -238,39 +241,48 @@ def extract_traffic(n_elements):
         return None, {"error": f"{type(e).__name__}: {e}"}
 
 
-def time_leg(dte, wl, device, steps, warmup, peak, capacity_frac=0.03, with_clocks=True):
+def time_leg(dte, make_wl, device, steps, warmup, peak, capacity_frac=0.03, with_clocks=True, copies=1):
     """One more workload through the same timed loop as the headline: resident state, `warmup`
-    untimed steps, `steps` timed steps of extract + apply (CUDA events per step), L2 flushed
-    between steps when the state could sit in it.  Returns the leg's numbers; frees its memory."""
-    plan = wl.plan
-    st, shards = materialize_resident(wl, device, dte)
-    lay = dte.Layout.from_plan(plan, device.index or 0)
-    N = lay.num_elements
-    delta = lay.new_delta(int(N * capacity_frac) + 1024)
-    tabs = lay.source_tables(st.theta, st.m, st.v)
-    shard_tab = lay.shard_table(shards)
-    hp = wl.hp.as_args()
-    stream = torch.cuda.current_stream()
-    dte.dte_extract_delta(lay, tabs, *hp, delta)
-    torch.cuda.synchronize()
-    if delta.status_bits() & dte.DTE_DEV_OVERFLOW:       # dense sweep points: size discovery, then grow
-        delta = lay.new_delta(delta.total() + 1024)
+    untimed steps, `steps` timed steps of extract + apply (CUDA events per step).  A state that
+    could sit in the 126 MB L2 is generated `copies` times (seeds differ) and the steps rotate
+    over the copies, each with a layout of its own, so that every step reads inputs the L2 does
+    not hold: inputs larger than L2, and no dirty lines left behind by a flushing write.
+    Returns the leg's numbers; frees its memory."""
+    sets, N, names = [], 0, None
+    for i in range(copies):
+        wl = make_wl(i)
+        plan = wl.plan
+        st, shards = materialize_resident(wl, device, dte)
+        lay = dte.Layout.from_plan(plan, device.index or 0)
+        N = lay.num_elements
+        delta = lay.new_delta(int(N * capacity_frac) + 1024)
+        tabs = lay.source_tables(st.theta, st.m, st.v)
+        hp = wl.hp.as_args()
         dte.dte_extract_delta(lay, tabs, *hp, delta)
         torch.cuda.synchronize()
-    if delta.status_bits():
-        return {"workload": wl.name, "error": f"device status bits {delta.status_bits()}"}
-    M = delta.total()
-    flush = torch.empty(1 << 28, dtype=torch.uint8, device=device) if 12 * N < 2e9 else None
+        if delta.status_bits() & dte.DTE_DEV_OVERFLOW:       # dense sweep points: the sizes are exact, grow and repeat
+            delta = lay.new_delta(delta.total() + 1024)
+            dte.dte_extract_delta(lay, tabs, *hp, delta)
+            torch.cuda.synchronize()
+        if delta.status_bits():
+            return {"workload": wl.name, "error": f"device status bits {delta.status_bits()}"}
+        sets.append(dict(wl=wl, st=st, shards=shards, lay=lay, delta=delta, tabs=tabs, hp=hp,
+                         shard_tab=lay.shard_table(shards), M=delta.total()))
+    wl, lay, plan = sets[0]["wl"], sets[0]["lay"], sets[0]["wl"].plan
+    resident = 12 * N * copies
+    flush = torch.empty(1 << 28, dtype=torch.uint8, device=device) if resident < 1e9 else None
+    stream = torch.cuda.current_stream()
 
-    def step(ev=None):
+    def step(i, ev=None):
+        s = sets[i % copies]
         if ev: ev[0].record(stream)
-        dte.dte_extract_delta(lay, tabs, *hp, delta)
+        dte.dte_extract_delta(s["lay"], s["tabs"], *s["hp"], s["delta"])
         if ev: ev[1].record(stream)
-        dte.dte_apply(lay, delta, shard_tab)
+        dte.dte_apply(s["lay"], s["delta"], s["shard_tab"])
         if ev: ev[2].record(stream)
 
-    for _ in range(max(warmup, 3)):
-        step()
+    for i in range(max(warmup, 3, copies)):
+        step(i)
     torch.cuda.synchronize()
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
     sampler = ClockSampler(device.index or 0)
@@ -281,23 +293,29 @@ def time_leg(dte, wl, device, steps, warmup, peak, capacity_frac=0.03, with_cloc
     for i in range(steps):
         if flush is not None:
             flush.zero_()
-        step(evs[i])
+        step(i, evs[i])
     torch.cuda.synchronize()
     w1 = time.time()
     clocks = sampler.stop(w0, w1) if with_clocks else None
     ext = [e[0].elapsed_time(e[1]) for e in evs]
     app = [e[1].elapsed_time(e[2]) for e in evs]
     ext_avg, app_avg = sum(ext) / len(ext), sum(app) / len(app)
+    M = sum(s["M"] for s in sets) / copies
     gbps = (12.0 * N + 6.0 * M) / (ext_avg * 1e-3) / 1e9
+    if flush is not None:
+        l2 = "256 MB written between timed steps"
+    elif copies > 1:
+        l2 = f"{copies} copies of the state ({resident / 1e9:.2f} GB), one per step in rotation: inputs larger than L2"
+    else:
+        l2 = "inputs larger than L2"
     out = {"workload": wl.name, "elements_scanned": N, "changed": M, "changed_frac": M / N,
            "lists": lay.num_lists, "operations": len(plan.ops), "steps": steps,
            "hyper": {"step": wl.hp.step, "lr": wl.hp.lr, "wd": wl.hp.wd},
            "extract_ms": ext_avg, "extract_ms_min": min(ext), "extract_GBps": gbps, "frac_of_peak": gbps / peak,
-           "apply_ms": app_avg, "apply_Mchanged_per_s": M / (app_avg * 1e-3) / 1e6 if M else None,
-           "l2": "inputs larger than L2" if flush is None else "256 MB written between timed steps",
+           "apply_ms": app_avg, "apply_Mchanged_per_s": M / (app_avg * 1e-3) / 1e6 if M else None, "l2": l2,
            "gpu_launches": (lay.last_launch()["kernels"] + 1) * steps, "launch": lay.last_launch(), "clocks": clocks,
            **{k: v for k, v in wl.notes.items() if k in ("cold_experts", "sigma_g")}}
-    del st, shards, delta, lay, tabs, shard_tab, flush
+    del sets, flush, lay, wl, plan
     import gc
     gc.collect()
     torch.cuda.empty_cache()
@@ -309,6 +327,35 @@ def density_sweep_points():
     five learning rates at t = 100, wd = 0.01, and the two dense points at lr = 1e-4."""
     return [(lr, 100, 0.01, 1e-3) for lr in (1e-8, 1e-7, 1e-6, 1e-5, 1e-4)] + [(1e-4, 100, 0.01, 3e-3),
                                                                                 (1e-4, 100, 0.01, 1e-2)]
+
+
+def run_probes(device):
+    """What the memory system does for the path's two access patterns, without the path: a
+    read-only stream (extract) and isolated small accesses at ascending offsets, one per 67
+    elements as at 1.5 % density (apply).  Prints one JSON line."""
+    from paper_2608_00455_b200 import probes
+    out = {"read_only_stream": read_ceiling(device)}
+    n, stride, jitter = 60 << 20, 67, 60
+    off = probes.make_offsets(n, stride, jitter, device)
+    dst = torch.zeros(n * stride + 256, dtype=torch.int16, device=device)
+    sink = torch.zeros(1, dtype=torch.int32, device=device)
+    stream = torch.cuda.current_stream()
+    rates = {}
+    for ctas in (6, 12):
+        for mode, name in probes.SPARSE_MODES.items():
+            ms = []
+            for rep in range(6):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                probes.sparse_access(mode, off, dst, sink, ctas)
+                e1.record(stream)
+                torch.cuda.synchronize()
+                if rep:
+                    ms.append(e0.elapsed_time(e1))
+            rates[f"{name}, {ctas} CTAs/SM"] = {"ms": sum(ms) / len(ms), "G_per_s": n / (sum(ms) / len(ms) * 1e-3) / 1e9}
+    out["sparse_access"] = {"entries": n, "stride_elements": stride, "jitter": jitter, "element_bytes": 2,
+                            "destination_bytes": int(dst.numel() * 2), "rates": rates}
+    print(json.dumps(out), flush=True)
 
 
 def read_ceiling(device, nbytes=4 << 30, reps=10):
@@ -469,6 +516,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-codec", action="store_true", help="skip the storage-mediated path's legs")
+    ap.add_argument("--probes", action="store_true",
+                    help="time the memory-system probes (read-only stream, isolated sparse accesses) and exit")
     ap.add_argument("--no-extra-workloads", action="store_true",
                     help="skip the config 4 / config 1 / density-sweep legs that follow the headline workload")
     args = ap.parse_args()
@@ -485,6 +534,10 @@ def main():
 
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
+    if args.probes:
+        if rank == 0:
+            run_probes(device)
+        return
     dist = None
     if world > 1:
         import torch.distributed as dist
@@ -638,13 +691,14 @@ def main():
         torch.cuda.empty_cache()
         legs = max(10, min(args.steps, 30))
         t0 = time.time()
-        extra["config4"] = time_leg(dte, configs.config4(device), device, legs, args.warmup, peak, 0.04)
+        extra["config4"] = time_leg(dte, lambda i: configs.config4(device), device, legs, args.warmup, peak, 0.04)
         log(f"[bench] config 4: {extra['config4']} ({time.time() - t0:.0f} s)")
-        extra["config1"] = time_leg(dte, configs.config1(), device, 50, args.warmup, peak)
+        extra["config1"] = time_leg(dte, lambda i: configs.config1(seed=1234 + i), device, 48, args.warmup, peak, copies=8)
         log(f"[bench] config 1: {extra['config1']}")
         sweep = []
         for (lr, step_t, wd, sg) in density_sweep_points():
-            r = time_leg(dte, configs.config5(lr, step_t, wd, sg), device, 20, args.warmup, peak, 0.03, with_clocks=False)
+            r = time_leg(dte, lambda i: configs.config5(lr, step_t, wd, sg), device, 20, args.warmup, peak, 0.03,
+                         with_clocks=False)
             r["sigma_g"] = sg
             sweep.append(r)
             log(f"[bench] sweep lr={lr:g} sigma_g={sg:g}: rho={r.get('changed_frac')} extract {r.get('extract_GBps')} GB/s")

@@ -65,7 +65,7 @@ typedef enum dte_status {
 #define DTE_DEV_OVERFLOW 1u /* more changed elements than `capacity`; lists not produced   */
 #define DTE_DEV_BOUNDS 2u   /* apply met an offset >= numel of its shard, an entry for a NULL
                                shard, or a canonical index outside its tensor; entry skipped */
-#define DTE_DEV_TIMEOUT 4u  /* reserved (no kernel of this library waits on another CTA)  */
+#define DTE_DEV_TIMEOUT 4u  /* dte_push_wait gave up; no other kernel of this library waits   */
 #define DTE_DEV_CORRUPT 8u  /* unpack rejected a chunk (header or checksum); lists have holes */
 
 /* Source tensor p of the canonical training-side space: fp32, row-major.  ndim is 1 or 2;
@@ -248,6 +248,70 @@ DTE_API dte_status dte_op_counts(const dte_layout* layout, const dte_delta* delt
                                  void* cuda_stream);
 /* Number of operations the layout was created with. */
 DTE_API size_t dte_layout_num_ops(const dte_layout* layout);
+
+/* ---- Same-cluster transfer fused into the extract's tail (Section 4.3) ----------------------------
+ * Section 4.3 moves the update in two rounds: first the entry count of every planned operation,
+ * zeros included, then indices and values in the same order; a receiver applies an update only
+ * once all of it has arrived.  With NVLink peer access the sender can store straight into the
+ * receivers' memory, so both rounds collapse into the kernel that already moves every changed
+ * entry from the staging buffer to its ordered position: dte_extract_delta_push makes that kernel
+ * store each entry a second time, into the landing buffers of the receiver that owns the entry's
+ * list, and a closing kernel delivers, per receiver, the list boundaries, the per-operation counts
+ * (plan order, zeros included) and - after a system-scope fence, last of all - a status block
+ * whose epoch word tells the receiver that everything before it is complete.
+ *
+ * A receiver is the value of dte_shard_desc.receiver; the shards of one receiver must be
+ * consecutive in shard order (then its entries are one contiguous slice of the output).  All
+ * pointers of a target are DEVICE pointers this GPU can store to: its own memory, or a peer's
+ * mapped by CUDA peer access or IPC.  Only plain stores go to them.
+ *   offsets / values : `capacity` entries; receive the receiver's slice, lists in shard order
+ *   list_ptr  : (n_shards + 1) x uint64, boundaries RELATIVE to the slice; lists of other
+ *               receivers come out empty, so {offsets, values, capacity, list_ptr, counters} is a
+ *               dte_delta that dte_apply takes with the full layout and NULL for foreign shards
+ *   op_counts : dte_layout_receiver_num_ops(layout, r) x uint64: c_o of the operations whose
+ *               shard belongs to receiver r, in plan order, zeros included
+ *   status    : 4 x uint64 = { entries of the slice, epoch, DTE_DEV_* bits, operations }.  The
+ *               epoch word is written last (release at system scope).  DTE_DEV_OVERFLOW: the slice
+ *               exceeds `capacity`, or the sender's own delta overflowed; the sizes are exact, the
+ *               entries are not usable. */
+typedef struct dte_push_target {
+    uint32_t* offsets;
+    uint16_t* values;
+    uint64_t capacity;
+    uint64_t* list_ptr;
+    uint64_t* op_counts;
+    uint64_t* status;
+} dte_push_target;
+
+/* Number of receivers (largest dte_shard_desc.receiver + 1; 0 without shards) and the number of
+ * operations whose shard belongs to `receiver`. */
+DTE_API size_t dte_layout_num_receivers(const dte_layout* layout);
+DTE_API size_t dte_layout_receiver_num_ops(const dte_layout* layout, uint32_t receiver);
+
+/* dte_extract_delta that also delivers every receiver's share (see above).  `out` is filled
+ * exactly as by dte_extract_delta (the sender keeps its lists: the storage path or a retry may
+ * need them).  targets: HOST array of n_receivers >= dte_layout_num_receivers(layout) entries; a
+ * receiver without shards is skipped, a target whose `status` is NULL as well (nothing is
+ * delivered to it).  `epoch` is the value the receivers wait for: use one the status word cannot
+ * hold already, e.g. the policy version.  The first call on a layout uploads its receiver tables
+ * (cudaMalloc, synchronous).  Errors: DTE_ERR_LAYOUT if some receiver's shards are not
+ * consecutive; DTE_ERR_INVALID_ARG for null buffers of a used target; else as dte_extract_delta. */
+DTE_API dte_status dte_extract_delta_push(const dte_layout* layout, const float* const* theta,
+                                          const float* const* m, const float* const* v, int64_t step,
+                                          double lr, double beta1, double beta2, double eps, double wd,
+                                          const dte_delta* out, const dte_push_target* targets,
+                                          size_t n_receivers, uint64_t epoch, void* cuda_stream);
+
+/* Receiver side: enqueues a one-thread kernel that waits until status[1] == epoch (acquire at
+ * system scope), for at most timeout_ms milliseconds, and then fills `counters` (DEVICE, 4 x
+ * uint64) = { status[0], 0, status[2], 0 } so that a dte_apply enqueued behind it on the same
+ * stream sees a complete dte_delta.  If the time runs out, DTE_DEV_TIMEOUT is set in counters[2]
+ * together with DTE_DEV_OVERFLOW (so that dte_apply writes nothing) and the kernel returns; the
+ * context stays usable.  The wait holds one thread of one SM; enqueue it only when the sender's
+ * push is known to be on its way (on one GPU: after it, on the same stream), never in front of
+ * work it depends on.  timeout_ms is capped at 10000. */
+DTE_API dte_status dte_push_wait(const uint64_t* status, uint64_t epoch, uint32_t timeout_ms,
+                                 uint64_t* counters, int device, void* cuda_stream);
 
 /* ---- Chunk codec of the storage-mediated path (Section 4.4) ---------------------------------
  * Between clusters the changes travel through object storage (Section 4.4): what changed is

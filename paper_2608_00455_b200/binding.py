@@ -27,7 +27,8 @@ SYMBOLS = [
     "dte_extract_delta_host", "dte_status_string", "dte_last_error", "dte_layout_last_launch",
     "dte_extract_delta_static", "dte_extract_delta_groups", "dte_layout_num_groups",
     "dte_op_counts", "dte_layout_num_ops", "dte_chunk_count_bound", "dte_chunk_bytes_bound",
-    "dte_pack_chunks", "dte_unpack_chunks", "dte_apply_canonical",
+    "dte_pack_chunks", "dte_unpack_chunks", "dte_apply_canonical", "dte_extract_delta_push",
+    "dte_push_wait", "dte_layout_num_receivers", "dte_layout_receiver_num_ops",
 ]
 
 
@@ -53,6 +54,11 @@ _OP_DTYPE = np.dtype([("src_tensor", np.uint32), ("dst_shard", np.uint32), ("src
 class DeltaStruct(C.Structure):
     _fields_ = [("offsets", C.c_void_p), ("values", C.c_void_p), ("capacity", C.c_uint64),
                 ("list_ptr", C.c_void_p), ("counters", C.c_void_p)]
+
+
+class PushTargetStruct(C.Structure):
+    _fields_ = [("offsets", C.c_void_p), ("values", C.c_void_p), ("capacity", C.c_uint64),
+                ("list_ptr", C.c_void_p), ("op_counts", C.c_void_p), ("status", C.c_void_p)]
 
 
 class DteError(RuntimeError):
@@ -107,6 +113,14 @@ def lib() -> C.CDLL:
         L.dte_pack_chunks.restype = C.c_int
         L.dte_unpack_chunks.argtypes = [vp, vp, u64, vp, u64, vp, vp]
         L.dte_unpack_chunks.restype = C.c_int
+        L.dte_extract_delta_push.argtypes = [vp, vp, vp, vp, i64, dbl, dbl, dbl, dbl, dbl, vp, vp, C.c_size_t, u64, vp]
+        L.dte_extract_delta_push.restype = C.c_int
+        L.dte_push_wait.argtypes = [vp, u64, C.c_uint32, vp, C.c_int, vp]
+        L.dte_push_wait.restype = C.c_int
+        L.dte_layout_num_receivers.argtypes = [vp]
+        L.dte_layout_num_receivers.restype = C.c_size_t
+        L.dte_layout_receiver_num_ops.argtypes = [vp, C.c_uint32]
+        L.dte_layout_receiver_num_ops.restype = C.c_size_t
         L.dte_apply_canonical.argtypes = [vp, vp, vp, vp]
         L.dte_apply_canonical.restype = C.c_int
         L.dte_apply.argtypes = [vp, vp, vp, vp]
@@ -263,6 +277,13 @@ class Layout:
         return int(lib().dte_layout_num_groups(self._h))
 
     @property
+    def num_receivers(self) -> int:
+        return int(lib().dte_layout_num_receivers(self._h))
+
+    def receiver_num_ops(self, receiver: int) -> int:
+        return int(lib().dte_layout_receiver_num_ops(self._h, int(receiver)))
+
+    @property
     def num_elements(self) -> int:
         return int(lib().dte_layout_num_elements(self._h))
 
@@ -340,6 +361,56 @@ def dte_extract_delta_static(layout: Layout, tables, step, lr, beta1, beta2, eps
     _check(lib().dte_extract_delta_static(layout._h, th, mm, vv, int(step), float(lr), float(beta1),
                                           float(beta2), float(eps), float(wd), C.byref(delta.struct),
                                           _stream_ptr(stream)))
+
+
+class PushTarget:
+    """Landing buffers of one receiver for dte_extract_delta_push (see dte_push_target in dte.h).
+    On one GPU they are ordinary allocations; across GPUs the receiver allocates them and the sender
+    reaches them through peer access."""
+
+    def __init__(self, n_lists: int, capacity: int, n_ops: int, device):
+        dev = torch.device(device)
+        self.capacity, self.n_lists = int(capacity), int(n_lists)
+        self.offsets = torch.empty(max(1, self.capacity), dtype=torch.int32, device=dev)
+        self.values = torch.empty(max(1, self.capacity), dtype=torch.int16, device=dev)
+        self.list_ptr = torch.zeros(self.n_lists + 1, dtype=torch.int64, device=dev)
+        self.op_counts = torch.zeros(max(1, int(n_ops)), dtype=torch.int64, device=dev)
+        self.n_ops = int(n_ops)
+        self.status = torch.zeros(4, dtype=torch.int64, device=dev)
+        self.counters = torch.zeros(4, dtype=torch.int64, device=dev)     # filled by dte_push_wait
+
+    def struct(self) -> PushTargetStruct:
+        return PushTargetStruct(self.offsets.data_ptr(), self.values.data_ptr(), self.capacity,
+                                self.list_ptr.data_ptr(), self.op_counts.data_ptr(), self.status.data_ptr())
+
+    def delta(self) -> Delta:
+        """The receiver's share as a dte_delta (no copy); counters are those dte_push_wait fills."""
+        d = Delta.__new__(Delta)
+        d.capacity, d.n_lists = self.capacity, self.n_lists
+        d.offsets, d.values, d.list_ptr, d.counters = self.offsets, self.values, self.list_ptr, self.counters
+        d.struct = DeltaStruct(d.offsets.data_ptr(), d.values.data_ptr(), d.capacity, d.list_ptr.data_ptr(),
+                               d.counters.data_ptr())
+        return d
+
+
+def dte_extract_delta_push(layout: Layout, tables, step, lr, beta1, beta2, eps, wd, delta: Delta,
+                           targets: Sequence[Optional[PushTarget]], epoch: int, stream=None) -> None:
+    """Extract into `delta` and deliver every receiver's share into targets[receiver] (None: skip)."""
+    th, mm, vv = tables
+    arr = (PushTargetStruct * max(1, len(targets)))()
+    for r, t in enumerate(targets):
+        if t is not None:
+            arr[r] = t.struct()
+    _check(lib().dte_extract_delta_push(layout._h, th, mm, vv, int(step), float(lr), float(beta1), float(beta2),
+                                        float(eps), float(wd), C.byref(delta.struct), arr, len(targets),
+                                        int(epoch), _stream_ptr(stream)))
+
+
+def dte_push_wait(target: PushTarget, epoch: int, timeout_ms: int = 1000, stream=None) -> None:
+    """Receiver side: wait (bounded) for `epoch` in the target's status block, then fill
+    target.counters so that dte_apply(layout, target.delta(), ...) can follow on the same stream."""
+    _check(lib().dte_push_wait(target.status.data_ptr(), int(epoch), int(timeout_ms), target.counters.data_ptr(),
+                               target.status.device.index or 0, _stream_ptr(stream)))
 
 
 def dte_op_counts(layout: Layout, delta: Delta, stream=None) -> torch.Tensor:

@@ -79,63 +79,29 @@ Screen make_screen(const Consts& c) {
 // Where one extract call keeps its placement records, block sums, staging cursor and staged
 // entries: the layout's own buffers, or the fixed array of the allocation-free entry point.
 struct Scratch {
-    uint64_t* cursor;
+    uint64_t* cursor;       // two words: the staging cursor, then the ticket of small layouts
     uint64_t* rec;
     uint64_t* block_sum;
     uint32_t* stage;
+    bool clear_first;       // the two words are not known to be zero: clear them in the stream
 };
 
-// Enqueues the kernels of one extract: both extract launches (regular and packed tiles), then
-// the scan and gather that put the staged entries in order.  `groups`: per-parameter-group
-// constants (NULL: `c` applies to every tensor).  out->counters is cleared here; the cursor is
-// the only scratch word that must start at zero (records and block sums are rewritten in full,
-// staged entries are read only where this call wrote them).
+// Enqueues the kernels of one extract: both extract launches (packed and regular tiles), then
+// what puts the staged entries in order - for layouts of at most kSmallBlocks gather blocks only
+// the move (the extract's last tile does the scan itself), else reduce, scan and move.  `groups`:
+// per-parameter-group constants (NULL: `c` applies to every tensor).  The scan writes every word
+// of out->counters, and it leaves the cursor and the ticket at zero, the only scratch words that
+// must start there (records and block sums are rewritten in full, staged entries are read only
+// where this call wrote them): an ordinary call enqueues kernels and nothing else.
 dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<GroupConsts>* groups,
-                           const Scratch& sc, const dte_delta* out, cudaStream_t st) {
-    DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
+                           const Scratch& sc, const dte_delta* out, cudaStream_t st, bool push = false) {
     if (L->n_tiles == 0) {
+        DTE_CUDA(cudaMemsetAsync(out->counters, 0, 4 * sizeof(uint64_t), st));
         DTE_CUDA(cudaMemsetAsync(out->list_ptr, 0, (L->n_lists + 1) * sizeof(uint64_t), st));
         L->last_launch[0] = 0; L->last_launch[1] = 0; L->last_launch[2] = 0;
         return DTE_OK;
     }
-    DTE_CUDA(cudaMemsetAsync(sc.cursor, 0, sizeof(uint64_t), st));
-    ExtractParams p;
-    p.segs = L->d_segs;
-    p.theta = L->d_ptrs;
-    p.m = L->d_ptrs + L->n_tensors;
-    p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
-    p.cursor = reinterpret_cast<unsigned long long*>(sc.cursor);
-    p.rec = sc.rec;
-    p.stage = sc.stage;
-    p.stage_capacity = out->capacity;
-    p.c = c;
-    p.s = make_screen(c);
-    p.tensor_group = nullptr;
-    p.groups = nullptr;
-    bool div_bc1 = c.bc1 != 1.0f, div_decay = c.decay != 1.0f;
-    if (groups) {
-        // pageable source: staged by the runtime before the call returns
-        DTE_CUDA(cudaMemcpyAsync(L->d_groups, groups->data(), groups->size() * sizeof(GroupConsts),
-                                 cudaMemcpyHostToDevice, st));
-        p.tensor_group = L->d_tensor_group;
-        p.groups = L->d_groups;
-        div_bc1 = div_decay = false;
-        for (const GroupConsts& g : *groups) {
-            div_bc1 |= g.c.bc1 != 1.0f;
-            div_decay |= g.c.decay != 1.0f;
-        }
-    }
-    // one CTA per tile; packed tiles (short runs sharing a CTA; few) first, then the full tiles,
-    // which may start while the packed launch is still running: the two share nothing but the
-    // staging cursor (atomic) and write different placement records
-    p.tiles = L->d_packed;
-    p.n_tiles = L->n_packed;
-    dte_status s = launch_extract(p, div_bc1, div_decay, true, false, st);
-    if (s != DTE_OK) return s;
-    p.tiles = L->d_tiles;
-    p.n_tiles = L->n_regular;
-    s = launch_extract(p, div_bc1, div_decay, false, L->n_packed != 0, st);
-    if (s != DTE_OK) return s;
+    if (sc.clear_first) DTE_CUDA(cudaMemsetAsync(sc.cursor, 0, 2 * sizeof(uint64_t), st));
     GatherParams g;
     g.rec = sc.rec;
     g.block_sum = sc.block_sum;
@@ -152,11 +118,58 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
     g.capacity = out->capacity;
     g.list_ptr = out->list_ptr;
     g.counters = out->counters;
-    s = launch_gather(g, st);
+    g.cursor = reinterpret_cast<unsigned long long*>(sc.cursor);
+    g.n_recv = push ? L->n_receivers : 0;
+    g.recv_first_list = L->d_recv_first_list;
+    g.recv_base = L->d_recv_base;
+    g.rec_recv = L->d_rec_recv;
+    g.targets = L->d_targets;
+    const bool small = g.n_blocks <= (uint32_t)kSmallBlocks;
+    ExtractParams p;
+    p.segs = L->d_segs;
+    p.theta = L->d_ptrs;
+    p.m = L->d_ptrs + L->n_tensors;
+    p.v = L->d_ptrs + 2 * (size_t)L->n_tensors;
+    p.cursor = reinterpret_cast<unsigned long long*>(sc.cursor);
+    p.rec = sc.rec;
+    p.stage = sc.stage;
+    p.stage_capacity = out->capacity;
+    p.c = c;
+    p.s = make_screen(c);
+    p.tensor_group = nullptr;
+    p.groups = nullptr;
+    p.ticket = small ? reinterpret_cast<unsigned int*>(sc.cursor + 1) : nullptr;
+    p.ticket_total = L->n_tiles;
+    p.g = g;
+    bool div_bc1 = c.bc1 != 1.0f, div_decay = c.decay != 1.0f;
+    if (groups) {
+        // pageable source: staged by the runtime before the call returns
+        DTE_CUDA(cudaMemcpyAsync(L->d_groups, groups->data(), groups->size() * sizeof(GroupConsts),
+                                 cudaMemcpyHostToDevice, st));
+        p.tensor_group = L->d_tensor_group;
+        p.groups = L->d_groups;
+        div_bc1 = div_decay = false;
+        for (const GroupConsts& gc : *groups) {
+            div_bc1 |= gc.c.bc1 != 1.0f;
+            div_decay |= gc.c.decay != 1.0f;
+        }
+    }
+    // one CTA per tile; packed tiles (short runs sharing a CTA; few) first, then the full tiles,
+    // which may start while the packed launch is still running: the two share nothing but the
+    // staging cursor and the ticket (atomics) and write different placement records
+    p.tiles = L->d_packed;
+    p.n_tiles = L->n_packed;
+    dte_status s = launch_extract(p, div_bc1, div_decay, true, false, st);
+    if (s != DTE_OK) return s;
+    p.tiles = L->d_tiles;
+    p.n_tiles = L->n_regular;
+    s = launch_extract(p, div_bc1, div_decay, false, L->n_packed != 0, st);
+    if (s != DTE_OK) return s;
+    s = launch_gather(g, small, st);
     if (s != DTE_OK) return s;
     L->last_launch[0] = L->n_tiles;
     L->last_launch[1] = L->n_tiles;                         // one CTA per tile
-    L->last_launch[2] = 3 + (L->n_regular ? 1 : 0) + (L->n_packed ? 1 : 0);
+    L->last_launch[2] = (small ? 1 : 3) + (L->n_regular ? 1 : 0) + (L->n_packed ? 1 : 0);
     return DTE_OK;
 }
 
@@ -164,7 +177,7 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
 // caller's capacity; it is (re)allocated only when a call brings a larger capacity than any
 // before it.
 dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out, cudaStream_t st,
-                           const std::vector<GroupConsts>* groups = nullptr) {
+                           const std::vector<GroupConsts>* groups = nullptr, bool push = false) {
     if (L->n_tiles && out->capacity > L->stage_capacity) {
         DTE_CUDA(cudaStreamSynchronize(st));
         cudaFree(L->d_stage);
@@ -173,8 +186,13 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
         DTE_CUDA(cudaMalloc((void**)&L->d_stage, out->capacity * sizeof(uint32_t)));
         L->stage_capacity = out->capacity;
     }
-    const Scratch sc{L->d_cursor, L->d_rec, L->d_block_sum, L->d_stage};
-    return enqueue_kernels(L, c, groups, sc, out, st);
+    // The kernels leave the cursor and the ticket at zero.  If an earlier call stopped half-way
+    // (a launch failed), they may not be: clear them in the stream this once.
+    const Scratch sc{L->d_cursor, L->d_rec, L->d_block_sum, L->d_stage, !L->scratch_clean};
+    L->scratch_clean = false;
+    const dte_status s = enqueue_kernels(L, c, groups, sc, out, st, push);
+    L->scratch_clean = (s == DTE_OK);
+    return s;
 }
 
 }  // namespace
@@ -225,6 +243,101 @@ extern "C" dte_status dte_extract_delta_groups(const dte_layout* layout, const f
     s = sync_source_table(L, theta, m, v, st);
     if (s != DTE_OK) return s;
     return enqueue_extract(L, groups[0].c, out, st, &groups);
+}
+
+// ---- extract + delivery to the receivers (Section 4.3) -----------------------------------------
+namespace {
+template <class T>
+dte_status upload_once(T** dst, const std::vector<T>& src) {
+    if (*dst) return DTE_OK;
+    T* ptr = nullptr;
+    DTE_CUDA(cudaMalloc((void**)&ptr, std::max<size_t>(1, src.size()) * sizeof(T)));
+    if (!src.empty()) {
+        const cudaError_t e = cudaMemcpy(ptr, src.data(), src.size() * sizeof(T), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) { cudaFree(ptr); return cuda_fail(e, "upload of the receiver tables"); }
+    }
+    *dst = ptr;
+    return DTE_OK;
+}
+}  // namespace
+
+extern "C" dte_status dte_extract_delta_push(const dte_layout* layout, const float* const* theta,
+                                             const float* const* m, const float* const* v, int64_t step,
+                                             double lr, double beta1, double beta2, double eps, double wd,
+                                             const dte_delta* out, const dte_push_target* targets,
+                                             size_t n_receivers, uint64_t epoch, void* cuda_stream) {
+    if (!layout) return fail(DTE_ERR_INVALID_ARG, "layout is null");
+    if (layout->n_tensors && (!theta || !m || !v)) return fail(DTE_ERR_INVALID_ARG, "null pointer table");
+    dte_status s = check_delta(out);
+    if (s != DTE_OK) return s;
+    dte_layout* L = const_cast<dte_layout*>(layout);
+    if (L->n_receivers == 0) return fail(DTE_ERR_LAYOUT, "the layout has no receivers (no shards, or receiver ids above 65534)");
+    if (!L->recv_contiguous)
+        return fail(DTE_ERR_LAYOUT, "the shards of some receiver are not consecutive in shard order: its entries are not one slice");
+    if (!targets || n_receivers < L->n_receivers) return fail(DTE_ERR_INVALID_ARG, "fewer targets than receivers");
+    std::vector<dte_push_target> tab(targets, targets + L->n_receivers);
+    for (uint32_t r = 0; r < L->n_receivers; ++r) {
+        dte_push_target& t = tab[r];
+        const bool has_shards = L->h_recv_first_list[L->n_receivers + r] > L->h_recv_first_list[r];
+        if (!has_shards || !t.status) { t = dte_push_target{}; continue; }     // nothing is delivered to it
+        if (!t.list_ptr || (t.capacity && (!t.offsets || !t.values)) || (L->h_recv_num_ops[r] && !t.op_counts))
+            return fail(DTE_ERR_INVALID_ARG, "a push target with a status block lacks list_ptr, entry or count buffers");
+    }
+    float c5[5];
+    s = dte_derive_constants(step, lr, beta1, beta2, eps, wd, c5);
+    if (s != DTE_OK) return s;
+    DeviceGuard g(L->device);
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // first use: receiver tables to the device
+    s = upload_once(&L->d_recv_first_list, L->h_recv_first_list);
+    if (s == DTE_OK) s = upload_once(&L->d_recv_num_ops, L->h_recv_num_ops);
+    if (s == DTE_OK) s = upload_once(&L->d_op_recv, L->h_op_recv);
+    if (s == DTE_OK) s = upload_once(&L->d_op_slot, L->h_op_slot);
+    if (s == DTE_OK) s = upload_once(&L->d_rec_recv, L->h_rec_recv);
+    if (s == DTE_OK && !L->d_recv_base) DTE_CUDA(cudaMalloc((void**)&L->d_recv_base, L->n_receivers * sizeof(uint64_t)));
+    if (s == DTE_OK && !L->d_targets) DTE_CUDA(cudaMalloc((void**)&L->d_targets, L->n_receivers * sizeof(dte_push_target)));
+    if (s != DTE_OK) return s;
+    const bool same = L->targets_valid && L->h_targets.size() == tab.size() &&
+                      std::memcmp(L->h_targets.data(), tab.data(), tab.size() * sizeof(dte_push_target)) == 0;
+    if (!same) {
+        L->targets_valid = false;
+        // pageable source: staged by the runtime before the call returns
+        DTE_CUDA(cudaMemcpyAsync(L->d_targets, tab.data(), tab.size() * sizeof(dte_push_target), cudaMemcpyHostToDevice, st));
+        L->h_targets.swap(tab);
+        L->targets_valid = true;
+    }
+    s = sync_source_table(L, theta, m, v, st);
+    if (s != DTE_OK) return s;
+    const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
+    s = enqueue_extract(L, c, out, st, nullptr, true);
+    if (s != DTE_OK) return s;
+    PushFinishParams f;
+    f.ranges = L->d_op_ranges;
+    f.n_ops = L->n_ops;
+    f.op_recv = L->d_op_recv;
+    f.op_slot = L->d_op_slot;
+    f.offsets = out->offsets;
+    f.list_ptr = out->list_ptr;
+    f.counters = out->counters;
+    f.capacity = out->capacity;
+    f.n_lists = L->n_lists;
+    f.n_recv = L->n_receivers;
+    f.recv_first_list = L->d_recv_first_list;
+    f.recv_num_ops = L->d_recv_num_ops;
+    f.targets = L->d_targets;
+    f.epoch = epoch;
+    f.ticket = reinterpret_cast<unsigned int*>(L->d_cursor + 2);
+    s = launch_push_finish(f, st);
+    if (s == DTE_OK) L->last_launch[2] += 1;
+    return s;
+}
+
+extern "C" dte_status dte_push_wait(const uint64_t* status, uint64_t epoch, uint32_t timeout_ms,
+                                    uint64_t* counters, int device, void* cuda_stream) {
+    if (!status || !counters) return fail(DTE_ERR_INVALID_ARG, "status / counters is null");
+    if (((uintptr_t)status | (uintptr_t)counters) & 7u) return fail(DTE_ERR_INVALID_ARG, "status / counters must be 8-byte aligned");
+    DeviceGuard g(device);
+    return launch_push_wait(status, epoch, timeout_ms, counters, (cudaStream_t)cuda_stream);
 }
 
 namespace {
@@ -525,12 +638,13 @@ extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const f
     if (s != DTE_OK) return s;
     s = sync_source_table(L, theta, m, v, st);
     if (s != DTE_OK) return s;
-    // the array keeps whatever the previous call left; enqueue_kernels clears the one word (the
-    // cursor) that must start at zero and every other part is written before it is read
+    // the array keeps whatever the previous call left - possibly a call on another layout, or one
+    // that was cut short - so the two words that must start at zero (cursor and ticket) are cleared
+    // in the stream every time; every other part is written before it is read
     const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
     const Scratch sc{reinterpret_cast<uint64_t*>(base + kStaticCursorOff),
                      reinterpret_cast<uint64_t*>(base + kStaticRecOff),
                      reinterpret_cast<uint64_t*>(base + kStaticBlockSumOff),
-                     reinterpret_cast<uint32_t*>(base + kStaticStageOff)};
+                     reinterpret_cast<uint32_t*>(base + kStaticStageOff), true};
     return enqueue_kernels(L, c, nullptr, sc, out, st);
 }

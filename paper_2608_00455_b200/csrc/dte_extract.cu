@@ -307,19 +307,54 @@ __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint3
     return qn;
 }
 
+// The tail of a small layout's extract: the CTA that finishes last (all launches of the call
+// counted) turns the placement records into the gather's block bases, the totals and the
+// boundaries of trailing empty lists - what gather_reduce and gather_scan do for large layouts -
+// and leaves the cursor and the ticket at zero for the next call.  Nobody waits for anybody.
+__device__ void finish_small(const ExtractParams& p, uint64_t* s_bsum) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const GatherParams& g = p.g;
+    for (uint32_t b = warp; b < g.n_blocks; b += kWarps) {
+        uint32_t sum = 0;
+        for (uint32_t j = lane; j < (uint32_t)kRecsPerBlock; j += 32) {
+            const uint32_t r = b * kRecsPerBlock + j;
+            if (r < g.n_rec) sum += (uint32_t)(__ldcg(g.rec + r) & kRecCountMask);   // written by other SMs: L2
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
+        if (lane == 0) s_bsum[b] = sum;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint64_t run = 0;
+        for (uint32_t b = 0; b < g.n_blocks; ++b) {
+            g.block_sum[b] = run;
+            run += s_bsum[b];
+        }
+        s_bsum[kSmallBlocks] = run;
+        *p.cursor = 0ull;
+        *p.ticket = 0u;
+    }
+    __syncthreads();
+    gather_finish_totals(g, s_bsum[kSmallBlocks], threadIdx.x, kThreads);
+}
+
 // GROUPS: the constants come from the tile's parameter group instead of the kernel parameters.
 template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED>
 __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const ExtractParams p) {
+    // Programmatic dependent launch.  The packed-tile launch of a call goes first and lets the
+    // regular-tile launch start at once: the two share nothing but the atomic staging cursor.  The
+    // regular-tile launch gives the signal late, so that what follows it (the gather of a small
+    // layout, launched the same way) is set up while the last tiles finish and does not sit on
+    // the SMs before.  A no-op when the next launch in the stream did not ask for it.
+    if (PACKED) asm volatile("griddepcontrol.launch_dependents;");
     // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
     // (dynamic shared memory: kWarps * kWarpTile words, may exceed the 48 KB static limit)
-    // The two launches of one extract (packed tiles, then regular tiles) are independent: let the
-    // second one start while this one still runs (programmatic dependent launch; a no-op when the
-    // next launch in the stream did not ask for it).
-    asm volatile("griddepcontrol.launch_dependents;");
     extern __shared__ __align__(16) uint32_t s_queue[];
     __shared__ uint32_t s_count[kWarps];
     __shared__ unsigned long long s_pos;
     __shared__ StridedGeom s_geom[kWarps];
+    __shared__ uint32_t s_last;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* queue = s_queue + warp * kWarpTile;
     Consts c = p.c;
@@ -339,6 +374,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
             sc.ka = __uint_as_float(g1.y); sc.kb = __uint_as_float(g1.z); sc.kc = __uint_as_float(g1.w);
             sc.kappa = __uint_as_float(g2.x);
         }
+
         const float lr = c.lr;
 
         // ---- phase A: stream, screen, queue the undecided elements in element order ---------
@@ -350,6 +386,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
         else
             qn = phase_a<DIV_BC1, DIV_DECAY, false>(cur, lane, queue, sc, lr);
         __syncwarp();
+        if (!PACKED) asm volatile("griddepcontrol.launch_dependents;");
 
         // ---- phase B: exact evaluation of the queue, 32 entries per round; the changed
         //      entries are compacted to the front of the queue as (index | value << 16) -----
@@ -407,6 +444,10 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
             if (total) pos0 = atomicAdd(p.cursor, (unsigned long long)total);
             s_pos = pos0;
             p.rec[tile] = ((uint64_t)pos0 << kRecCountBits) | total;
+            if (p.ticket) {       // small layout: is this the last tile of the call to finish?
+                __threadfence();
+                s_last = atomicAdd(p.ticket, 1u) == p.ticket_total - 1u;
+            }
         }
         __syncthreads();
         const unsigned long long pos = s_pos + before;
@@ -414,6 +455,11 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
         for (uint32_t q = lane; q < n_changed; q += 32)
             if (pos + q < p.stage_capacity)               // beyond it the call overflows anyway
                 p.stage[pos + q] = queue[q] + rel;
+    }
+    if (p.ticket && s_last) {
+        __syncthreads();                                   // the queues are free now
+        __threadfence();
+        finish_small(p, reinterpret_cast<uint64_t*>(s_queue));
     }
     // The launch of the regular tiles may have begun before the launch of the packed tiles ended.
     // What follows in the stream (the gather) is ordered after THIS grid only, so this grid must

@@ -1,9 +1,12 @@
 // Ordered placement of the staged entries ("count, then write"): a scan over the
 // per-tile placement records gives every tile its position in the concatenated,
 // list-ordered output (lists in shard order, ascending offsets within a list), and a gather
-// moves its entries from the staging buffer to that position.  Three small launches; the
-// data they touch are the records (8 bytes per 9216 scanned elements) and the changed
+// moves its entries from the staging buffer to that position.  Three small launches (for small
+// layouts the extract's last tile does the first two steps itself and only the move is launched);
+// the data they touch are the records (8 bytes per 9216 scanned elements) and the changed
 // entries themselves.  No kernel waits on another CTA.
+#include <algorithm>
+
 #include "dte_internal.cuh"
 
 namespace dte {
@@ -69,20 +72,19 @@ __global__ void __launch_bounds__(kScanThreads) gather_scan_kernel(const GatherP
         if (threadIdx.x == kScanThreads - 1) s_carry = excl + x;
         __syncthreads();
     }
-    const uint64_t total = s_carry;
-    if (threadIdx.x == 0) {
-        p.counters[0] = total;
-        p.counters[1] = p.scanned;
-        p.list_ptr[p.n_lists] = total;
-        if (total > p.capacity) atomicOr((unsigned long long*)(p.counters + 2), (unsigned long long)DTE_DEV_OVERFLOW);
-    }
-    // lists after which no tile follows end (and start) at the total
-    for (uint32_t k = threadIdx.x; k < p.n_lists; k += kScanThreads)
-        if (p.list_first_rec[k] >= p.n_rec) p.list_ptr[k] = total;
+    gather_finish_totals(p, s_carry, threadIdx.x, kScanThreads);
+    if (threadIdx.x == 0) *p.cursor = 0ull;     // every tile has reserved its room: ready for the next call
 }
 
 // ---- 3. per block: local scan, list starts, gather ---------------------------------------------
-__global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const GatherParams p) {
+// PUSH: every entry is also stored into the landing buffers of the receiver that owns its list
+// (dte_extract_delta_push): plain stores to memory that may be a peer GPU's.
+template <bool PUSH>
+__global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kernel(const GatherParams p) {
+    // Small layouts launch this kernel so that it may be set up while the last extract tiles still
+    // run (programmatic dependent launch): nothing the extract wrote may be read before this.
+    // Returns at once in an ordinary launch.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     __shared__ uint32_t s_prefix[kRecsPerBlock + 1];   // exclusive prefix of counts within the block
     __shared__ uint64_t s_pos[kRecsPerBlock];          // staging position of each record
     __shared__ uint32_t s_warp[kGatherThreads / 32];
@@ -140,6 +142,10 @@ __global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const Ga
     const uint32_t* src8[kRecsPerWarp];
     uint32_t* off8[kRecsPerWarp];
     uint16_t* val8[kRecsPerWarp];
+    // PUSH: the same run in the receiver's buffers, cut where the receiver's capacity ends
+    uint32_t* roff8[kRecsPerWarp];
+    uint16_t* rval8[kRecsPerWarp];
+    uint32_t rcnt8[kRecsPerWarp];
     uint32_t longest = 0, packed_recs = 0;
 #pragma unroll
     for (int r = 0; r < kRecsPerWarp; ++r) {
@@ -153,6 +159,21 @@ __global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const Ga
         base8[r] = (uint32_t)b;
         if (b & kRecBasePacked) packed_recs |= 1u << r;
         longest = max(longest, cnt8[r]);
+        if (PUSH) {
+            rcnt8[r] = 0;
+            roff8[r] = nullptr;
+            rval8[r] = nullptr;
+            if (cnt8[r]) {
+                const uint32_t recv = p.rec_recv[base_rec + j];
+                const dte_push_target t = p.targets[recv];
+                const uint64_t at = out_base + first - p.recv_base[recv];     // position in the receiver's slice
+                if (t.status && at < t.capacity) {
+                    rcnt8[r] = (uint32_t)min((uint64_t)cnt8[r], t.capacity - at);
+                    roff8[r] = t.offsets + at;
+                    rval8[r] = t.values + at;
+                }
+            }
+        }
     }
     for (uint32_t q = lane; q < longest; q += 32) {
         uint32_t w[kRecsPerWarp];
@@ -164,30 +185,158 @@ __global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const Ga
             if (q < cnt8[r]) {
                 // a regular tile is one destination run: base + (warp * kWarpTile + index); the
                 // offsets of packed tiles are put right below
-                off8[r][q] = base8[r] + (w[r] & 0xFFFFu);
+                const uint32_t off = base8[r] + (w[r] & 0xFFFFu);
+                off8[r][q] = off;
                 val8[r][q] = (uint16_t)(w[r] >> 16);
+                if (PUSH && q < rcnt8[r]) {
+                    roff8[r][q] = off;
+                    rval8[r][q] = (uint16_t)(w[r] >> 16);
+                }
             }
     }
     // packed tiles (few): every piece has a destination base of its own
-    if (packed_recs == 0) return;
+    if (packed_recs) {
 #pragma unroll
-    for (int r = 0; r < kRecsPerWarp; ++r) {
-        if (!(packed_recs & (1u << r))) continue;
-        const TileDesc* d = p.packed + (size_t)base8[r] * kSub;
-        for (uint32_t q = lane; q < cnt8[r]; q += 32) {
-            const uint32_t idx = src8[r][q] & 0xFFFFu;
-            const uint32_t piece = idx / kWarpTile;
-            off8[r][q] = __ldg(&d[piece].dst_off) + (idx - piece * kWarpTile);
+        for (int r = 0; r < kRecsPerWarp; ++r) {
+            if (!(packed_recs & (1u << r))) continue;
+            const TileDesc* d = p.packed + (size_t)base8[r] * kSub;
+            for (uint32_t q = lane; q < cnt8[r]; q += 32) {
+                const uint32_t idx = src8[r][q] & 0xFFFFu;
+                const uint32_t piece = idx / kWarpTile;
+                const uint32_t off = __ldg(&d[piece].dst_off) + (idx - piece * kWarpTile);
+                off8[r][q] = off;
+                if (PUSH && q < rcnt8[r]) roff8[r][q] = off;
+            }
         }
+    }
+    // the receivers' memory may be another GPU's: this thread's stores must have arrived there
+    // before anything later in the stream (the status block) tells the receiver so
+    if (PUSH) __threadfence_system();
+}
+
+// ---- 4. closing kernel of a push: counts, boundaries and the status block of every receiver -----
+__device__ __forceinline__ uint64_t lower_bound_offset(const uint32_t* offsets, uint64_t lo, uint64_t hi, uint64_t key) {
+    while (lo < hi) {          // first entry in [lo, hi) with offset >= key
+        const uint64_t mid = (lo + hi) >> 1;
+        if ((uint64_t)offsets[mid] < key) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+constexpr int kFinishThreads = 256;
+
+__global__ void __launch_bounds__(kFinishThreads) push_finish_kernel(const PushFinishParams p) {
+    __shared__ uint32_t s_last;
+    const uint64_t bits = p.counters[2];
+    const uint64_t total = p.list_ptr[p.n_lists];
+    const bool incomplete = total > p.capacity || (bits & (DTE_DEV_OVERFLOW | DTE_DEV_CORRUPT));
+    const uint32_t tid = blockIdx.x * kFinishThreads + threadIdx.x, n_thr = gridDim.x * kFinishThreads;
+    // c_o of every operation, into its receiver's count array at the operation's plan position
+    for (uint32_t o = tid; o < p.n_ops; o += n_thr) {
+        const dte_push_target t = p.targets[p.op_recv[o]];
+        if (!t.status) continue;
+        uint64_t c = 0;
+        if (!incomplete) {
+            const OpRange r = p.ranges[o];
+            const uint64_t a = p.list_ptr[r.list], b = p.list_ptr[r.list + 1];
+            c = lower_bound_offset(p.offsets, a, b, r.end) - lower_bound_offset(p.offsets, a, b, r.begin);
+        }
+        t.op_counts[p.op_slot[o]] = c;
+    }
+    // list boundaries relative to the receiver's slice (lists of other receivers: empty)
+    const uint32_t per = p.n_lists + 1;
+    for (uint64_t i = tid; i < (uint64_t)p.n_recv * per; i += n_thr) {
+        const uint32_t r = (uint32_t)(i / per), k = (uint32_t)(i - (uint64_t)r * per);
+        const dte_push_target t = p.targets[r];
+        if (!t.status) continue;
+        const uint64_t lo = p.list_ptr[p.recv_first_list[r]], hi = p.list_ptr[p.recv_first_list[p.n_recv + r]];
+        t.list_ptr[k] = min(max(p.list_ptr[k], lo), hi) - lo;
+    }
+    // the block that finishes last publishes: everything above must have arrived first
+    __threadfence_system();
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = atomicAdd(p.ticket, 1u) == gridDim.x - 1;
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence_system();
+    for (uint32_t r = threadIdx.x; r < p.n_recv; r += kFinishThreads) {
+        const dte_push_target t = p.targets[r];
+        if (!t.status) continue;
+        const uint64_t n = p.list_ptr[p.recv_first_list[p.n_recv + r]] - p.list_ptr[p.recv_first_list[r]];
+        t.status[0] = n;
+        t.status[2] = (bits & ~(uint64_t)DTE_DEV_OVERFLOW) | ((incomplete || n > t.capacity) ? DTE_DEV_OVERFLOW : 0u);
+        t.status[3] = p.recv_num_ops[r];
+        __threadfence_system();
+        asm volatile("st.release.sys.global.u64 [%0], %1;" ::"l"(t.status + 1), "l"(p.epoch) : "memory");
+    }
+    if (threadIdx.x == 0) *p.ticket = 0u;
+}
+
+dte_status launch_push_finish(const PushFinishParams& p, cudaStream_t st) {
+    const uint64_t work = std::max<uint64_t>(p.n_ops, (uint64_t)p.n_recv * (p.n_lists + 1));
+    const int blocks = (int)std::min<uint64_t>(std::max<uint64_t>(1, (work + kFinishThreads - 1) / kFinishThreads), 1024);
+    push_finish_kernel<<<blocks, kFinishThreads, 0, st>>>(p);
+    DTE_CUDA(cudaGetLastError());
+    return DTE_OK;
+}
+
+// ---- receiver side: wait (bounded) for the status block of an epoch -----------------------------
+__global__ void push_wait_kernel(const uint64_t* status, uint64_t epoch, uint64_t timeout_ns, uint64_t max_polls,
+                                 uint64_t* counters) {
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    unsigned long long t0, now;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+    bool arrived = false;
+    for (uint64_t i = 0; i < max_polls; ++i) {       // two limits: the clock, and a poll count should the clock stall
+        unsigned long long v;
+        asm volatile("ld.acquire.sys.global.u64 %0, [%1];" : "=l"(v) : "l"(status + 1) : "memory");
+        if (v == epoch) { arrived = true; break; }
+        asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(now));
+        if (now - t0 > timeout_ns) break;
+        __nanosleep(500);
+    }
+    if (arrived) {
+        unsigned long long n, b;
+        asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(n) : "l"(status) : "memory");
+        asm volatile("ld.relaxed.sys.global.u64 %0, [%1];" : "=l"(b) : "l"(status + 2) : "memory");
+        counters[0] = n; counters[1] = 0; counters[2] = b; counters[3] = 0;
+    } else {
+        counters[0] = 0; counters[1] = 0; counters[3] = 0;
+        counters[2] = DTE_DEV_TIMEOUT | DTE_DEV_OVERFLOW;     // nothing usable: apply must not write
     }
 }
 
-dte_status launch_gather(const GatherParams& p, cudaStream_t st) {
+dte_status launch_push_wait(const uint64_t* status, uint64_t epoch, uint32_t timeout_ms, uint64_t* counters,
+                            cudaStream_t st) {
+    const uint64_t ms = std::min<uint32_t>(timeout_ms, 10000u);
+    push_wait_kernel<<<1, 32, 0, st>>>(status, epoch, ms * 1000000ull, ms * 2000ull + 1, counters);
+    DTE_CUDA(cudaGetLastError());
+    return DTE_OK;
+}
+
+// small: the extract's last tile has done the scan already (finish_small in dte_extract.cu); only
+// the move is left, launched so that it can be set up under the extract's tail.
+dte_status launch_gather(const GatherParams& p, bool small, cudaStream_t st) {
+    if (small) {
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(p.n_blocks);
+        cfg.blockDim = dim3(kGatherThreads);
+        cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = 1;
+        if (p.n_recv) DTE_CUDA(cudaLaunchKernelEx(&cfg, gather_move_kernel<true>, p));
+        else DTE_CUDA(cudaLaunchKernelEx(&cfg, gather_move_kernel<false>, p));
+        return DTE_OK;
+    }
     gather_reduce_kernel<<<p.n_blocks, kGatherThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     gather_scan_kernel<<<1, kScanThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
-    gather_move_kernel<<<p.n_blocks, kGatherThreads, 0, st>>>(p);
+    if (p.n_recv) gather_move_kernel<true><<<p.n_blocks, kGatherThreads, 0, st>>>(p);
+    else gather_move_kernel<false><<<p.n_blocks, kGatherThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }

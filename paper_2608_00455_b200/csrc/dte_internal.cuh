@@ -69,6 +69,7 @@ struct SegRec {
 constexpr int kRecCountBits = 14;                      // count <= kTile
 constexpr uint64_t kRecCountMask = (1ull << kRecCountBits) - 1;
 constexpr int kRecsPerBlock = 64;                      // records one gather CTA handles
+constexpr int kSmallBlocks = 64;                       // layouts up to this many gather blocks take the short path
 // A staged entry is one 32-bit word: (warp * kWarpTile + element index in the warp-tile) in the low
 // 16 bits, the BF16 value in the high 16.  The gather turns it into (offset, value) with the tile's
 // destination base: rec_base[r] = dst_off of a regular tile, or kRecBasePacked | index of a packed
@@ -93,23 +94,6 @@ struct __align__(16) GroupConsts {
 };
 static_assert(sizeof(GroupConsts) == 48, "GroupConsts is read as three uint4");
 
-struct ExtractParams {
-    const TileDesc* tiles;       // regular tiles: one descriptor each; packed tiles: kSub each
-    const SegRec* segs;
-    const float* const* theta;   // device table, n_tensors
-    const float* const* m;
-    const float* const* v;
-    unsigned long long* cursor;  // zeroed before launch: entries appended to the staging buffer
-    uint64_t* rec;               // n_tiles placement records (written in full)
-    uint32_t* stage;             // staging buffer, stage_capacity words: tile-relative index | value << 16
-    uint64_t stage_capacity;
-    uint32_t n_tiles;            // tiles handled by this launch
-    Consts c;                    // single-group calls: constants in the kernel parameters
-    Screen s;
-    const uint32_t* tensor_group;   // per-group calls: group of each source tensor ...
-    const GroupConsts* groups;      // ... and the constants of each group (NULL otherwise)
-};
-
 struct GatherParams {
     const uint64_t* rec;
     uint64_t* block_sum;             // n_blocks; reduce writes sums, scan turns them into bases
@@ -125,7 +109,37 @@ struct GatherParams {
     uint64_t capacity;
     uint64_t* list_ptr;
     uint64_t* counters;
+    unsigned long long* cursor;      // staging cursor: left at zero for the next call
+    // delivery to the receivers (dte_extract_delta_push); n_recv == 0: none
+    uint32_t n_recv;
+    const uint32_t* recv_first_list; // n_recv: first list of each receiver (then n_recv: one past its last)
+    uint64_t* recv_base;             // n_recv: output position where each receiver's slice starts
+    const uint16_t* rec_recv;        // n_rec: receiver of each tile's list
+    const dte_push_target* targets;  // n_recv, device copy
 };
+
+struct ExtractParams {
+    const TileDesc* tiles;       // regular tiles: one descriptor each; packed tiles: kSub each
+    const SegRec* segs;
+    const float* const* theta;   // device table, n_tensors
+    const float* const* m;
+    const float* const* v;
+    unsigned long long* cursor;  // zeroed before launch: entries appended to the staging buffer
+    uint64_t* rec;               // n_tiles placement records (written in full)
+    uint32_t* stage;             // staging buffer, stage_capacity words: tile-relative index | value << 16
+    uint64_t stage_capacity;
+    uint32_t n_tiles;            // tiles handled by this launch
+    Consts c;                    // single-group calls: constants in the kernel parameters
+    Screen s;
+    const uint32_t* tensor_group;   // per-group calls: group of each source tensor ...
+    const GroupConsts* groups;      // ... and the constants of each group (NULL otherwise)
+    // small layouts (at most kSmallBlocks gather blocks): the tile that finishes last, counted over
+    // all launches of the call on `ticket`, does the scan itself (see finish_small); NULL otherwise
+    unsigned int* ticket;
+    uint32_t ticket_total;
+    GatherParams g;
+};
+
 
 struct ApplyParams {
     const uint32_t* offsets;
@@ -171,6 +185,26 @@ struct OpRange {
     uint64_t begin, end;   // receiver-local flat range [begin, end); begin == end for empty overlaps
 };
 
+// Closing kernel of dte_extract_delta_push: per-operation counts, list boundaries and the status
+// block of every receiver.
+struct PushFinishParams {
+    const OpRange* ranges;
+    uint32_t n_ops;
+    const uint32_t* op_recv;          // n_ops: receiver of the operation's shard
+    const uint32_t* op_slot;          // n_ops: position among that receiver's operations (plan order)
+    const uint32_t* offsets;          // the sender's own lists
+    const uint64_t* list_ptr;
+    const uint64_t* counters;
+    uint64_t capacity;
+    uint32_t n_lists;
+    uint32_t n_recv;
+    const uint32_t* recv_first_list;  // 2 n_recv: first list, then one past the last list
+    const uint32_t* recv_num_ops;     // n_recv
+    const dte_push_target* targets;   // n_recv, device copy
+    uint64_t epoch;
+    unsigned int* ticket;             // rests at zero
+};
+
 // Chunk codec (storage-mediated path).
 struct PackParams {
     const uint32_t* offsets;
@@ -199,6 +233,37 @@ struct UnpackParams {
     uint64_t* counters;   // {entries written, chunks accepted, DTE_DEV_* bits, chunks rejected}
 };
 
+#ifdef __CUDACC__
+// Totals of one extract, once the number of changed entries is known: every counter word is
+// written (no memset of the caller's counters is needed), and lists after which no tile follows
+// end - and start - at the total.  Called by `n_threads` threads of one CTA with tid = 0 .. n_threads-1.
+__device__ __forceinline__ void gather_finish_totals(const GatherParams& p, uint64_t total, uint32_t tid,
+                                                     uint32_t n_threads) {
+    if (tid == 0) {
+        p.counters[0] = total;
+        p.counters[1] = p.scanned;
+        p.counters[2] = total > p.capacity ? (uint64_t)DTE_DEV_OVERFLOW : 0ull;
+        p.counters[3] = 0;
+        p.list_ptr[p.n_lists] = total;
+    }
+    for (uint32_t k = tid; k < p.n_lists; k += n_threads)
+        if (p.list_first_rec[k] >= p.n_rec) p.list_ptr[k] = total;
+    // where each receiver's slice starts: the output position of the first tile of its first list
+    // (block bases are final and visible to this CTA by now)
+    for (uint32_t r = tid; r < p.n_recv; r += n_threads) {
+        const uint32_t fl = p.recv_first_list[r];
+        const uint32_t fr = fl < p.n_lists ? p.list_first_rec[fl] : p.n_rec;
+        uint64_t pos = total;
+        if (fr < p.n_rec) {
+            const uint32_t b = fr / kRecsPerBlock;
+            pos = __ldcg(p.block_sum + b);
+            for (uint32_t j = b * kRecsPerBlock; j < fr; ++j) pos += __ldcg(p.rec + j) & kRecCountMask;
+        }
+        p.recv_base[r] = pos;
+    }
+}
+#endif
+
 void set_error(const std::string& msg);
 dte_status cuda_fail(cudaError_t e, const char* what);
 
@@ -210,11 +275,14 @@ dte_status cuda_fail(cudaError_t e, const char* what);
 
 dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, bool overlap,
                           cudaStream_t st);
-dte_status launch_gather(const GatherParams& p, cudaStream_t st);
+dte_status launch_gather(const GatherParams& p, bool small, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 dte_status launch_apply_canonical(const CanonParams& p, int device, cudaStream_t st);
 dte_status launch_pack_chunks(const PackParams& p, int device, cudaStream_t st);
 dte_status launch_unpack_chunks(const UnpackParams& p, int device, cudaStream_t st);
+dte_status launch_push_finish(const PushFinishParams& p, cudaStream_t st);
+dte_status launch_push_wait(const uint64_t* status, uint64_t epoch, uint32_t timeout_ms, uint64_t* counters,
+                            cudaStream_t st);
 dte_status launch_op_counts(const OpRange* ranges, uint32_t n_ops, const dte_delta& d, uint32_t n_lists,
                             uint64_t* counts, cudaStream_t st);
 
@@ -235,7 +303,8 @@ struct dte_layout {
     dte::SegRec* d_segs = nullptr;
     uint64_t* d_rec = nullptr;             // n_tiles placement records
     uint64_t* d_block_sum = nullptr;       // one word per gather block
-    uint64_t* d_cursor = nullptr;          // staging cursor
+    uint64_t* d_cursor = nullptr;          // staging cursor, then the ticket of small layouts; both rest at zero
+    bool scratch_clean = false;            // the last call was enqueued completely, so they are at zero
     uint32_t* d_stage = nullptr;           // staging buffer, grown on demand to the caller's capacity
     uint64_t* d_rec_base = nullptr;        // n_tiles: destination base per placement record
     uint64_t stage_capacity = 0;
@@ -257,6 +326,20 @@ struct dte_layout {
     uint32_t* d_src_op_ptr = nullptr;
     uint32_t* d_tensor_cols = nullptr;
     uint32_t* d_tensor_numel32 = nullptr;
+    // receivers (dte_extract_delta_push): host tables from create, device copies on first use
+    uint32_t n_receivers = 0;
+    bool recv_contiguous = true;           // every receiver's shards are consecutive in shard order
+    std::vector<uint32_t> h_recv_first_list, h_recv_num_ops, h_op_recv, h_op_slot;
+    std::vector<uint16_t> h_rec_recv;
+    uint32_t* d_recv_first_list = nullptr;
+    uint32_t* d_recv_num_ops = nullptr;
+    uint32_t* d_op_recv = nullptr;
+    uint32_t* d_op_slot = nullptr;
+    uint16_t* d_rec_recv = nullptr;
+    uint64_t* d_recv_base = nullptr;
+    dte_push_target* d_targets = nullptr;
+    std::vector<dte_push_target> h_targets;
+    bool targets_valid = false;
     // host mirrors of the pointer tables last uploaded
     std::vector<const float*> h_ptrs;
     std::vector<uint16_t*> h_shards;

@@ -98,6 +98,13 @@ extern "C" void dte_layout_destroy(dte_layout* L) {
     cudaFree(L->d_src_op_ptr);
     cudaFree(L->d_tensor_cols);
     cudaFree(L->d_tensor_numel32);
+    cudaFree(L->d_recv_first_list);
+    cudaFree(L->d_recv_num_ops);
+    cudaFree(L->d_op_recv);
+    cudaFree(L->d_op_slot);
+    cudaFree(L->d_rec_recv);
+    cudaFree(L->d_recv_base);
+    cudaFree(L->d_targets);
     if (prev >= 0) cudaSetDevice(prev);
     delete L;
 }
@@ -106,6 +113,10 @@ extern "C" size_t dte_layout_num_lists(const dte_layout* L) { return L ? L->n_li
 extern "C" uint64_t dte_layout_num_elements(const dte_layout* L) { return L ? L->scanned : 0; }
 extern "C" size_t dte_layout_num_ops(const dte_layout* L) { return L ? L->n_ops : 0; }
 extern "C" size_t dte_layout_num_groups(const dte_layout* L) { return L ? L->n_groups : 0; }
+extern "C" size_t dte_layout_num_receivers(const dte_layout* L) { return L ? L->n_receivers : 0; }
+extern "C" size_t dte_layout_receiver_num_ops(const dte_layout* L, uint32_t receiver) {
+    return (L && receiver < L->h_recv_num_ops.size()) ? L->h_recv_num_ops[receiver] : 0;
+}
 
 extern "C" uint64_t dte_layout_host_workspace_bytes(const dte_layout* L) {
     if (!L) return 0;
@@ -199,6 +210,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
 
     std::vector<TileDesc> tiles, packed;            // regular: one per tile; packed: kSub per tile
     uint32_t n_rec = 0;                             // tiles so far, in output order
+    std::vector<uint32_t> rec_list;                 // list of each tile
     std::vector<uint32_t> list_first_tile(n_shards + 1, 0);
     std::vector<SegRec> segs;
     std::vector<uint8_t> has_tiles(n_shards, 0);
@@ -219,6 +231,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         auto flush_pending = [&]() {
             if (pending.empty()) return;
             const uint32_t tile = n_rec++;
+            rec_list.push_back((uint32_t)k);
             note_tile(tile);
             TileDesc empty;
             std::memset(&empty, 0, sizeof empty);
@@ -242,6 +255,7 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
                 if (len == (uint64_t)kTile) {
                     flush_pending();
                     t.tile = n_rec++;
+                    rec_list.push_back((uint32_t)k);
                     note_tile(t.tile);
                     tiles.push_back(t);
                     return;
@@ -373,6 +387,38 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
                 L->h_src_ops[at[op.src_tensor]++] = so;
             }
     }
+    {   // receivers: who owns which list, tile and operation (used by dte_extract_delta_push only)
+        uint32_t n_recv = 0;
+        for (size_t k = 0; k < n_shards; ++k) n_recv = std::max(n_recv, shards[k].receiver + 1);
+        if (n_shards && n_recv <= 65535) {
+            L->n_receivers = n_recv;
+            // [0, n_recv): first list of each receiver; [n_recv, 2 n_recv): one past its last list
+            // (both 0 for a receiver without shards: an empty slice)
+            L->h_recv_first_list.assign(2 * (size_t)n_recv, 0u);
+            std::vector<uint32_t> count(n_recv, 0);
+            for (size_t k = n_shards; k-- > 0;) L->h_recv_first_list[shards[k].receiver] = (uint32_t)k;
+            for (size_t k = 0; k < n_shards; ++k) {
+                L->h_recv_first_list[n_recv + shards[k].receiver] = (uint32_t)k + 1;
+                count[shards[k].receiver] += 1;
+            }
+            // the slice of a receiver is contiguous in the output iff its shards are consecutive
+            for (uint32_t r = 0; r < n_recv; ++r)
+                if (count[r] && L->h_recv_first_list[n_recv + r] - L->h_recv_first_list[r] != count[r])
+                    L->recv_contiguous = false;
+            L->h_recv_num_ops.assign(n_recv, 0);
+            L->h_op_recv.resize(n_ops);
+            L->h_op_slot.resize(n_ops);
+            for (size_t o = 0; o < n_ops; ++o) {
+                const uint32_t r = shards[ops[o].dst_shard].receiver;
+                L->h_op_recv[o] = r;
+                L->h_op_slot[o] = L->h_recv_num_ops[r]++;
+            }
+            L->h_rec_recv.resize(rec_list.size());
+            for (size_t t = 0; t < rec_list.size(); ++t) L->h_rec_recv[t] = (uint16_t)shards[rec_list[t]].receiver;
+        } else {
+            L->recv_contiguous = false;
+        }
+    }
     {
         std::vector<uint32_t> grp(n_tensors);
         for (size_t p = 0; p < n_tensors; ++p) {
@@ -386,7 +432,10 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         const size_t n_blocks = (n_rec + kRecsPerBlock - 1) / kRecsPerBlock;
         cudaError_t e = cudaMalloc((void**)&L->d_rec, std::max<size_t>(1, n_rec) * sizeof(uint64_t));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_block_sum, std::max<size_t>(1, n_blocks) * sizeof(uint64_t));
-        if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_cursor, sizeof(uint64_t));
+        // cursor, extract ticket, push ticket, spare: all rest at zero
+        if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_cursor, 4 * sizeof(uint64_t));
+        if (e == cudaSuccess) e = cudaMemset(L->d_cursor, 0, 4 * sizeof(uint64_t));
+        if (e == cudaSuccess) L->scratch_clean = true;
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_groups, L->n_groups * sizeof(GroupConsts));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_ptrs, std::max<size_t>(1, 3 * n_tensors) * sizeof(void*));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_shards, std::max<size_t>(1, n_shards) * sizeof(void*));
