@@ -79,20 +79,20 @@ Screen make_screen(const Consts& c) {
 // Where one extract call keeps its placement records, block sums, staging cursor and staged
 // entries: the layout's own buffers, or the fixed array of the allocation-free entry point.
 struct Scratch {
-    uint64_t* cursor;       // two words: the staging cursor, then the ticket of small layouts
+    uint64_t* cursor;       // the staging cursor
     uint64_t* rec;
     uint64_t* block_sum;
     uint32_t* stage;
-    bool clear_first;       // the two words are not known to be zero: clear them in the stream
+    bool clear_first;       // the cursor is not known to be zero: clear it in the stream
 };
 
 // Enqueues the kernels of one extract: both extract launches (packed and regular tiles), then
-// what puts the staged entries in order - for layouts of at most kSmallBlocks gather blocks only
-// the move (the extract's last tile does the scan itself), else reduce, scan and move.  `groups`:
+// what puts the staged entries in order - one launch for layouts of at most kSmallBlocks gather
+// blocks (every block scans the records itself), else reduce, scan and move.  `groups`:
 // per-parameter-group constants (NULL: `c` applies to every tensor).  The scan writes every word
-// of out->counters, and it leaves the cursor and the ticket at zero, the only scratch words that
-// must start there (records and block sums are rewritten in full, staged entries are read only
-// where this call wrote them): an ordinary call enqueues kernels and nothing else.
+// of out->counters, and it leaves the cursor at zero, the only scratch word that must start
+// there (records and block sums are rewritten in full, staged entries are read only where this
+// call wrote them): an ordinary call enqueues kernels and nothing else.
 dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<GroupConsts>* groups,
                            const Scratch& sc, const dte_delta* out, cudaStream_t st, bool push = false) {
     if (L->n_tiles == 0) {
@@ -101,7 +101,7 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
         L->last_launch[0] = 0; L->last_launch[1] = 0; L->last_launch[2] = 0;
         return DTE_OK;
     }
-    if (sc.clear_first) DTE_CUDA(cudaMemsetAsync(sc.cursor, 0, 2 * sizeof(uint64_t), st));
+    if (sc.clear_first) DTE_CUDA(cudaMemsetAsync(sc.cursor, 0, sizeof(uint64_t), st));
     GatherParams g;
     g.rec = sc.rec;
     g.block_sum = sc.block_sum;
@@ -138,9 +138,6 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
     p.s = make_screen(c);
     p.tensor_group = nullptr;
     p.groups = nullptr;
-    p.ticket = small ? reinterpret_cast<unsigned int*>(sc.cursor + 1) : nullptr;
-    p.ticket_total = L->n_tiles;
-    p.g = g;
     bool div_bc1 = c.bc1 != 1.0f, div_decay = c.decay != 1.0f;
     if (groups) {
         // pageable source: staged by the runtime before the call returns
@@ -154,16 +151,13 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
             div_decay |= gc.c.decay != 1.0f;
         }
     }
-    // one CTA per tile; packed tiles (short runs sharing a CTA; few) first, then the full tiles,
-    // which may start while the packed launch is still running: the two share nothing but the
-    // staging cursor and the ticket (atomics) and write different placement records
-    p.tiles = L->d_packed;
-    p.n_tiles = L->n_packed;
-    dte_status s = launch_extract(p, div_bc1, div_decay, true, false, st);
-    if (s != DTE_OK) return s;
+    // one CTA per tile, packed tiles (short runs sharing a CTA; few) and full tiles: they share
+    // nothing but the staging cursor (atomic) and write different placement records
     p.tiles = L->d_tiles;
-    p.n_tiles = L->n_regular;
-    s = launch_extract(p, div_bc1, div_decay, false, L->n_packed != 0, st);
+    p.packed = L->d_packed;
+    p.n_regular = L->n_regular;
+    p.n_packed = L->n_packed;
+    dte_status s = launch_extract(p, div_bc1, div_decay, st);
     if (s != DTE_OK) return s;
     s = launch_gather(g, small, st);
     if (s != DTE_OK) return s;
@@ -186,8 +180,8 @@ dte_status enqueue_extract(dte_layout* L, const Consts& c, const dte_delta* out,
         DTE_CUDA(cudaMalloc((void**)&L->d_stage, out->capacity * sizeof(uint32_t)));
         L->stage_capacity = out->capacity;
     }
-    // The kernels leave the cursor and the ticket at zero.  If an earlier call stopped half-way
-    // (a launch failed), they may not be: clear them in the stream this once.
+    // The kernels leave the cursor at zero.  If an earlier call stopped half-way (a launch failed),
+    // it may not be: clear it in the stream this once.
     const Scratch sc{L->d_cursor, L->d_rec, L->d_block_sum, L->d_stage, !L->scratch_clean};
     L->scratch_clean = false;
     const dte_status s = enqueue_kernels(L, c, groups, sc, out, st, push);
@@ -639,8 +633,8 @@ extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const f
     s = sync_source_table(L, theta, m, v, st);
     if (s != DTE_OK) return s;
     // the array keeps whatever the previous call left - possibly a call on another layout, or one
-    // that was cut short - so the two words that must start at zero (cursor and ticket) are cleared
-    // in the stream every time; every other part is written before it is read
+    // that was cut short - so the one word that must start at zero (the cursor) is cleared in the
+    // stream every time; every other part is written before it is read
     const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
     const Scratch sc{reinterpret_cast<uint64_t*>(base + kStaticCursorOff),
                      reinterpret_cast<uint64_t*>(base + kStaticRecOff),

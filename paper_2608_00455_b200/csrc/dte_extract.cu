@@ -91,13 +91,30 @@ __device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, 
     // range) and is dropped by the |.| operand modifiers, which cost nothing
     const uint32_t u = __float_as_uint(theta);
     const float at = fabsf(theta);
-    float room;
+    // the step lr * u has the sign of lr * m (den >= +0 or NaN): sign bit of x set <=> it shrinks |theta|
+    const uint32_t x = u ^ __float_as_uint(m) ^ __float_as_uint(lr);
     if (DIV_DECAY) {
-        // the division by decay moves |theta| one way and the step possibly the other: both sides
+        // The step moves |theta| by at most S in a KNOWN direction; the division by decay then
+        // moves it by at most D = a(1+2^-7)(|1/decay - 1| + 2^-24) in either direction.  So the
+        // boundary the step moves towards must be further than S + D, the other one further than
+        // D only - a few ulps, which nearly always holds.  (Testing both sides against S + D sent
+        // about twice as many elements to the exact path.)  A step larger than the room on its
+        // side fails there, so it cannot flip the sign either.
         const uint32_t hi = ((u + 0x8000u) & 0xFFFF0000u) | 0x7FFEu;   // boundary above |theta|, minus 2 ulp
         const uint32_t lo = hi - 0xFFFCu;                               // boundary below, plus 2 ulp
-        room = min_nan(fabsf(__uint_as_float(hi)) - at, at - fabsf(__uint_as_float(lo)));   // exact differences
-    } else {
+        const float room_up = fabsf(__uint_as_float(hi)) - at;          // exact differences; NaN for theta = 0,
+        const float room_dn = at - fabsf(__uint_as_float(lo));          // Inf, NaN; a tie has room_dn < 0
+        const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
+        const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);   // -Inf for v = -0 or a negative subnormal
+        const float sa = fabsf(__fmul_rn(__fmul_rn(am, w), fabsf(lr))); // |.|: a negative v must not pass
+        const float d_only = __fmul_rn(at, s.kappa);
+        const float s_and_d = __fmaf_rn(at, s.kappa, sa);
+        const bool down = (int32_t)x < 0;
+        // ordered, strict compares: NaN anywhere fails, and an infinite bound never passes
+        return (down ? d_only : s_and_d) < room_up && (down ? s_and_d : d_only) < room_dn;
+    }
+    float room;
+    {
         // Without it the reconstruction is RN(theta + lr * u) and u has the sign of m (den >= +0 or
         // NaN), so the direction is known: |theta| grows when theta and lr * m agree in sign and
         // shrinks otherwise, and only the boundary on that side matters.  This halves the elements
@@ -105,7 +122,6 @@ __device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, 
         // cannot change the pattern).  A theta exactly on a tie point belongs to the cell above or
         // below it depending on parity; each direction takes the cell that has the tie as its
         // boundary on that side, so a tie never passes.
-        const uint32_t x = u ^ __float_as_uint(m) ^ __float_as_uint(lr);   // sign bit set: shrinks
         const bool down = (int32_t)x < 0;
         const uint32_t cell = (u + (down ? 0x8000u : 0x7FFFu)) & 0xFFFF0000u;
         const uint32_t bnd = down ? cell - 0x7FFEu : cell + 0x7FFEu;       // 2 ulp inside the boundary
@@ -114,8 +130,7 @@ __device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, 
     }
     const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
     const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);   // -Inf for v = -0 or a negative subnormal
-    float b = __fmul_rn(__fmul_rn(am, w), fabsf(lr));
-    if (DIV_DECAY) b = __fmaf_rn(at, s.kappa, b);
+    const float b = __fmul_rn(__fmul_rn(am, w), fabsf(lr));
     // |b|: a negative v (w = -Inf or NaN) must not pass.  Strict: theta = +-Inf has room = +Inf on
     // its lower side, and an infinite bound (the step may be -Inf, the sum NaN) must not pass it.
     return fabsf(b) < room;
@@ -158,10 +173,10 @@ struct WarpTile {
 // the CTA shares one (its address depends on blockIdx only: uniform registers) and warp w
 // takes the w-th kWarpTile slots of it.
 template <bool PACKED>
-__device__ __forceinline__ uint32_t decode(const ExtractParams& p, int lane, int warp, StridedGeom* geom,
-                                           WarpTile& wt, uint32_t& tile) {
-    const uint4* td = reinterpret_cast<const uint4*>(PACKED ? p.tiles + ((size_t)blockIdx.x * kSub + warp)
-                                                            : p.tiles + blockIdx.x);
+__device__ __forceinline__ uint32_t decode(const ExtractParams& p, uint32_t index, int lane, int warp,
+                                           StridedGeom* geom, WarpTile& wt, uint32_t& tile) {
+    const uint4* td = reinterpret_cast<const uint4*>(PACKED ? p.packed + ((size_t)index * kSub + warp)
+                                                            : p.tiles + index);
     const uint4 d0 = __ldg(td), d1 = __ldg(td + 1);
     const uint32_t e0 = PACKED ? 0u : (uint32_t)warp * kWarpTile;
     const uint32_t run_len = d1.x & kLenMask;
@@ -307,54 +322,13 @@ __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint3
     return qn;
 }
 
-// The tail of a small layout's extract: the CTA that finishes last (all launches of the call
-// counted) turns the placement records into the gather's block bases, the totals and the
-// boundaries of trailing empty lists - what gather_reduce and gather_scan do for large layouts -
-// and leaves the cursor and the ticket at zero for the next call.  Nobody waits for anybody.
-__device__ void finish_small(const ExtractParams& p, uint64_t* s_bsum) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const GatherParams& g = p.g;
-    for (uint32_t b = warp; b < g.n_blocks; b += kWarps) {
-        uint32_t sum = 0;
-        for (uint32_t j = lane; j < (uint32_t)kRecsPerBlock; j += 32) {
-            const uint32_t r = b * kRecsPerBlock + j;
-            if (r < g.n_rec) sum += (uint32_t)(__ldcg(g.rec + r) & kRecCountMask);   // written by other SMs: L2
-        }
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, d);
-        if (lane == 0) s_bsum[b] = sum;
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint64_t run = 0;
-        for (uint32_t b = 0; b < g.n_blocks; ++b) {
-            g.block_sum[b] = run;
-            run += s_bsum[b];
-        }
-        s_bsum[kSmallBlocks] = run;
-        *p.cursor = 0ull;
-        *p.ticket = 0u;
-    }
-    __syncthreads();
-    gather_finish_totals(g, s_bsum[kSmallBlocks], threadIdx.x, kThreads);
-}
-
-// GROUPS: the constants come from the tile's parameter group instead of the kernel parameters.
-template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED>
-__global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const ExtractParams p) {
-    // Programmatic dependent launch.  The packed-tile launch of a call goes first and lets the
-    // regular-tile launch start at once: the two share nothing but the atomic staging cursor.  The
-    // regular-tile launch gives the signal late, so that what follows it (the gather of a small
-    // layout, launched the same way) is set up while the last tiles finish and does not sit on
-    // the SMs before.  A no-op when the next launch in the stream did not ask for it.
-    if (PACKED) asm volatile("griddepcontrol.launch_dependents;");
-    // per warp: queue of element indices awaiting exact evaluation, later (index | value << 16)
-    // (dynamic shared memory: kWarps * kWarpTile words, may exceed the 48 KB static limit)
-    extern __shared__ __align__(16) uint32_t s_queue[];
-    __shared__ uint32_t s_count[kWarps];
-    __shared__ unsigned long long s_pos;
-    __shared__ StridedGeom s_geom[kWarps];
-    __shared__ uint32_t s_last;
+// One tile: `index` counts within the tiles of its kind.  GROUPS: the constants come from the
+// tile's parameter group instead of the kernel parameters.  EARLY: give the dependent-launch
+// signal at once instead of after the stream (see the kernels below).
+template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED, bool EARLY>
+__device__ __forceinline__ void extract_tile(const ExtractParams& p, uint32_t index, uint32_t* s_queue,
+                                             uint32_t* s_count, unsigned long long& s_pos, StridedGeom* s_geom) {
+    if (EARLY) asm volatile("griddepcontrol.launch_dependents;");
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     uint32_t* queue = s_queue + warp * kWarpTile;
     Consts c = p.c;
@@ -365,7 +339,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
     WarpTile cur;
     uint32_t tile;
     {
-        const uint32_t tensor = decode<PACKED>(p, lane, warp, &s_geom[warp], cur, tile);
+        const uint32_t tensor = decode<PACKED>(p, index, lane, warp, &s_geom[warp], cur, tile);
         if (GROUPS) {   // one 48-byte record per parameter group
             const uint4* gp = reinterpret_cast<const uint4*>(p.groups + __ldg(p.tensor_group + tensor));
             const uint4 g0 = __ldg(gp), g1 = __ldg(gp + 1), g2 = __ldg(gp + 2);
@@ -386,7 +360,7 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
         else
             qn = phase_a<DIV_BC1, DIV_DECAY, false>(cur, lane, queue, sc, lr);
         __syncwarp();
-        if (!PACKED) asm volatile("griddepcontrol.launch_dependents;");
+        if (!EARLY) asm volatile("griddepcontrol.launch_dependents;");
 
         // ---- phase B: exact evaluation of the queue, 32 entries per round; the changed
         //      entries are compacted to the front of the queue as (index | value << 16) -----
@@ -444,10 +418,6 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
             if (total) pos0 = atomicAdd(p.cursor, (unsigned long long)total);
             s_pos = pos0;
             p.rec[tile] = ((uint64_t)pos0 << kRecCountBits) | total;
-            if (p.ticket) {       // small layout: is this the last tile of the call to finish?
-                __threadfence();
-                s_last = atomicAdd(p.ticket, 1u) == p.ticket_total - 1u;
-            }
         }
         __syncthreads();
         const unsigned long long pos = s_pos + before;
@@ -456,11 +426,27 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
             if (pos + q < p.stage_capacity)               // beyond it the call overflows anyway
                 p.stage[pos + q] = queue[q] + rel;
     }
-    if (p.ticket && s_last) {
-        __syncthreads();                                   // the queues are free now
-        __threadfence();
-        finish_small(p, reinterpret_cast<uint64_t*>(s_queue));
-    }
+}
+
+// Shared memory of a CTA: per warp the queue of element indices awaiting exact evaluation, later
+// (index | value << 16) - dynamic, kWarps * kWarpTile words, may exceed the 48 KB static limit.
+#define DTE_EXTRACT_SHARED                              \
+    extern __shared__ __align__(16) uint32_t s_queue[]; \
+    __shared__ uint32_t s_count[kWarps];                \
+    __shared__ unsigned long long s_pos;                \
+    __shared__ StridedGeom s_geom[kWarps]
+
+// One launch per kind of tile.  The packed-tile launch (few CTAs, each a serial chain of short
+// runs) goes first and lets the regular-tile launch start at once (programmatic dependent
+// launch): the two share nothing but the atomic staging cursor.  The regular-tile launch keeps
+// its descriptor address a function of blockIdx alone (uniform registers; one kernel with a
+// branch for both kinds of tile ran the regular tiles 15 % slower).  It gives its own signal
+// after the stream, so that the gather of a small layout, launched the same way, is set up while
+// the last tiles finish and does not sit on the SMs before.
+template <bool DIV_BC1, bool DIV_DECAY, bool GROUPS, bool PACKED>
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const ExtractParams p) {
+    DTE_EXTRACT_SHARED;
+    extract_tile<DIV_BC1, DIV_DECAY, GROUPS, PACKED, PACKED>(p, blockIdx.x, s_queue, s_count, s_pos, s_geom);
     // The launch of the regular tiles may have begun before the launch of the packed tiles ended.
     // What follows in the stream (the gather) is ordered after THIS grid only, so this grid must
     // not complete before the one it overlapped: wait for it here, where nothing is left to do.
@@ -470,23 +456,23 @@ __global__ void __launch_bounds__(kThreads, kMinCtasPerSm) extract_kernel(const 
 
 constexpr size_t kQueueBytes = (size_t)kWarps * kWarpTile * sizeof(uint32_t);
 
-// `overlap`: the launch may begin before the previous kernel in the stream has finished (it must
-// not depend on that kernel's results).
-template <bool A, bool B, bool G, bool P>
-static dte_status launch_t(const ExtractParams& p, bool overlap, cudaStream_t st) {
-    // per device, once: allow more than 48 KB of dynamic shared memory.  Host threads may race
-    // here (two layouts on two threads); setting the attribute twice is harmless, so an atomic
-    // flag per device is enough.
-    static std::atomic<bool> configured[kMaxDevices];
+// Per device, once: allow more than 48 KB of dynamic shared memory.  Host threads may race here
+// (two layouts on two threads); setting the attribute twice is harmless, so an atomic flag per
+// device and kernel is enough.
+template <class K>
+static dte_status allow_queue_memory(K kernel, std::atomic<bool>* configured) {
     int dev = 0;
     DTE_CUDA(cudaGetDevice(&dev));
     if (dev < 0 || dev >= kMaxDevices || !configured[dev].load(std::memory_order_acquire)) {
-        DTE_CUDA(cudaFuncSetAttribute(extract_kernel<A, B, G, P>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                      (int)kQueueBytes));
+        DTE_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kQueueBytes));
         if (dev >= 0 && dev < kMaxDevices) configured[dev].store(true, std::memory_order_release);
     }
+    return DTE_OK;
+}
+
+static dte_status launch_on(const void* kernel, const ExtractParams& p, uint32_t grid, bool overlap, cudaStream_t st) {
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(p.n_tiles);
+    cfg.gridDim = dim3(grid);
     cfg.blockDim = dim3(kThreads);
     cfg.dynamicSmemBytes = kQueueBytes;
     cfg.stream = st;
@@ -494,32 +480,43 @@ static dte_status launch_t(const ExtractParams& p, bool overlap, cudaStream_t st
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = overlap ? 1 : 0;
-    DTE_CUDA(cudaLaunchKernelEx(&cfg, extract_kernel<A, B, G, P>, p));
+    cfg.numAttrs = overlap ? 1 : 0;      // may begin before the previous kernel in the stream has finished
+    void* args[] = {const_cast<ExtractParams*>(&p)};
+    DTE_CUDA(cudaLaunchKernelExC(&cfg, kernel, args));
     return DTE_OK;
 }
 
+// One call's extract launches: the packed tiles first, the regular tiles overlapping them.
 template <bool A, bool B, bool G>
-static dte_status launch_p(const ExtractParams& p, bool packed, bool overlap, cudaStream_t st) {
-    return packed ? launch_t<A, B, G, true>(p, overlap, st) : launch_t<A, B, G, false>(p, overlap, st);
+static dte_status launch_t(const ExtractParams& p, cudaStream_t st) {
+    static std::atomic<bool> cfg_packed[kMaxDevices], cfg_regular[kMaxDevices];
+    if (p.n_packed) {
+        dte_status s = allow_queue_memory(extract_kernel<A, B, G, true>, cfg_packed);
+        if (s == DTE_OK) s = launch_on((const void*)extract_kernel<A, B, G, true>, p, p.n_packed, false, st);
+        if (s != DTE_OK) return s;
+    }
+    if (p.n_regular) {
+        dte_status s = allow_queue_memory(extract_kernel<A, B, G, false>, cfg_regular);
+        if (s == DTE_OK) s = launch_on((const void*)extract_kernel<A, B, G, false>, p, p.n_regular, p.n_packed != 0, st);
+        if (s != DTE_OK) return s;
+    }
+    return DTE_OK;
 }
 
 // div_bc1 / div_decay: whether any group in the call has a divisor different from 1.0f.
-// One launch covers p.n_tiles tiles of one kind (p.tiles = their descriptors).
-dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, bool overlap,
-                          cudaStream_t st) {
-    if (p.n_tiles == 0) return DTE_OK;
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, cudaStream_t st) {
+    if (p.n_packed + p.n_regular == 0) return DTE_OK;
     const bool a = div_bc1, b = div_decay;
     if (p.groups) {
-        if (a && b) return launch_p<true, true, true>(p, packed, overlap, st);
-        if (a) return launch_p<true, false, true>(p, packed, overlap, st);
-        if (b) return launch_p<false, true, true>(p, packed, overlap, st);
-        return launch_p<false, false, true>(p, packed, overlap, st);
+        if (a && b) return launch_t<true, true, true>(p, st);
+        if (a) return launch_t<true, false, true>(p, st);
+        if (b) return launch_t<false, true, true>(p, st);
+        return launch_t<false, false, true>(p, st);
     }
-    if (a && b) return launch_p<true, true, false>(p, packed, overlap, st);
-    if (a) return launch_p<true, false, false>(p, packed, overlap, st);
-    if (b) return launch_p<false, true, false>(p, packed, overlap, st);
-    return launch_p<false, false, false>(p, packed, overlap, st);
+    if (a && b) return launch_t<true, true, false>(p, st);
+    if (a) return launch_t<true, false, false>(p, st);
+    if (b) return launch_t<false, true, false>(p, st);
+    return launch_t<false, false, false>(p, st);
 }
 
 }  // namespace dte

@@ -1,8 +1,8 @@
 // Ordered placement of the staged entries ("count, then write"): a scan over the
 // per-tile placement records gives every tile its position in the concatenated,
 // list-ordered output (lists in shard order, ascending offsets within a list), and a gather
-// moves its entries from the staging buffer to that position.  Three small launches (for small
-// layouts the extract's last tile does the first two steps itself and only the move is launched);
+// moves its entries from the staging buffer to that position.  Three small launches (one for small
+// layouts, whose blocks each scan all records themselves);
 // the data they touch are the records (8 bytes per 9216 scanned elements) and the changed
 // entries themselves.  No kernel waits on another CTA.
 #include <algorithm>
@@ -72,19 +72,61 @@ __global__ void __launch_bounds__(kScanThreads) gather_scan_kernel(const GatherP
         if (threadIdx.x == kScanThreads - 1) s_carry = excl + x;
         __syncthreads();
     }
-    gather_finish_totals(p, s_carry, threadIdx.x, kScanThreads);
+    gather_finish_totals(p, s_carry, threadIdx.x, kScanThreads, true);
     if (threadIdx.x == 0) *p.cursor = 0ull;     // every tile has reserved its room: ready for the next call
 }
 
 // ---- 3. per block: local scan, list starts, gather ---------------------------------------------
 // PUSH: every entry is also stored into the landing buffers of the receiver that owns its list
 // (dte_extract_delta_push): plain stores to memory that may be a peer GPU's.
-template <bool PUSH>
-__global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kernel(const GatherParams p) {
-    // Small layouts launch this kernel so that it may be set up while the last extract tiles still
-    // run (programmatic dependent launch): nothing the extract wrote may be read before this.
-    // Returns at once in an ordinary launch.
+// SMALL (at most kSmallBlocks blocks, i.e. 4096 tiles): the only gather launch of the call.  Every
+// block scans ALL placement records itself (32 KB from L2 at most, cheaper than two more launches
+// in front of a 30 microsecond stream), so it knows its output base, the total and where each
+// receiver's slice starts without help; the last block also writes the totals and puts the
+// staging cursor back to zero.
+constexpr int kSmallRecs = kSmallBlocks * kRecsPerBlock;     // 4096
+constexpr int kSmallPerThread = kSmallRecs / kGatherThreads; // 16
+
+template <bool PUSH, bool SMALL>
+__global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const GatherParams p) {
+    // A small layout's gather is launched so that it may be set up while the last extract tiles
+    // still run (programmatic dependent launch): nothing the extract wrote may be read before
+    // this.  Returns at once in an ordinary launch.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    __shared__ uint32_t s_all[SMALL ? kSmallRecs + 1 : 1];      // exclusive prefix of the counts of all records
+    // the block's own records (threads 0 .. kRecsPerBlock-1 own one each): asked for first, so that
+    // a small layout's scan of all records below does not stand between the request and its use
+    uint64_t own_rec = 0;
+    if (threadIdx.x < kRecsPerBlock && blockIdx.x * kRecsPerBlock + threadIdx.x < p.n_rec)
+        own_rec = __ldcg(p.rec + blockIdx.x * kRecsPerBlock + threadIdx.x);
+    if (SMALL) {
+        __shared__ uint32_t s_thread_sum[kGatherThreads / 32];
+        uint32_t c[kSmallPerThread];
+        const uint32_t r0 = threadIdx.x * kSmallPerThread;
+#pragma unroll
+        for (int i = 0; i < kSmallPerThread; ++i)                 // independent loads; the records come from other SMs: L2
+            c[i] = r0 + i < p.n_rec ? (uint32_t)(__ldcg(p.rec + r0 + i) & kRecCountMask) : 0u;
+        uint32_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < kSmallPerThread; ++i) mine += c[i];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t up = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if ((threadIdx.x & 31) >= d) incl += up;
+        }
+        if ((threadIdx.x & 31) == 31) s_thread_sum[threadIdx.x >> 5] = incl;
+        __syncthreads();
+        uint32_t run = incl - mine;
+        for (int w = 0; w < (int)(threadIdx.x >> 5); ++w) run += s_thread_sum[w];
+#pragma unroll
+        for (int i = 0; i < kSmallPerThread; ++i) {
+            s_all[r0 + i] = run;
+            run += c[i];
+        }
+        if (threadIdx.x == kGatherThreads - 1) s_all[kSmallRecs] = run;
+        __syncthreads();
+    }
     __shared__ uint32_t s_prefix[kRecsPerBlock + 1];   // exclusive prefix of counts within the block
     __shared__ uint64_t s_pos[kRecsPerBlock];          // staging position of each record
     __shared__ uint32_t s_warp[kGatherThreads / 32];
@@ -96,10 +138,8 @@ __global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kern
     static_assert(kRecsPerBlock == 64, "two warps scan the block's records");
     uint32_t cnt = 0;
     if (tid < kRecsPerBlock) {
-        uint64_t r = 0;
-        if ((uint32_t)tid < n_here) r = p.rec[base_rec + tid];
-        cnt = (uint32_t)(r & kRecCountMask);
-        s_pos[tid] = r >> kRecCountBits;
+        cnt = (uint32_t)(own_rec & kRecCountMask);
+        s_pos[tid] = own_rec >> kRecCountBits;
     }
     uint32_t incl = cnt;
 #pragma unroll
@@ -116,7 +156,12 @@ __global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kern
     }
     __syncthreads();
     const uint32_t block_total = s_prefix[kRecsPerBlock];
-    const uint64_t out_base = p.block_sum[blockIdx.x];
+    const uint64_t out_base = SMALL ? (uint64_t)s_all[base_rec] : p.block_sum[blockIdx.x];
+    const uint64_t total = SMALL ? (uint64_t)s_all[kSmallRecs] : p.counters[0];
+    if (SMALL && blockIdx.x == gridDim.x - 1) {
+        gather_finish_totals(p, total, threadIdx.x, kGatherThreads, false);
+        if (threadIdx.x == 0) *p.cursor = 0ull;     // every tile has reserved its room: ready for the next call
+    }
 
     // list starts that fall into this block (list_first_rec is non-decreasing)
     {
@@ -133,7 +178,6 @@ __global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kern
     }
 
     // the staged entries are complete only if everything fitted
-    const uint64_t total = p.counters[0];
     if (total > p.capacity) return;
     // warp w moves records 8w .. 8w+7; the eight copies are interleaved so that eight
     // independent loads per lane are in flight (a record holds ~125 entries: few rounds)
@@ -142,10 +186,34 @@ __global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kern
     const uint32_t* src8[kRecsPerWarp];
     uint32_t* off8[kRecsPerWarp];
     uint16_t* val8[kRecsPerWarp];
-    // PUSH: the same run in the receiver's buffers, cut where the receiver's capacity ends
-    uint32_t* roff8[kRecsPerWarp];
-    uint16_t* rval8[kRecsPerWarp];
-    uint32_t rcnt8[kRecsPerWarp];
+    // PUSH: the same run in the receiver's buffers, cut where the receiver's capacity ends; kept in
+    // shared memory (one set per record, written by the record's thread) to spare registers
+    __shared__ uint32_t* s_roff[PUSH ? kRecsPerBlock : 1];
+    __shared__ uint16_t* s_rval[PUSH ? kRecsPerBlock : 1];
+    __shared__ uint32_t s_rcnt[PUSH ? kRecsPerBlock : 1];
+    if (PUSH) {
+        if (tid < kRecsPerBlock) {
+            uint32_t n = 0;
+            uint32_t* ro = nullptr;
+            uint16_t* rv = nullptr;
+            const uint32_t c = s_prefix[tid + 1] - s_prefix[tid];
+            if (c) {
+                const uint32_t recv = p.rec_recv[base_rec + tid];
+                const dte_push_target t = p.targets[recv];
+                // where the receiver's slice starts: the output position of the first tile of its first list
+                const uint64_t slice0 = SMALL ? (uint64_t)s_all[p.list_first_rec[p.recv_first_list[recv]]]
+                                              : p.recv_base[recv];
+                const uint64_t at = out_base + s_prefix[tid] - slice0;          // position in the receiver's slice
+                if (t.status && at < t.capacity) {
+                    n = (uint32_t)min((uint64_t)c, t.capacity - at);
+                    ro = t.offsets + at;
+                    rv = t.values + at;
+                }
+            }
+            s_rcnt[tid] = n; s_roff[tid] = ro; s_rval[tid] = rv;
+        }
+        __syncthreads();
+    }
     uint32_t longest = 0, packed_recs = 0;
 #pragma unroll
     for (int r = 0; r < kRecsPerWarp; ++r) {
@@ -159,21 +227,6 @@ __global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kern
         base8[r] = (uint32_t)b;
         if (b & kRecBasePacked) packed_recs |= 1u << r;
         longest = max(longest, cnt8[r]);
-        if (PUSH) {
-            rcnt8[r] = 0;
-            roff8[r] = nullptr;
-            rval8[r] = nullptr;
-            if (cnt8[r]) {
-                const uint32_t recv = p.rec_recv[base_rec + j];
-                const dte_push_target t = p.targets[recv];
-                const uint64_t at = out_base + first - p.recv_base[recv];     // position in the receiver's slice
-                if (t.status && at < t.capacity) {
-                    rcnt8[r] = (uint32_t)min((uint64_t)cnt8[r], t.capacity - at);
-                    roff8[r] = t.offsets + at;
-                    rval8[r] = t.values + at;
-                }
-            }
-        }
     }
     for (uint32_t q = lane; q < longest; q += 32) {
         uint32_t w[kRecsPerWarp];
@@ -188,9 +241,9 @@ __global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kern
                 const uint32_t off = base8[r] + (w[r] & 0xFFFFu);
                 off8[r][q] = off;
                 val8[r][q] = (uint16_t)(w[r] >> 16);
-                if (PUSH && q < rcnt8[r]) {
-                    roff8[r][q] = off;
-                    rval8[r][q] = (uint16_t)(w[r] >> 16);
+                if (PUSH && q < s_rcnt[warp * kRecsPerWarp + r]) {
+                    s_roff[warp * kRecsPerWarp + r][q] = off;
+                    s_rval[warp * kRecsPerWarp + r][q] = (uint16_t)(w[r] >> 16);
                 }
             }
     }
@@ -205,7 +258,7 @@ __global__ void __launch_bounds__(kGatherThreads, PUSH ? 2 : 3) gather_move_kern
                 const uint32_t piece = idx / kWarpTile;
                 const uint32_t off = __ldg(&d[piece].dst_off) + (idx - piece * kWarpTile);
                 off8[r][q] = off;
-                if (PUSH && q < rcnt8[r]) roff8[r][q] = off;
+                if (PUSH && q < s_rcnt[warp * kRecsPerWarp + r]) s_roff[warp * kRecsPerWarp + r][q] = off;
             }
         }
     }
@@ -314,8 +367,7 @@ dte_status launch_push_wait(const uint64_t* status, uint64_t epoch, uint32_t tim
     return DTE_OK;
 }
 
-// small: the extract's last tile has done the scan already (finish_small in dte_extract.cu); only
-// the move is left, launched so that it can be set up under the extract's tail.
+// small: one launch (every block scans the records itself), set up under the extract's tail.
 dte_status launch_gather(const GatherParams& p, bool small, cudaStream_t st) {
     if (small) {
         cudaLaunchConfig_t cfg = {};
@@ -327,16 +379,16 @@ dte_status launch_gather(const GatherParams& p, bool small, cudaStream_t st) {
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = 1;
-        if (p.n_recv) DTE_CUDA(cudaLaunchKernelEx(&cfg, gather_move_kernel<true>, p));
-        else DTE_CUDA(cudaLaunchKernelEx(&cfg, gather_move_kernel<false>, p));
+        if (p.n_recv) DTE_CUDA(cudaLaunchKernelEx(&cfg, gather_move_kernel<true, true>, p));
+        else DTE_CUDA(cudaLaunchKernelEx(&cfg, gather_move_kernel<false, true>, p));
         return DTE_OK;
     }
     gather_reduce_kernel<<<p.n_blocks, kGatherThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     gather_scan_kernel<<<1, kScanThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
-    if (p.n_recv) gather_move_kernel<true><<<p.n_blocks, kGatherThreads, 0, st>>>(p);
-    else gather_move_kernel<false><<<p.n_blocks, kGatherThreads, 0, st>>>(p);
+    if (p.n_recv) gather_move_kernel<true, false><<<p.n_blocks, kGatherThreads, 0, st>>>(p);
+    else gather_move_kernel<false, false><<<p.n_blocks, kGatherThreads, 0, st>>>(p);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }

@@ -69,7 +69,7 @@ struct SegRec {
 constexpr int kRecCountBits = 14;                      // count <= kTile
 constexpr uint64_t kRecCountMask = (1ull << kRecCountBits) - 1;
 constexpr int kRecsPerBlock = 64;                      // records one gather CTA handles
-constexpr int kSmallBlocks = 64;                       // layouts up to this many gather blocks take the short path
+constexpr int kSmallBlocks = 64;                       // layouts up to this many gather blocks: one gather launch
 // A staged entry is one 32-bit word: (warp * kWarpTile + element index in the warp-tile) in the low
 // 16 bits, the BF16 value in the high 16.  The gather turns it into (offset, value) with the tile's
 // destination base: rec_base[r] = dst_off of a regular tile, or kRecBasePacked | index of a packed
@@ -119,7 +119,9 @@ struct GatherParams {
 };
 
 struct ExtractParams {
-    const TileDesc* tiles;       // regular tiles: one descriptor each; packed tiles: kSub each
+    const TileDesc* tiles;       // regular tiles: one descriptor each
+    const TileDesc* packed;      // packed tiles: kSub descriptors each
+    uint32_t n_regular, n_packed;
     const SegRec* segs;
     const float* const* theta;   // device table, n_tensors
     const float* const* m;
@@ -128,16 +130,10 @@ struct ExtractParams {
     uint64_t* rec;               // n_tiles placement records (written in full)
     uint32_t* stage;             // staging buffer, stage_capacity words: tile-relative index | value << 16
     uint64_t stage_capacity;
-    uint32_t n_tiles;            // tiles handled by this launch
     Consts c;                    // single-group calls: constants in the kernel parameters
     Screen s;
     const uint32_t* tensor_group;   // per-group calls: group of each source tensor ...
     const GroupConsts* groups;      // ... and the constants of each group (NULL otherwise)
-    // small layouts (at most kSmallBlocks gather blocks): the tile that finishes last, counted over
-    // all launches of the call on `ticket`, does the scan itself (see finish_small); NULL otherwise
-    unsigned int* ticket;
-    uint32_t ticket_total;
-    GatherParams g;
 };
 
 
@@ -238,7 +234,7 @@ struct UnpackParams {
 // written (no memset of the caller's counters is needed), and lists after which no tile follows
 // end - and start - at the total.  Called by `n_threads` threads of one CTA with tid = 0 .. n_threads-1.
 __device__ __forceinline__ void gather_finish_totals(const GatherParams& p, uint64_t total, uint32_t tid,
-                                                     uint32_t n_threads) {
+                                                     uint32_t n_threads, bool with_recv_base) {
     if (tid == 0) {
         p.counters[0] = total;
         p.counters[1] = p.scanned;
@@ -250,7 +246,7 @@ __device__ __forceinline__ void gather_finish_totals(const GatherParams& p, uint
         if (p.list_first_rec[k] >= p.n_rec) p.list_ptr[k] = total;
     // where each receiver's slice starts: the output position of the first tile of its first list
     // (block bases are final and visible to this CTA by now)
-    for (uint32_t r = tid; r < p.n_recv; r += n_threads) {
+    for (uint32_t r = tid; with_recv_base && r < p.n_recv; r += n_threads) {
         const uint32_t fl = p.recv_first_list[r];
         const uint32_t fr = fl < p.n_lists ? p.list_first_rec[fl] : p.n_rec;
         uint64_t pos = total;
@@ -273,8 +269,7 @@ dte_status cuda_fail(cudaError_t e, const char* what);
         if (e__ != cudaSuccess) return dte::cuda_fail(e__, #call); \
     } while (0)
 
-dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, bool packed, bool overlap,
-                          cudaStream_t st);
+dte_status launch_extract(const ExtractParams& p, bool div_bc1, bool div_decay, cudaStream_t st);
 dte_status launch_gather(const GatherParams& p, bool small, cudaStream_t st);
 dte_status launch_apply(const ApplyParams& p, int device, cudaStream_t st);
 dte_status launch_apply_canonical(const CanonParams& p, int device, cudaStream_t st);
@@ -303,7 +298,7 @@ struct dte_layout {
     dte::SegRec* d_segs = nullptr;
     uint64_t* d_rec = nullptr;             // n_tiles placement records
     uint64_t* d_block_sum = nullptr;       // one word per gather block
-    uint64_t* d_cursor = nullptr;          // staging cursor, then the ticket of small layouts; both rest at zero
+    uint64_t* d_cursor = nullptr;          // staging cursor (rests at zero), a spare word, the ticket of the push's closing kernel
     bool scratch_clean = false;            // the last call was enqueued completely, so they are at zero
     uint32_t* d_stage = nullptr;           // staging buffer, grown on demand to the caller's capacity
     uint64_t* d_rec_base = nullptr;        // n_tiles: destination base per placement record
