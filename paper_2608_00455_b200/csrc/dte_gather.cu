@@ -179,13 +179,15 @@ __global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const Ga
 
     // the staged entries are complete only if everything fitted
     if (total > p.capacity) return;
-    // warp w moves records 8w .. 8w+7; the eight copies are interleaved so that eight
-    // independent loads per lane are in flight (a record holds ~125 entries: few rounds)
+    // warp w moves records 8w .. 8w+7; the eight copies are interleaved, two rounds at a time, so
+    // that sixteen independent loads per lane are in flight (the kernel is bound by memory
+    // latency: a block holds only 64 records, and a one-layer workload has a few hundred blocks).
+    // Output positions are kept as 32-bit distances from the block's base to spare registers.
     (void)block_total;
-    uint32_t cnt8[kRecsPerWarp], base8[kRecsPerWarp];
+    uint32_t cnt8[kRecsPerWarp], base8[kRecsPerWarp], first8[kRecsPerWarp];
     const uint32_t* src8[kRecsPerWarp];
-    uint32_t* off8[kRecsPerWarp];
-    uint16_t* val8[kRecsPerWarp];
+    uint32_t* const out_off = p.offsets + out_base;
+    uint16_t* const out_val = p.values + out_base;
     // PUSH: the same run in the receiver's buffers, cut where the receiver's capacity ends; kept in
     // shared memory (one set per record, written by the record's thread) to spare registers
     __shared__ uint32_t* s_roff[PUSH ? kRecsPerBlock : 1];
@@ -218,32 +220,36 @@ __global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const Ga
 #pragma unroll
     for (int r = 0; r < kRecsPerWarp; ++r) {
         const uint32_t j = warp * kRecsPerWarp + r;
-        const uint32_t first = s_prefix[j];
-        cnt8[r] = s_prefix[j + 1] - first;
+        first8[r] = s_prefix[j];
+        cnt8[r] = s_prefix[j + 1] - first8[r];
         src8[r] = p.stage + s_pos[j];
-        off8[r] = p.offsets + (out_base + first);
-        val8[r] = p.values + (out_base + first);
         const uint64_t b = cnt8[r] ? p.rec_base[base_rec + j] : 0ull;
         base8[r] = (uint32_t)b;
         if (b & kRecBasePacked) packed_recs |= 1u << r;
         longest = max(longest, cnt8[r]);
     }
-    for (uint32_t q = lane; q < longest; q += 32) {
-        uint32_t w[kRecsPerWarp];
+    for (uint32_t q0 = lane; q0 < longest; q0 += 64) {
+        uint32_t w[2][kRecsPerWarp];
 #pragma unroll
-        for (int r = 0; r < kRecsPerWarp; ++r)
-            if (q < cnt8[r]) w[r] = src8[r][q];
+        for (int h = 0; h < 2; ++h)
 #pragma unroll
-        for (int r = 0; r < kRecsPerWarp; ++r)
-            if (q < cnt8[r]) {
-                // a regular tile is one destination run: base + (warp * kWarpTile + index); the
-                // offsets of packed tiles are put right below
-                const uint32_t off = base8[r] + (w[r] & 0xFFFFu);
-                off8[r][q] = off;
-                val8[r][q] = (uint16_t)(w[r] >> 16);
-                if (PUSH && q < s_rcnt[warp * kRecsPerWarp + r]) {
-                    s_roff[warp * kRecsPerWarp + r][q] = off;
-                    s_rval[warp * kRecsPerWarp + r][q] = (uint16_t)(w[r] >> 16);
+            for (int r = 0; r < kRecsPerWarp; ++r)
+                if (q0 + 32 * h < cnt8[r]) w[h][r] = src8[r][q0 + 32 * h];
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int r = 0; r < kRecsPerWarp; ++r) {
+                const uint32_t q = q0 + 32 * h;
+                if (q < cnt8[r]) {
+                    // a regular tile is one destination run: base + (warp * kWarpTile + index); the
+                    // offsets of packed tiles are put right below
+                    const uint32_t off = base8[r] + (w[h][r] & 0xFFFFu);
+                    out_off[first8[r] + q] = off;
+                    out_val[first8[r] + q] = (uint16_t)(w[h][r] >> 16);
+                    if (PUSH && q < s_rcnt[warp * kRecsPerWarp + r]) {
+                        s_roff[warp * kRecsPerWarp + r][q] = off;
+                        s_rval[warp * kRecsPerWarp + r][q] = (uint16_t)(w[h][r] >> 16);
+                    }
                 }
             }
     }
@@ -257,7 +263,7 @@ __global__ void __launch_bounds__(kGatherThreads, 3) gather_move_kernel(const Ga
                 const uint32_t idx = src8[r][q] & 0xFFFFu;
                 const uint32_t piece = idx / kWarpTile;
                 const uint32_t off = __ldg(&d[piece].dst_off) + (idx - piece * kWarpTile);
-                off8[r][q] = off;
+                out_off[first8[r] + q] = off;
                 if (PUSH && q < s_rcnt[warp * kRecsPerWarp + r]) s_roff[warp * kRecsPerWarp + r][q] = off;
             }
         }
