@@ -489,6 +489,43 @@ def time_storage_path(dte, wl, st, shards, hp, capacity, device, peak, chunk_ent
             "gpu_launches": (5 + 2 + 1 + 1) * reps, "l2": "256 MB written before each timed call"}
 
 
+def time_push(dte, lay, tabs, hp, delta, device, steps=10):
+    """The same-cluster transfer fused into the extract (Section 4.3), outside the timed step: one
+    extract call that also stores every receiver's lists, counts and status block into landing
+    buffers.  This run has one GPU, so the landing buffers are local allocations: the number is the
+    kernel-side cost of the second store of every entry and of the closing kernel, not NVLink time."""
+    R = lay.num_receivers
+    if R == 0:
+        return None
+    cap = delta.capacity
+    try:
+        targets = [dte.PushTarget(lay.num_lists, cap, lay.receiver_num_ops(r), device) for r in range(R)]
+        stream = torch.cuda.current_stream()
+        for i in range(2):
+            dte.dte_extract_delta_push(lay, tabs, *hp, delta, targets, 100 + i)
+        torch.cuda.synchronize()
+        ms = []
+        for i in range(steps):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            dte.dte_extract_delta_push(lay, tabs, *hp, delta, targets, 200 + i)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        status = [t.status.cpu().tolist() for t in targets]
+        delivered = [int(s[0]) for s in status]
+        ok = all(int(s[1]) == 200 + steps - 1 and int(s[2]) == 0 for s in status) and sum(delivered) == delta.total()
+        # the first receiver's slice must equal the head of the sender's own lists
+        n0 = delivered[0]
+        same = bool(torch.equal(targets[0].offsets[:n0], delta.offsets[:n0]) and
+                    torch.equal(targets[0].values[:n0], delta.values[:n0]))
+        return {"ms": sum(ms) / len(ms), "ms_min": min(ms), "receivers": R, "entries_delivered": delivered,
+                "status_ok": bool(ok), "first_slice_equal": same, "launches_per_call": lay.last_launch()["kernels"],
+                "note": "landing buffers on the same GPU (one GPU per run): kernel-side cost only, no NVLink"}
+    except dte.DteError as e:
+        return {"error": str(e)}
+
+
 def aggregate_over_ranks(ms_local: float, units_local: float, dist, device):
     """Weak scaling: the job's time is the slowest rank's, its units the sum over ranks."""
     if dist is None:
@@ -643,6 +680,14 @@ def main():
         ceiling = read_ceiling(device)
         log(f"[bench] read-only streaming ceiling: {ceiling}")
 
+    # ---- same-cluster transfer fused into the extract (outside the timed step) --------------------
+    push = None
+    if rank == 0 and not args.no_codec:
+        push = time_push(dte, lay, tabs, hp, delta, device)
+        if push and "ms" in push:
+            push["extra_ms_over_extract"] = push["ms"] - ext_avg
+        log(f"[bench] push: {push}")
+
     # ---- storage path: chunk codec on the step's lists (outside the timed step) ------------------
     codec = None
     if rank == 0 and not args.no_codec:
@@ -725,7 +770,7 @@ def main():
                          "read_only_ceiling": ceiling,
                          "frac_of_read_only_ceiling": achieved / ceiling["GBps"] if ceiling else None},
             "reconstruction_vs_truth": {"false_negatives": fn, "false_positives": fp, "variant": wl.variant},
-            "storage_path": codec,
+            "storage_path": codec, "push": push,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
             "launch": launch_info, **extra,
         }

@@ -113,6 +113,35 @@ def test_row_parallel_non_multiple_of_four_and_single_rows():
     assert lp[2] == lp[3] == lp[4]          # empty and untouched lists keep their slot
 
 
+@pytest.mark.parametrize("rows", [600, 40000])
+def test_mostly_packed_tiles_with_a_few_regular_ones(rows):
+    # thousands of one-row operations (every one a piece of a packed tile) around two operations
+    # large enough for regular tiles: the packed launch is the long one here and the regular launch,
+    # which starts while it runs, may finish first; the gather must still see every record.
+    # rows = 600 stays under 4096 tiles (one gather launch), rows = 40000 goes over (three).
+    p = plans.Plan()
+    a = p.add_tensor("rows", (rows, 700))
+    b = p.add_tensor("block", (64, 9216))
+    k0 = p.add_shard("r0.rows", 0, rows * 350)
+    k1 = p.add_shard("r0.block", 0, 32 * 9216)
+    k2 = p.add_shard("r1.rows", 1, rows * 350)
+    k3 = p.add_shard("r1.block", 1, 32 * 9216)
+    for r in range(rows):                       # column halves, one row per operation
+        p.add_op(a, k0, (r, 0), (1, 350), r * 350, 350, (0, 0))
+        p.add_op(a, k2, (r, 350), (1, 350), r * 350, 350, (0, 0))
+    p.add_op(b, k1, (0, 0), (32, 9216), 0, 9216, (0, 0))
+    p.add_op(b, k3, (32, 0), (32, 9216), 0, 9216, (0, 0))
+    wl = configs.Workload("packed", p, Hyper(step=50, lr=2e-5, wd=0.01), [Spec(), Spec()], 13)
+    st, lay, d, got, bufs = _full_parity(wl)
+    tiles = lay.last_launch()["tiles"]
+    assert (tiles <= 4096) == (rows == 600) and tiles > 64 + rows * 2 // 8 - 2
+    for _ in range(5):                          # and the same bytes every time
+        d2 = lay.new_delta(d.capacity)
+        run_extract(p, st, wl.hp, layout=lay, delta=d2)
+        assert torch.equal(d2.list_ptr, d.list_ptr)
+        assert torch.equal(d2.offsets[:d.total()], d.offsets[:d.total()])
+
+
 def test_all_changed_and_none_changed():
     plan = plans.qwen3_dense_plan(1, 4, False, configs.SMALL_DENSE)
     # beta = 0.5, t = 1, m = v = 0.5, eps = 0: u = 1 exactly; lr = 8 moves every element far

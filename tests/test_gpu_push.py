@@ -95,6 +95,19 @@ def test_push_delivers_every_receivers_lists_counts_and_status(name):
         assert np.array_equal(shards[k].cpu().numpy().view(np.uint16), host[k]), plan.shard_names[k]
 
 
+def test_push_full_dimension_layer_large_layout_path():
+    # config 2 at full dimensions: 20 9xx tiles, so the three-launch gather and its scan of the
+    # receivers' slice starts are used (the small plans above take the one-launch gather)
+    wl = configs.config2()
+    st = wl.materialize("cuda")
+    want = _oracle_with_counts(wl.plan, st, wl.hp)
+    lay, d, targets = _push(wl.plan, st, wl.hp, capacities=[1 << 20] * 4, epoch=3)
+    assert lay.last_launch()["tiles"] > 4096 and d.status_bits() == 0
+    assert_lists_equal(d.to_host(), want[:3], wl.plan)
+    for r, t in enumerate(targets):
+        _check_receiver(wl.plan, lay, t, r, want, 3)
+
+
 def test_push_when_nothing_changed_still_delivers_zero_counts_and_the_status_block():
     plan = plans.qwen3_dense_plan(2, 4, True, configs.SMALL_DENSE)
     hp = Hyper(step=100, lr=1e-3, wd=0.0)
