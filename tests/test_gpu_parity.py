@@ -113,28 +113,30 @@ def test_row_parallel_non_multiple_of_four_and_single_rows():
     assert lp[2] == lp[3] == lp[4]          # empty and untouched lists keep their slot
 
 
-@pytest.mark.parametrize("rows", [600, 40000])
-def test_mostly_packed_tiles_with_a_few_regular_ones(rows):
-    # thousands of one-row operations (every one a piece of a packed tile) around two operations
-    # large enough for regular tiles: the packed launch is the long one here and the regular launch,
-    # which starts while it runs, may finish first; the gather must still see every record.
-    # rows = 600 stays under 4096 tiles (one gather launch), rows = 40000 goes over (three).
+@pytest.mark.parametrize("rows,block_rows", [(1500, 16), (1500, 8400)])
+def test_packed_tiles_next_to_regular_ones(rows, block_rows):
+    # thousands of one-row operations (every one a piece of a packed tile) next to two operations
+    # made of regular tiles.  With 16 regular tiles the packed launch is the long one and the
+    # regular launch, which starts while it runs, finishes first; the gather must still see every
+    # record (one gather launch: under 4096 tiles).  With 8400 regular tiles the three-launch
+    # gather runs behind both.
     p = plans.Plan()
     a = p.add_tensor("rows", (rows, 700))
-    b = p.add_tensor("block", (64, 9216))
+    b = p.add_tensor("block", (block_rows, 9216))
+    half = block_rows // 2
     k0 = p.add_shard("r0.rows", 0, rows * 350)
-    k1 = p.add_shard("r0.block", 0, 32 * 9216)
+    k1 = p.add_shard("r0.block", 0, half * 9216)
     k2 = p.add_shard("r1.rows", 1, rows * 350)
-    k3 = p.add_shard("r1.block", 1, 32 * 9216)
+    k3 = p.add_shard("r1.block", 1, half * 9216)
     for r in range(rows):                       # column halves, one row per operation
         p.add_op(a, k0, (r, 0), (1, 350), r * 350, 350, (0, 0))
         p.add_op(a, k2, (r, 350), (1, 350), r * 350, 350, (0, 0))
-    p.add_op(b, k1, (0, 0), (32, 9216), 0, 9216, (0, 0))
-    p.add_op(b, k3, (32, 0), (32, 9216), 0, 9216, (0, 0))
+    p.add_op(b, k1, (0, 0), (half, 9216), 0, 9216, (0, 0))
+    p.add_op(b, k3, (half, 0), (half, 9216), 0, 9216, (0, 0))
     wl = configs.Workload("packed", p, Hyper(step=50, lr=2e-5, wd=0.01), [Spec(), Spec()], 13)
     st, lay, d, got, bufs = _full_parity(wl)
     tiles = lay.last_launch()["tiles"]
-    assert (tiles <= 4096) == (rows == 600) and tiles > 64 + rows * 2 // 8 - 2
+    assert tiles == block_rows + 2 * ((rows + 7) // 8) and (tiles <= 4096) == (block_rows == 16)
     for _ in range(5):                          # and the same bytes every time
         d2 = lay.new_delta(d.capacity)
         run_extract(p, st, wl.hp, layout=lay, delta=d2)
