@@ -98,7 +98,8 @@ def full_oracle_parity(wl, st, delta, shards_before=None, shards_after=None, thr
     The state stays on the GPU; one group of tensors at a time is copied to the host (at most
     `budget_bytes` in flight) and handed to a pool of host threads that each run the plain
     single-threaded oracle on it.  Lists no operation feeds must be empty.  Returns
-    (lists compared, entries compared)."""
+    (lists compared, entries compared, the oracle's entry count c_o of every operation in plan
+    order)."""
     import os
     import threading
     from concurrent.futures import ThreadPoolExecutor
@@ -112,16 +113,19 @@ def full_oracle_parity(wl, st, delta, shards_before=None, shards_after=None, thr
     cond = threading.Condition()
     in_flight = [0.0]
     errors, stats = [], [0, 0]
+    op_counts = np.zeros(all_ops.shape[0], np.uint64)
 
     def job(tensors, lists, host, nbytes, before, after):
         try:
             ts = set(tensors)
-            ops = all_ops[np.isin(all_ops[:, 0], np.asarray(tensors))]
+            op_idx = np.nonzero(np.isin(all_ops[:, 0], np.asarray(tensors)))[0]
+            ops = all_ops[op_idx]
             zero = np.zeros(0, np.float32)
             shapes = [s if p in ts else (0, 1) for p, s in enumerate(plan.tensor_shapes)]
             full = [[host[a][p] if p in ts else zero for p in range(plan.n_tensors)] for a in range(3)]
-            want = oracle.extract(shapes, plan.shard_numels, ops, *full, consts)
-            assert_lists_equal((lp_g, off_g, val_g), want, plan, lists)
+            want = oracle.extract(shapes, plan.shard_numels, ops, *full, consts, with_op_counts=True)
+            op_counts[op_idx] = want[3]            # disjoint index sets per job
+            assert_lists_equal((lp_g, off_g, val_g), want[:3], plan, lists)
             n = 0
             for i, k in enumerate(lists):
                 c, d = int(want[0][k]), int(want[0][k + 1])
@@ -164,4 +168,4 @@ def full_oracle_parity(wl, st, delta, shards_before=None, shards_after=None, thr
         if k not in fed:
             assert lp_g[k] == lp_g[k + 1], f"list {plan.shard_names[k]} has no operation but is not empty"
     assert stats[1] == int(lp_g[-1]), "entries compared vs total"
-    return stats[0], stats[1]
+    return stats[0], stats[1], op_counts

@@ -93,7 +93,10 @@ def test_config3_full_qwen3_8b_state():
     N = lay.num_elements
     assert N == 8191035392
     d = lay.new_delta(int(N * 0.03))
-    dte.dte_extract_delta(lay, lay.source_tables(st.theta, st.m, st.v), *wl.hp.as_args(), d)
+    # the extract that also delivers every receiver's share (Section 4.3 fused into the gather);
+    # `d` itself is filled exactly as by dte_extract_delta
+    targets = [dte.PushTarget(lay.num_lists, d.capacity, lay.receiver_num_ops(r), "cuda") for r in range(2)]
+    dte.dte_extract_delta_push(lay, lay.source_tables(st.theta, st.m, st.v), *wl.hp.as_args(), d, targets, 500)
     torch.cuda.synchronize()
     lp = _global_properties(plan, lay, d)
     assert 0.01 < lp[-1] / N < 0.02
@@ -103,9 +106,12 @@ def test_config3_full_qwen3_8b_state():
     dte.dte_apply(lay, d, lay.shard_table(after))
     torch.cuda.synchronize()
     assert d.status_bits() == 0
-    n_lists, n_entries = full_oracle_parity(wl, st, d, shards, after)
+    n_lists, n_entries, op_counts = full_oracle_parity(wl, st, d, shards, after)
     assert n_lists == 580 and n_entries == int(lp[-1])
     del after
+    _free()
+    _receivers_hold_their_share(plan, lay, d, targets, op_counts, 500)
+    del targets
     _free()
     # the storage-path leg below also needs complete oracle lists of a few tensors
     names = plan.tensor_names
@@ -118,6 +124,25 @@ def test_config3_full_qwen3_8b_state():
     _storage_path_at_full_size(wl, st, lay, d, lists, want)
     del st, d, lay
     _free()
+
+
+def _receivers_hold_their_share(plan, lay, d, targets, op_counts, epoch):
+    """What the push delivered: every receiver's slice of the (oracle-checked) lists, its list
+    boundaries relative to the slice, the oracle's per-operation counts in plan order, the status."""
+    lp = d.list_ptr.cpu().numpy().astype(np.int64)
+    recv = np.asarray(plan.shard_receivers)
+    op_recv = recv[plan.ops_array()[:, 1]]
+    for r, t in enumerate(targets):
+        mine = np.nonzero(recv == r)[0]
+        a, b = int(lp[mine[0]]), int(lp[mine[-1] + 1])
+        assert t.status.cpu().tolist() == [b - a, epoch, 0, lay.receiver_num_ops(r)]
+        assert torch.equal(t.offsets[:b - a], d.offsets[a:b]) and torch.equal(t.values[:b - a], d.values[a:b])
+        want_lp = np.clip(lp, a, b) - a
+        assert np.array_equal(t.list_ptr.cpu().numpy(), want_lp)
+        mask = op_recv == r
+        assert int(mask.sum()) == lay.receiver_num_ops(r)
+        assert np.array_equal(t.op_counts[:int(mask.sum())].cpu().numpy().astype(np.uint64), op_counts[mask])
+        assert int(op_counts[mask].sum()) == b - a
 
 
 def _storage_path_at_full_size(wl, st, lay, d, lists, want):
@@ -185,7 +210,7 @@ def test_config4_qwen3_30b_a3b_slice():
     dte.dte_apply(lay, d, lay.shard_table(after))
     torch.cuda.synchronize()
     assert d.status_bits() == 0
-    n_lists, n_entries = full_oracle_parity(wl, st, d, shards, after)
+    n_lists, n_entries, op_counts = full_oracle_parity(wl, st, d, shards, after)
     assert n_lists == 432 and n_entries == d.total()
     # cold experts (zero state) contribute nothing
     cold = [p for p, n in enumerate(plan.tensor_names) if "experts" in n and wl.specs[p].scale == 0.0]
@@ -233,7 +258,7 @@ def test_config5_density_and_edge_grid_full_dimensions(point):
     dte.dte_apply(lay, d, lay.shard_table(after))
     torch.cuda.synchronize()
     assert d.status_bits() == 0
-    n_lists, n_entries = full_oracle_parity(wl, st, d, before, after)
+    n_lists, n_entries, op_counts = full_oracle_parity(wl, st, d, before, after)
     assert n_lists == 32 and n_entries == d.total()
     del st, before, after, d, lay
     _free()
