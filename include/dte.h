@@ -18,7 +18,10 @@
  * Conventions
  *   - "device pointer" = CUDA global memory of the layout's device; "host pointer" =
  *     ordinary or pinned host memory.  The library never frees or keeps caller memory.
- *   - All tensors are row-major and contiguous.  fp32 inputs must be 16-byte aligned.
+ *   - All tensors are row-major and contiguous.  fp32 inputs should be 16-byte aligned (any
+ *     framework allocation is); a call in which some theta / m / v pointer is only 4-byte aligned -
+ *     a view into a flat buffer at an odd element - is served with scalar loads throughout, at a
+ *     fraction of the speed.
  *   - Every call that takes a stream enqueues on it (void* = cudaStream_t; NULL = the
  *     default stream) and returns without synchronising unless stated otherwise.
  *   - Functions return DTE_OK or an error detected on the host.  Conditions only the
@@ -160,7 +163,7 @@ DTE_API dte_status dte_derive_constants(int64_t step, double lr, double beta1, d
                                 double wd, float* out5);
 
 /* Eq. 2 + Eq. 4 + Eq. 5-6 in one streaming pass.  theta / m / v: HOST arrays of
- * n_tensors DEVICE pointers (fp32, 16-byte aligned; entries of tensors no operation
+ * n_tensors DEVICE pointers (fp32, 16-byte aligned for full speed; entries of tensors no operation
  * reads may be NULL).  `step` is the 1-based index of the optimizer step that produced
  * theta.  Arithmetic: IEEE binary32, every operation rounded to nearest-even on its own,
  * no fused multiply-add across operations, subnormals kept; BF16 by round-to-nearest-even

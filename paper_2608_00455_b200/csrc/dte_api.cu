@@ -38,13 +38,18 @@ dte_status sync_source_table(dte_layout* L, const float* const* theta, const flo
                              const float* const* v, cudaStream_t st) {
     const size_t n = L->n_tensors;
     std::vector<const float*> tab(3 * n);
+    bool unaligned = false;
     for (size_t p = 0; p < n; ++p) {
         tab[p] = theta[p]; tab[n + p] = m[p]; tab[2 * n + p] = v[p];
         if (!L->tensor_used[p]) continue;
         if (!theta[p] || !m[p] || !v[p]) return fail(DTE_ERR_INVALID_ARG, "null theta / m / v pointer for a tensor the plan reads");
-        if (((uintptr_t)theta[p] | (uintptr_t)m[p] | (uintptr_t)v[p]) & 15u)
-            return fail(DTE_ERR_INVALID_ARG, "theta / m / v must be 16-byte aligned");
+        const uintptr_t bits = (uintptr_t)theta[p] | (uintptr_t)m[p] | (uintptr_t)v[p];
+        if (bits & 3u) return fail(DTE_ERR_INVALID_ARG, "theta / m / v must be 4-byte aligned");
+        // A tensor that is only 4-byte aligned (a view into a flat buffer at an odd element)
+        // cannot be read with 128-bit loads: the whole call then takes the scalar-load path.
+        if (bits & 15u) unaligned = true;
     }
+    L->scalar_loads = unaligned;
     if (L->ptrs_valid && tab == L->h_ptrs) return DTE_OK;
     L->ptrs_valid = false;
     // pageable source: the runtime stages the bytes before returning, so `tab` may die
@@ -138,6 +143,7 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
     p.s = make_screen(c);
     p.tensor_group = nullptr;
     p.groups = nullptr;
+    p.force_flags = L->scalar_loads ? kFlagScalar : 0u;
     bool div_bc1 = c.bc1 != 1.0f, div_decay = c.decay != 1.0f;
     if (groups) {
         // pageable source: staged by the runtime before the call returns

@@ -181,7 +181,7 @@ __device__ __forceinline__ uint32_t decode(const ExtractParams& p, uint32_t inde
     const uint32_t e0 = PACKED ? 0u : (uint32_t)warp * kWarpTile;
     const uint32_t run_len = d1.x & kLenMask;
     tile = d1.y;
-    wt.len_flags = d1.x;
+    wt.len_flags = d1.x | p.force_flags;
     wt.len = run_len > e0 ? min(run_len - e0, (uint32_t)kWarpTile) : 0u;
     wt.dst0 = d0.w + e0;
     wt.geom = geom;

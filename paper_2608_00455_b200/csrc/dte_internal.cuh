@@ -132,6 +132,7 @@ struct ExtractParams {
     uint64_t stage_capacity;
     Consts c;                    // single-group calls: constants in the kernel parameters
     Screen s;
+    uint32_t force_flags;           // OR-ed into every tile's flags: kFlagScalar when a source pointer of the call is not 16-byte aligned
     const uint32_t* tensor_group;   // per-group calls: group of each source tensor ...
     const GroupConsts* groups;      // ... and the constants of each group (NULL otherwise)
 };
@@ -339,5 +340,6 @@ struct dte_layout {
     std::vector<const float*> h_ptrs;
     std::vector<uint16_t*> h_shards;
     bool ptrs_valid = false, shards_valid = false;
+    bool scalar_loads = false;             // the current call's source pointers are not all 16-byte aligned
     uint64_t last_launch[3] = {0, 0, 0};
 };

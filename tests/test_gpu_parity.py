@@ -277,12 +277,41 @@ def test_layout_errors():
         assert e.value.status == 2
     lay = dte.Layout([(8, 8)], [64], ok_ops)
     t = torch.zeros(65, dtype=torch.float32, device="cuda")
-    with pytest.raises(dte.DteError):                                     # misaligned theta
-        dte.dte_extract_delta(lay, lay.source_tables([t[1:]], [t[1:]], [t[1:]]), 1, 1e-3, 0.9, 0.999, 1e-8, 0.0,
-                              lay.new_delta(64))
     with pytest.raises(dte.DteError):                                     # step 0
         dte.dte_extract_delta(lay, lay.source_tables([t[:64]], [t[:64]], [t[:64]]), 0, 1e-3, 0.9, 0.999, 1e-8, 0.0,
                               lay.new_delta(64))
+
+
+def test_source_tensors_that_are_only_four_byte_aligned():
+    # views into flat buffers at odd element offsets (a flat optimizer buffer cut at arbitrary
+    # elements): 128-bit loads are not possible, the call falls back to scalar loads and must give
+    # the same lists; the next call with aligned tensors goes back to the fast path
+    plan = plans.qwen3_dense_plan(1, 4, True, configs.SMALL_DENSE)
+    wl = configs.Workload("views", plan, Hyper(step=100, lr=1e-5, wd=0.01), configs._specs(plan), 19)
+    st = wl.materialize("cuda")
+    want = oracle_extract(plan, st, wl.hp)
+
+    def shifted(lst, k):
+        out = []
+        for x in lst:
+            buf = torch.empty(x.numel() + 4, dtype=torch.float32, device="cuda")
+            buf[k:k + x.numel()] = x
+            out.append(buf[k:k + x.numel()])
+        return out
+
+    lay = dte.Layout.from_plan(plan, 0)
+    for k_theta, k_m, k_v in [(1, 2, 3), (3, 0, 0), (0, 0, 1)]:
+        th, mm, vv = shifted(st.theta, k_theta), shifted(st.m, k_m), shifted(st.v, k_v)
+        assert th[0].data_ptr() % 16 == 4 * k_theta
+        d = lay.new_delta(lay.num_elements)
+        dte.dte_extract_delta(lay, lay.source_tables(th, mm, vv), *wl.hp.as_args(), d)
+        torch.cuda.synchronize()
+        assert d.status_bits() == 0
+        assert_lists_equal(d.to_host(), want, plan)
+    d = lay.new_delta(lay.num_elements)
+    dte.dte_extract_delta(lay, lay.source_tables(st.theta, st.m, st.v), *wl.hp.as_args(), d)
+    torch.cuda.synchronize()
+    assert_lists_equal(d.to_host(), want, plan)
 
 
 def test_empty_layouts_and_empty_operations():
