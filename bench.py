@@ -37,6 +37,7 @@ FALLBACK_HBM_GBS = 6650.0
 # of one launch over a one-layer case, and the elements that launch scanned), kept as data next
 # to the capture's summary; `roofline.traffic` scales it to the workload's element count.
 EXTRACT_TRAFFIC_JSON = os.path.join(ROOT, "profiles", "extract_kernel.qwen3-8b-one-layer.traffic.json")
+APPLY_TRAFFIC_JSON = os.path.join(ROOT, "profiles", "apply_kernel.qwen3-8b-one-layer.traffic.json")
 
 
 def log(*a):
@@ -239,6 +240,17 @@ def extract_traffic(n_elements):
                                      "scaled_from_elements": int(t["elements_scanned"])}
     except Exception as e:      # no capture committed: say so instead of inventing a number
         return None, {"error": f"{type(e).__name__}: {e}"}
+
+
+def apply_traffic_per_entry():
+    """DRAM bytes per entry of apply_kernel at the headline density, from the committed ncu capture
+    (sector fill + write-back of the touched sectors + the lists); None without a capture."""
+    try:
+        with open(APPLY_TRAFFIC_JSON) as f:
+            t = json.load(f)
+        return (float(t["dram_bytes_read"]) + float(t["dram_bytes_write"])) / float(t["entries"])
+    except Exception:
+        return None
 
 
 def time_leg(dte, make_wl, device, steps, warmup, peak, capacity_frac=0.03, with_clocks=True, copies=1):
@@ -670,6 +682,7 @@ def main():
     value = bytes_all / (ms_per_step * 1e-3) / 1e9
     ext_avg = sum(ext_ms) / len(ext_ms)
     app_avg = sum(app_ms) / len(app_ms)
+    apply_bpe = apply_traffic_per_entry()
     peak, peak_kind = measured_peak()
     achieved = bytes_per_step / (ext_avg * 1e-3) / 1e9
     traffic, traffic_src = extract_traffic(N)
@@ -757,13 +770,17 @@ def main():
             "config": {"workload": wl.name, "elements_scanned": N, "changed": M, "changed_frac": M / N,
                        "lists": n_lists, "l2": "inputs larger than L2 (no flush needed)" if flush is None else "256 MB written between timed steps to flush L2",
                        "hyper": {"step": wl.hp.step, "lr": wl.hp.lr, "wd": wl.hp.wd}, **wl.notes},
-            "extract": {"ms": ext_avg, "ms_min": min(ext_ms), "GBps": achieved, "elements_per_s": N / (ext_avg * 1e-3),
+            "extract": {"ms": ext_avg, "ms_min": min(ext_ms), "ms_median": statistics.median(ext_ms), "GBps": achieved, "elements_per_s": N / (ext_avg * 1e-3),
                         "frac_of_8TBps": achieved / 8000.0},
-            "apply": {"ms": app_avg, "ms_min": min(app_ms), "Mchanged_per_s": M / (app_avg * 1e-3) / 1e6,
+            "apply": {"ms": app_avg, "ms_min": min(app_ms), "ms_median": statistics.median(app_ms),
+                      "Mchanged_per_s": M / (app_avg * 1e-3) / 1e6,
                       "GBps_algorithmic": 8.0 * M / (app_avg * 1e-3) / 1e9,
-                      # isolated 2-byte writes: 6 B of list read + a 32 B sector fill + a 32 B write-back
-                      "GBps_sector_traffic": 70.0 * M / (app_avg * 1e-3) / 1e9,
-                      "frac_of_peak_sector_traffic": 70.0 * M / (app_avg * 1e-3) / 1e9 / peak},
+                      # DRAM traffic per entry measured by ncu at this density (sector fill and
+                      # write-back of every touched sector + the lists); model figure if no capture
+                      "dram_bytes_per_entry": apply_bpe if apply_bpe else 70.0,
+                      "dram_bytes_per_entry_source": os.path.basename(APPLY_TRAFFIC_JSON) if apply_bpe else "model: 32 B fill + 32 B write-back + 6 B list",
+                      "GBps_dram_traffic": (apply_bpe or 70.0) * M / (app_avg * 1e-3) / 1e9,
+                      "frac_of_peak_dram_traffic": (apply_bpe or 70.0) * M / (app_avg * 1e-3) / 1e9 / peak},
             "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                          "traffic": traffic, "traffic_source": traffic_src, "peak_source": peak_kind,
                          "kernel": "extract call (extract_kernel launches + scan + gather)",
