@@ -368,7 +368,9 @@ __global__ void push_wait_kernel(const uint64_t* status, uint64_t epoch, uint64_
 dte_status launch_push_wait(const uint64_t* status, uint64_t epoch, uint32_t timeout_ms, uint64_t* counters,
                             cudaStream_t st) {
     const uint64_t ms = std::min<uint32_t>(timeout_ms, 10000u);
-    push_wait_kernel<<<1, 32, 0, st>>>(status, epoch, ms * 1000000ull, ms * 2000ull + 1, counters);
+    // the poll count is the second limit, for a clock that does not advance: generous enough (a
+    // poll is a system-scope load and a sleep, never under 50 ns) not to cut the time limit short
+    push_wait_kernel<<<1, 32, 0, st>>>(status, epoch, ms * 1000000ull, ms * 20000ull + 1000, counters);
     DTE_CUDA(cudaGetLastError());
     return DTE_OK;
 }
