@@ -1,0 +1,98 @@
+"""Every fp32 bit pattern of theta, once: a 65536 x 65536 source tensor whose element i has the
+bit pattern i, with moments that cycle through small tables (signs, magnitudes from far below to
+far above the distance to a BF16 rounding boundary, zeros, a negative and a subnormal second
+moment).  The changed set, offsets and values of the CUDA path must equal the oracle's Eq. 4 mask
+on all 2^32 elements - NaNs, infinities, subnormals, ties and the overflow threshold included -
+for hyper-parameters with and without the divisions by the bias correction and the decay factor.
+"""
+import os
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2608_00455_b200 as dte
+from synth import plans
+
+pytestmark = pytest.mark.gpu
+
+N = 1 << 32
+HALF = 1 << 31
+CHUNK = 1 << 25
+M_TABLE = np.array([3e-4, -3e-4, 1e-6, -2e-2, 0.0, 5e-9, -1.5e-3], np.float32)            # period 7
+V_TABLE = np.array([1e-6, 4e-10, 0.0, 2.5e-3, 1e-40, -1e-6, 9e-8, 1e-12, 3e-5, 1e-6, 6e-7], np.float32)   # period 11
+
+
+def _tables(lo, n):
+    i = np.arange(lo, lo + n, dtype=np.int64)
+    return M_TABLE[i % 7], V_TABLE[i % 11]
+
+
+@pytest.mark.parametrize("hp", [(500, 1e-6, 0.9, 0.999, 1e-8, 0.01),      # bc1 = decay = 1: no constant division
+                                (3, 2e-4, 0.9, 0.999, 1e-8, 0.1),          # both divisions, direction-aware screen with decay
+                                (40, 1e-3, 0.8, 0.99, 0.0, 0.0)],          # eps = 0: m = v = 0 gives 0/0
+                         ids=["t500-lr1e-6", "t3-lr2e-4-wd0.1", "eps0"])
+def test_every_fp32_pattern_of_theta(hp):
+    free, _ = torch.cuda.mem_get_info()
+    if free < 110e9:
+        pytest.skip("needs 110 GB of free device memory")
+    dev = torch.device("cuda", 0)
+    theta = torch.empty(N, dtype=torch.float32, device=dev)
+    m = torch.empty(N, dtype=torch.float32, device=dev)
+    v = torch.empty(N, dtype=torch.float32, device=dev)
+    mt, vt = torch.from_numpy(M_TABLE).to(dev), torch.from_numpy(V_TABLE).to(dev)
+    for lo in range(0, N, 1 << 28):
+        i = torch.arange(lo, lo + (1 << 28), dtype=torch.int64, device=dev)
+        theta[lo:lo + (1 << 28)] = i.to(torch.int32).view(torch.float32) if lo < HALF else (i - N).to(torch.int32).view(torch.float32)
+        m[lo:lo + (1 << 28)] = mt[i % 7]
+        v[lo:lo + (1 << 28)] = vt[i % 11]
+        del i
+    assert int(theta[12345].view(torch.int32)) == 12345 and int(theta[N - 1].view(torch.int32)) == -1
+    # two receivers, 2^31 elements each (a destination tensor must have fewer than 2^32)
+    plan = plans.Plan()
+    a = plan.add_tensor("all", (1 << 16, 1 << 16))
+    for r in range(2):
+        k = plan.add_shard(f"half{r}", r, HALF)
+        plan.add_op(a, k, (r << 15, 0), (1 << 15, 1 << 16), 0, 1 << 16, (0, 0))
+    lay = dte.Layout.from_plan(plan, 0)
+    assert lay.num_elements == N
+    # size discovery first (about half of all patterns change: every theta smaller than the step
+    # does), then buffers of exactly that size
+    tabs = lay.source_tables([theta], [m], [v])
+    d = lay.new_delta(1024)
+    dte.dte_extract_delta(lay, tabs, *hp, d)
+    torch.cuda.synchronize()
+    assert d.status_bits() == dte.DTE_DEV_OVERFLOW
+    total = d.total()
+    assert N // 100 < total < N
+    d = lay.new_delta(total)
+    dte.dte_extract_delta(lay, tabs, *hp, d)
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0 and d.total() == total
+    del theta, m, v
+    torch.cuda.empty_cache()
+    lp = d.list_ptr.cpu().numpy().astype(np.int64)
+    consts = oracle.derive_constants(*hp)
+
+    def job(lo):
+        bits = np.arange(lo, lo + CHUNK, dtype=np.int64).astype(np.uint32)
+        mm, vv = _tables(lo, CHUNK)
+        mask, v16 = oracle.changed_mask(bits.view(np.float32), mm, vv, consts)
+        idx = np.nonzero(mask)[0]
+        return lo, (idx + (lo % HALF)).astype(np.uint32), v16[idx]
+
+    cursor = 0
+    with ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as pool:
+        for lo, want_off, want_val in pool.map(job, range(0, N, CHUNK)):
+            if lo == HALF:
+                assert cursor == int(lp[1]), "boundary between the two lists"
+            n = want_off.size
+            assert cursor + n <= total, f"more entries expected than produced, chunk at {lo:#x}"
+            off = d.offsets[cursor:cursor + n].cpu().numpy().view(np.uint32)
+            val = d.values[cursor:cursor + n].cpu().numpy().view(np.uint16)
+            assert np.array_equal(off, want_off), f"offsets of chunk at {lo:#x}"
+            assert np.array_equal(val, want_val), f"values of chunk at {lo:#x}"
+            cursor += n
+    assert cursor == total
