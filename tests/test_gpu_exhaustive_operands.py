@@ -4,6 +4,8 @@ far above the distance to a BF16 rounding boundary, zeros, a negative and a subn
 moment).  The changed set, offsets and values of the CUDA path must equal the oracle's Eq. 4 mask
 on all 2^32 elements - NaNs, infinities, subnormals, ties and the overflow threshold included -
 for hyper-parameters with and without the divisions by the bias correction and the decay factor.
+The same for every bit pattern of the first moment and of the second moment, theta then cycling
+through weights, ties, zeros and extremes.
 """
 import os
 from concurrent.futures import ThreadPoolExecutor
@@ -25,16 +27,31 @@ M_TABLE = np.array([3e-4, -3e-4, 1e-6, -2e-2, 0.0, 5e-9, -1.5e-3], np.float32)  
 V_TABLE = np.array([1e-6, 4e-10, 0.0, 2.5e-3, 1e-40, -1e-6, 9e-8, 1e-12, 3e-5, 1e-6, 6e-7], np.float32)   # period 11
 
 
-def _tables(lo, n):
+# theta when it is not the exhaustive operand: weights, BF16 ties and their neighbours, zeros,
+# the overflow threshold, a subnormal tie, +-65504                                             period 13
+T_TABLE = np.array([0x3C23D70A, 0xBCA3D70A, 0x3F808000, 0x3F807FFF, 0x3F808001, 0x00000000, 0x80000000,
+                    0x7F7F8000, 0x00008000, 0x3F800000, 0xC77FE000, 0x3A83126F, 0xBF818000], np.uint32).view(np.float32)
+
+
+def _operands(which, lo, n):
+    """(theta, m, v) of elements lo .. lo+n-1: operand `which` has bit pattern i, the others cycle."""
     i = np.arange(lo, lo + n, dtype=np.int64)
-    return M_TABLE[i % 7], V_TABLE[i % 11]
+    exhaustive = i.astype(np.uint32).view(np.float32)
+    th = exhaustive if which == "theta" else T_TABLE[i % 13]
+    mm = exhaustive if which == "m" else M_TABLE[i % 7]
+    vv = exhaustive if which == "v" else V_TABLE[i % 11]
+    return th, mm, vv
 
 
-@pytest.mark.parametrize("hp", [(500, 1e-6, 0.9, 0.999, 1e-8, 0.01),      # bc1 = decay = 1: no constant division
-                                (3, 2e-4, 0.9, 0.999, 1e-8, 0.1),          # both divisions, direction-aware screen with decay
-                                (40, 1e-3, 0.8, 0.99, 0.0, 0.0)],          # eps = 0: m = v = 0 gives 0/0
-                         ids=["t500-lr1e-6", "t3-lr2e-4-wd0.1", "eps0"])
-def test_every_fp32_pattern_of_theta(hp):
+HP_PLAIN = (500, 1e-6, 0.9, 0.999, 1e-8, 0.01)     # bc1 = decay = 1: no constant division
+HP_DECAY = (3, 2e-4, 0.9, 0.999, 1e-8, 0.1)         # both divisions, direction-aware screen with decay
+HP_EPS0 = (40, 1e-3, 0.8, 0.99, 0.0, 0.0)           # eps = 0: m = v = 0 gives 0/0
+
+
+@pytest.mark.parametrize("which,hp", [("theta", HP_PLAIN), ("theta", HP_DECAY), ("theta", HP_EPS0),
+                                      ("m", HP_DECAY), ("v", HP_DECAY), ("v", HP_PLAIN)],
+                         ids=["theta-plain", "theta-decay", "theta-eps0", "m-decay", "v-decay", "v-plain"])
+def test_every_fp32_pattern_of_one_operand(which, hp):
     free, _ = torch.cuda.mem_get_info()
     if free < 110e9:
         pytest.skip("needs 110 GB of free device memory")
@@ -42,14 +59,17 @@ def test_every_fp32_pattern_of_theta(hp):
     theta = torch.empty(N, dtype=torch.float32, device=dev)
     m = torch.empty(N, dtype=torch.float32, device=dev)
     v = torch.empty(N, dtype=torch.float32, device=dev)
-    mt, vt = torch.from_numpy(M_TABLE).to(dev), torch.from_numpy(V_TABLE).to(dev)
+    tt, mt, vt = (torch.from_numpy(x.copy()).to(dev) for x in (T_TABLE, M_TABLE, V_TABLE))
     for lo in range(0, N, 1 << 28):
+        sl = slice(lo, lo + (1 << 28))
         i = torch.arange(lo, lo + (1 << 28), dtype=torch.int64, device=dev)
-        theta[lo:lo + (1 << 28)] = i.to(torch.int32).view(torch.float32) if lo < HALF else (i - N).to(torch.int32).view(torch.float32)
-        m[lo:lo + (1 << 28)] = mt[i % 7]
-        v[lo:lo + (1 << 28)] = vt[i % 11]
-        del i
-    assert int(theta[12345].view(torch.int32)) == 12345 and int(theta[N - 1].view(torch.int32)) == -1
+        bits = (i if lo < HALF else i - N).to(torch.int32).view(torch.float32)      # element i has bit pattern i
+        theta[sl] = bits if which == "theta" else tt[i % 13]
+        m[sl] = bits if which == "m" else mt[i % 7]
+        v[sl] = bits if which == "v" else vt[i % 11]
+        del i, bits
+    probe = {"theta": theta, "m": m, "v": v}[which]
+    assert int(probe[12345].view(torch.int32)) == 12345 and int(probe[N - 1].view(torch.int32)) == -1
     # two receivers, 2^31 elements each (a destination tensor must have fewer than 2^32)
     plan = plans.Plan()
     a = plan.add_tensor("all", (1 << 16, 1 << 16))
@@ -58,15 +78,15 @@ def test_every_fp32_pattern_of_theta(hp):
         plan.add_op(a, k, (r << 15, 0), (1 << 15, 1 << 16), 0, 1 << 16, (0, 0))
     lay = dte.Layout.from_plan(plan, 0)
     assert lay.num_elements == N
-    # size discovery first (about half of all patterns change: every theta smaller than the step
-    # does), then buffers of exactly that size
+    # size discovery first (with theta exhaustive about half of all patterns change: every theta
+    # smaller than the step does), then buffers of exactly that size
     tabs = lay.source_tables([theta], [m], [v])
     d = lay.new_delta(1024)
     dte.dte_extract_delta(lay, tabs, *hp, d)
     torch.cuda.synchronize()
     assert d.status_bits() == dte.DTE_DEV_OVERFLOW
     total = d.total()
-    assert N // 100 < total < N
+    assert N // 1000 < total < N
     d = lay.new_delta(total)
     dte.dte_extract_delta(lay, tabs, *hp, d)
     torch.cuda.synchronize()
@@ -77,9 +97,8 @@ def test_every_fp32_pattern_of_theta(hp):
     consts = oracle.derive_constants(*hp)
 
     def job(lo):
-        bits = np.arange(lo, lo + CHUNK, dtype=np.int64).astype(np.uint32)
-        mm, vv = _tables(lo, CHUNK)
-        mask, v16 = oracle.changed_mask(bits.view(np.float32), mm, vv, consts)
+        th, mm, vv = _operands(which, lo, CHUNK)
+        mask, v16 = oracle.changed_mask(th, mm, vv, consts)
         idx = np.nonzero(mask)[0]
         return lo, (idx + (lo % HALF)).astype(np.uint32), v16[idx]
 
