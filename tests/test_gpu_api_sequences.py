@@ -83,3 +83,45 @@ def test_random_call_sequences(seed):
         exp = _expected_shards(plan, want, fill)
         for k in range(plan.n_shards):
             assert np.array_equal(shards[k].cpu().numpy().view(np.uint16), exp[k]), (step, kind, plan.shard_names[k])
+
+
+def test_two_layouts_on_two_streams_and_two_host_threads():
+    """Different layouts are independent: two host threads, each with a layout and a stream of its
+    own, extract and apply at the same time (the per-device host state of the library - kernel
+    attributes, cached tables - is shared between them).  Every result must equal the oracle's."""
+    import threading
+    cases = []
+    for i, plan in enumerate([plans.qwen3_dense_plan(2, 2, True, configs.SMALL_DENSE),
+                              plans.qwen3_moe_plan(2, 4, 4, configs.SMALL_MOE)]):
+        hp = Hyper(step=50 + i, lr=2e-5, wd=0.01 * i)        # one call with, one without the decay division
+        wl = configs.Workload(f"t{i}", plan, hp, configs._specs(plan), 70 + i)
+        st = wl.materialize("cuda")
+        cases.append((plan, hp, st, oracle_extract(plan, st, hp)))
+    errors = []
+
+    def work(plan, hp, st, want):
+        try:
+            stream = torch.cuda.Stream()
+            lay = dte.Layout.from_plan(plan, 0)
+            tabs = lay.source_tables(st.theta, st.m, st.v)
+            for it in range(20):
+                d = lay.new_delta(int(want[0][-1]) + 16 * it)
+                shards = [torch.zeros(n, dtype=torch.int16, device="cuda") for n in plan.shard_numels]
+                stream.wait_stream(torch.cuda.current_stream())        # the zero fills above
+                dte.dte_extract_delta(lay, tabs, *hp.as_args(), d, stream=stream)
+                dte.dte_apply(lay, d, lay.shard_table(shards), stream=stream)
+                stream.synchronize()
+                assert d.status_bits() == 0
+                assert_lists_equal(d.to_host(), want, plan)
+                exp = _expected_shards(plan, want, 0)
+                assert all(np.array_equal(shards[k].cpu().numpy().view(np.uint16), exp[k]) for k in range(plan.n_shards))
+        except BaseException as e:
+            errors.append(e)
+
+    threads = [threading.Thread(target=work, args=c) for c in cases]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    if errors:
+        raise errors[0]
