@@ -181,3 +181,45 @@ def test_push_needs_consecutive_shards_per_receiver():
         dte.dte_extract_delta_push(lay, lay.source_tables([z], [z], [z]), 1, 1e-3, 0.9, 0.999, 1e-8, 0.0,
                                    lay.new_delta(64), targets, 1)
     assert e.value.status == 2
+
+
+def test_push_into_a_second_gpus_memory_when_there_is_one():
+    """The intended deployment: the landing buffers live on the receiver's GPU and the sender's
+    gather kernel stores into them through peer access.  Needs two GPUs that can reach each other
+    (this test is skipped on a single-GPU machine; everything else about the push is covered above
+    with landing buffers on the sender's own GPU)."""
+    if torch.cuda.device_count() < 2 or not torch.cuda.can_device_access_peer(0, 1):
+        pytest.skip("needs two GPUs with peer access")
+    torch.zeros(8, device="cuda:0").to("cuda:1")               # lets torch enable peer access 0 -> 1
+    plan = plans.qwen3_dense_plan(2, 2, True, configs.SMALL_DENSE)
+    hp = Hyper(step=100, lr=1e-5, wd=0.01)
+    wl = configs.Workload("p2p", plan, hp, configs._specs(plan), 77)
+    st = wl.materialize("cuda:0")
+    want = _oracle_with_counts(plan, st, hp)
+    send = dte.Layout.from_plan(plan, 0)
+    recv = dte.Layout.from_plan(plan, 1)                       # the receiver compiles the same plan
+    d = send.new_delta(send.num_elements)
+    # receiver 0 stays on the sender's GPU, receiver 1 is the second GPU
+    targets = [dte.PushTarget(send.num_lists, send.num_elements, send.receiver_num_ops(0), "cuda:0"),
+               dte.PushTarget(send.num_lists, send.num_elements, send.receiver_num_ops(1), "cuda:1")]
+    mine = [k for k, r in enumerate(plan.shard_receivers) if r == 1]
+    with torch.cuda.device(1):
+        shards = [torch.zeros(n, dtype=torch.int16, device="cuda:1") if k in mine else None
+                  for k, n in enumerate(plan.shard_numels)]
+        s1 = torch.cuda.current_stream(1)
+        torch.cuda.synchronize(1)
+        # the receiver waits (at most 5 s) on its own GPU while the sender works on the other
+        dte.dte_push_wait(targets[1], 9, timeout_ms=5000, stream=s1)
+        dte.dte_apply(recv, targets[1].delta(), recv.shard_table(shards), stream=s1)
+    dte.dte_extract_delta_push(send, send.source_tables(st.theta, st.m, st.v), *hp.as_args(), d, targets, 9)
+    torch.cuda.synchronize(0)
+    torch.cuda.synchronize(1)
+    _check_receiver(plan, send, targets[0], 0, want, 9)
+    _check_receiver(plan, send, targets[1], 1, want, 9)
+    assert targets[1].counters.cpu().tolist()[2] == 0
+    lp_w, off_w, val_w, _ = want
+    for k in mine:
+        exp = np.zeros(plan.shard_numels[k], np.uint16)
+        seg = slice(int(lp_w[k]), int(lp_w[k + 1]))
+        exp[off_w[seg]] = val_w[seg]
+        assert np.array_equal(shards[k].cpu().numpy().view(np.uint16), exp), plan.shard_names[k]
