@@ -277,8 +277,9 @@ DTE_API size_t dte_layout_num_ops(const dte_layout* layout);
  *               shard belongs to receiver r, in plan order, zeros included
  *   status    : 4 x uint64 = { entries of the slice, epoch, DTE_DEV_* bits, operations }.  The
  *               epoch word is written last (release at system scope).  DTE_DEV_OVERFLOW: the slice
- *               exceeds `capacity`, or the sender's own delta overflowed; the sizes are exact, the
- *               entries are not usable. */
+ *               exceeds `capacity`, or the sender's own delta overflowed; list_ptr and the entry
+ *               total are exact, the entries are not usable (and if it was the sender's delta
+ *               that overflowed, the per-operation counts are all zero). */
 typedef struct dte_push_target {
     uint32_t* offsets;
     uint16_t* values;
