@@ -61,6 +61,20 @@ def test_static_scratch_extract_matches_the_allocating_one_twice_in_a_row():
     assert_lists_equal(got2.to_host(), oracle_extract(wl2.plan, st2, wl2.hp), wl2.plan)
 
 
+def test_static_scratch_extract_on_a_layout_with_thousands_of_tiles():
+    # 67 M elements = 7 282 tiles: beyond the one-launch gather, so the fixed array also carries the
+    # block sums of the three-launch gather; compared with the allocating call, twice in a row
+    from synth import plans
+    plan = plans.single_matrix_plan(8192, 8192, 2)
+    wl = configs.Workload("wide", plan, Hyper(step=100, lr=1e-6, wd=0.01), configs._specs(plan), 14)
+    st = wl.materialize("cuda")
+    lay = dte.Layout.from_plan(plan, 0)
+    for _ in range(2):
+        ref, got = _both(lay, st, wl.hp, 1 << 20)
+        _assert_same(ref, got)
+    assert lay.last_launch()["tiles"] > 4096 and lay.last_launch()["kernels"] == 5
+
+
 def test_static_scratch_extract_overflow_and_empty_plan():
     # capacity below the number of changed elements: exact sizes reported, nothing written past
     # the caller's arrays (they sit inside a canary pool), same answer as the allocating call
