@@ -755,8 +755,7 @@ def main():
         log(f"[bench] config 1: {extra['config1']}")
         sweep = []
         for (lr, step_t, wd, sg) in density_sweep_points():
-            r = time_leg(dte, lambda i: configs.config5(lr, step_t, wd, sg), device, 20, args.warmup, peak, 0.03,
-                         with_clocks=False)
+            r = time_leg(dte, lambda i: configs.config5(lr, step_t, wd, sg), device, 20, args.warmup, peak, 0.03)
             r["sigma_g"] = sg
             sweep.append(r)
             log(f"[bench] sweep lr={lr:g} sigma_g={sg:g}: rho={r.get('changed_frac')} extract {r.get('extract_GBps')} GB/s")
