@@ -56,6 +56,8 @@ def lib() -> ctypes.CDLL:
             L.oracle_result_copy.restype = None
             L.oracle_result_op_counts.argtypes = [c.c_void_p, c.c_void_p]
             L.oracle_result_op_counts.restype = None
+            L.oracle_result_nonfinite.argtypes = [c.c_void_p]
+            L.oracle_result_nonfinite.restype = c.c_uint64
             L.oracle_result_free.argtypes = [c.c_void_p]
             L.oracle_result_free.restype = None
             L.oracle_apply.argtypes = [c.c_uint64, c.c_void_p, c.c_void_p, c.c_void_p, c.c_void_p,
@@ -121,7 +123,7 @@ def _ptr_array(arrs):
     return (ctypes.c_void_p * len(arrs))(*[a.ctypes.data for a in arrs])
 
 
-def extract(tensor_shapes, shard_numels, ops, theta, m, v, consts, with_op_counts=False):
+def extract(tensor_shapes, shard_numels, ops, theta, m, v, consts, with_op_counts=False, with_nonfinite=False):
     """Full extract (Eq. 2, 4, 5, 6) over a transfer plan.
 
     tensor_shapes: [(n0, n1)] per source tensor; shard_numels: [numel] per
@@ -160,11 +162,15 @@ def extract(tensor_shapes, shard_numels, ops, theta, m, v, consts, with_op_count
         L.oracle_result_copy(h, list_ptr.ctypes.data, offsets.ctypes.data, values.ctypes.data)
         op_counts = np.zeros(op.shape[0], np.uint64)
         L.oracle_result_op_counts(h, op_counts.ctypes.data)
+        nonfinite = int(L.oracle_result_nonfinite(h))
     finally:
         L.oracle_result_free(h)
+    out = (list_ptr, offsets, values)
     if with_op_counts:          # c_o per operation, plan order, zeros included (Section 4.3)
-        return list_ptr, offsets, values, op_counts
-    return list_ptr, offsets, values
+        out += (op_counts,)
+    if with_nonfinite:          # receiver slots whose theta_t or reconstruction is NaN / Inf
+        out += (nonfinite,)
+    return out
 
 
 def apply(shard_numels, list_ptr, offsets, values, shards) -> None:

@@ -79,6 +79,7 @@ struct Result {
     std::vector<uint64_t> list_ptr;   // n_shards + 1
     std::vector<uint32_t> offsets;
     std::vector<uint16_t> values;
+    uint64_t nonfinite = 0;           // scanned slots whose theta_t or reconstruction is NaN or +-Inf
     std::string error;
 };
 
@@ -173,7 +174,10 @@ void* oracle_extract(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n
             float prev = invert_one(theta[p][i], m[p][i], v[p][i], c);
             uint16_t bt = bf16_rne(theta[p][i]);
             uint16_t bp = bf16_rne(prev);
-            if (bt == bp) continue;
+            // The paper says nothing about NaN or Inf; they are compared like any other pattern,
+            // and counted (once per receiver slot the element maps to) so that a caller can notice.
+            const bool odd = !std::isfinite(theta[p][i]) || !std::isfinite(prev);
+            if (bt == bp && !odd) continue;
             // Eq. 5: u = unravel(i, n_s)
             const uint64_t u0 = i / n1, u1 = i % n1;
             for (uint64_t o : ops_of[p]) {
@@ -182,6 +186,8 @@ void* oracle_extract(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n
                 const uint64_t e0 = (uint64_t)op[4], e1 = (uint64_t)op[5];
                 // a_s <= u < a_s + e, component-wise
                 if (u0 < as0 || u0 >= as0 + e0 || u1 < as1 || u1 >= as1 + e1) continue;
+                if (odd) res->nonfinite += 1;
+                if (bt == bp) continue;
                 // Eq. 6: j = ravel(u - a_s + a_r, n_r)
                 const uint64_t j = (uint64_t)op[6] + (u0 - as0 + (uint64_t)op[8]) * (uint64_t)op[7] +
                                    (u1 - as1 + (uint64_t)op[9]);
@@ -236,6 +242,9 @@ void oracle_result_op_counts(void* h, uint64_t* out) {
     std::copy(r->op_count.begin(), r->op_count.end(), out);
 }
 
+// Scanned receiver slots whose theta_t or reconstructed theta_{t-1} is not finite.
+uint64_t oracle_result_nonfinite(void* h) { return ((Result*)h)->nonfinite; }
+
 void oracle_result_free(void* h) { delete (Result*)h; }
 
 // Eq. 7: vec(W_r)[I] <- V for every list.  Returns 0, or 1 if an index lies
@@ -253,7 +262,7 @@ int oracle_apply(uint64_t n_shards, const int64_t* shard_numel, const uint64_t* 
 }  // extern "C"
 
 // Destination-side mapping of canonical entries (Section 4.4: the storage-mediated path ships
-// canonical changes and "performs the final inference-layout mapping inside the destination").
+// canonical changes and leaves the mapping into the inference layout to the destination).
 // list p = changed flat indices i of canonical tensor p with their target values.  Literally
 // Eq. 5-7: for every entry, u = unravel(i, n_s); for every operation on tensor p in plan order
 // with a_s <= u < a_s + e: j = ravel(u - a_s + a_r, n_r) and shard[dst][j] <- value.  Operations

@@ -416,3 +416,37 @@ def test_canonical_mapping_skips_other_receivers_and_reports_bad_entries():
     bad[0] = plan.numel(0)                                   # one past the end of tensor 0
     with pytest.raises(ValueError):
         oracle.apply_canonical(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), lp, bad, val, shards)
+
+
+def test_nonfinite_slots_are_counted_once_per_receiver_copy():
+    """The count of receiver slots whose theta_t or reconstruction is NaN / Inf, against an
+    element-wise numpy fp32 evaluation of Eq. 2 (separately rounded operations) and the plan's
+    replication: a sharded tensor counts once, a replicated one once per receiver."""
+    rng = np.random.default_rng(5)
+    n = 4096
+    th = (rng.standard_normal(n) * 0.02).astype(np.float32)
+    mm = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+    vv = np.abs(rng.standard_normal(n) * 1e-6).astype(np.float32)
+    th[[3, 700]] = np.nan
+    th[[9, 1500]] = [np.inf, -np.inf]
+    vv[[20, 21, 3000]] = -1e-6                      # sqrt of a negative: NaN reconstruction
+    mm[[40, 41]] = [3e38, -3e38]                    # the update overflows: Inf reconstruction
+    vv[[40, 41]] = 1e-30
+    c = oracle.derive_constants(7, 1e-2, 0.9, 0.999, 1e-8, 0.1)
+    with np.errstate(all="ignore"):
+        mhat = mm / c[0]
+        den = np.sqrt(vv / c[1]) + c[4]
+        prev = (th + c[3] * (mhat / den)) / c[2]
+    odd = ~np.isfinite(th) | ~np.isfinite(prev)
+    assert odd.sum() == 9
+    # tensor 0: rows split over two receivers; tensor 1 (same data): replicated on three
+    shapes = [(64, 64), (64, 64)]
+    numels = [2048, 2048, 4096, 4096, 4096]
+    ops = [(0, 0, 0, 0, 32, 64, 0, 64, 0, 0), (0, 1, 32, 0, 32, 64, 0, 64, 0, 0)] + \
+          [(1, 2 + r, 0, 0, 64, 64, 0, 64, 0, 0) for r in range(3)]
+    res = oracle.extract(shapes, numels, ops, [th, th], [mm, mm], [vv, vv], c, with_nonfinite=True)
+    assert res[3] == int(odd.sum()) * (1 + 3)
+    # and nothing is counted when everything is finite
+    ok = np.where(odd, np.float32(0.01), th)
+    res = oracle.extract(shapes, numels, ops, [ok, ok], [np.zeros_like(mm)] * 2, [np.abs(vv)] * 2, c, with_nonfinite=True)
+    assert res[3] == 0
