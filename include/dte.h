@@ -119,7 +119,13 @@ typedef struct dte_layout dte_layout;
  * bit patterns of theta_t, Eq. 4).  Empty lists keep their slot.
  *   offsets  : capacity x uint32        values : capacity x uint16
  *   list_ptr : (n_shards + 1) x uint64
- *   counters : 4 x uint64 = { total changed, elements scanned, DTE_DEV_* bits, 0 }
+ *   counters : 4 x uint64 = { total changed, elements scanned, DTE_DEV_* bits, non-finite }
+ *              non-finite: scanned elements (a replicated element once per receiver) whose
+ *              reconstructed previous value broke - it is NaN (a NaN in theta or a moment, a
+ *              negative v, 0/0), or +-Inf although theta is finite (the update overflowed).  The
+ *              paper does not say what to do with such values; they are compared like any other
+ *              bit pattern, and counted here so that the caller can notice a diverged optimizer
+ *              state.  An infinite theta that stays infinite is not counted.
  * If the total exceeds `capacity`, DTE_DEV_OVERFLOW is set, offsets / values hold nothing
  * usable, and list_ptr / counters[0] still hold the exact sizes, so the caller can grow
  * the buffers and call again (Section 3: sizes are learnt in a step of their own, before

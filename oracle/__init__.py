@@ -168,7 +168,7 @@ def extract(tensor_shapes, shard_numels, ops, theta, m, v, consts, with_op_count
     out = (list_ptr, offsets, values)
     if with_op_counts:          # c_o per operation, plan order, zeros included (Section 4.3)
         out += (op_counts,)
-    if with_nonfinite:          # receiver slots whose theta_t or reconstruction is NaN / Inf
+    if with_nonfinite:          # receiver slots whose reconstruction is NaN, or Inf from a finite theta_t
         out += (nonfinite,)
     return out
 

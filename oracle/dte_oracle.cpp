@@ -79,7 +79,7 @@ struct Result {
     std::vector<uint64_t> list_ptr;   // n_shards + 1
     std::vector<uint32_t> offsets;
     std::vector<uint16_t> values;
-    uint64_t nonfinite = 0;           // scanned slots whose theta_t or reconstruction is NaN or +-Inf
+    uint64_t nonfinite = 0;           // scanned slots whose reconstruction broke: NaN, or +-Inf from a finite theta_t
     std::string error;
 };
 
@@ -174,9 +174,12 @@ void* oracle_extract(uint64_t n_tensors, const int64_t* tensor_shape, uint64_t n
             float prev = invert_one(theta[p][i], m[p][i], v[p][i], c);
             uint16_t bt = bf16_rne(theta[p][i]);
             uint16_t bp = bf16_rne(prev);
-            // The paper says nothing about NaN or Inf; they are compared like any other pattern,
-            // and counted (once per receiver slot the element maps to) so that a caller can notice.
-            const bool odd = !std::isfinite(theta[p][i]) || !std::isfinite(prev);
+            // The paper says nothing about NaN or Inf; they are compared like any other pattern.
+            // Reconstructions that broke - NaN (a NaN theta_t or moment, a negative v, 0/0), or an
+            // overflow to +-Inf from a finite theta_t - are counted, once per receiver slot the
+            // element maps to, so that a caller can notice; an infinite theta_t that stays
+            // infinite is a value the model already held and is not.
+            const bool odd = std::isnan(prev) || (std::isinf(prev) && std::isfinite(theta[p][i]));
             if (bt == bp && !odd) continue;
             // Eq. 5: u = unravel(i, n_s)
             const uint64_t u0 = i / n1, u1 = i % n1;
@@ -242,7 +245,7 @@ void oracle_result_op_counts(void* h, uint64_t* out) {
     std::copy(r->op_count.begin(), r->op_count.end(), out);
 }
 
-// Scanned receiver slots whose theta_t or reconstructed theta_{t-1} is not finite.
+// Scanned receiver slots whose reconstructed theta_{t-1} is NaN, or infinite from a finite theta_t.
 uint64_t oracle_result_nonfinite(void* h) { return ((Result*)h)->nonfinite; }
 
 void oracle_result_free(void* h) { delete (Result*)h; }

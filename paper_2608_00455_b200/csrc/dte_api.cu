@@ -84,11 +84,11 @@ Screen make_screen(const Consts& c) {
 // Where one extract call keeps its placement records, block sums, staging cursor and staged
 // entries: the layout's own buffers, or the fixed array of the allocation-free entry point.
 struct Scratch {
-    uint64_t* cursor;       // the staging cursor
+    uint64_t* cursor;       // two words: the staging cursor, the count of non-finite elements
     uint64_t* rec;
     uint64_t* block_sum;
     uint32_t* stage;
-    bool clear_first;       // the cursor is not known to be zero: clear it in the stream
+    bool clear_first;       // the two words are not known to be zero: clear them in the stream
 };
 
 // Enqueues the kernels of one extract: both extract launches (packed and regular tiles), then
@@ -106,7 +106,7 @@ dte_status enqueue_kernels(dte_layout* L, const Consts& c, const std::vector<Gro
         L->last_launch[0] = 0; L->last_launch[1] = 0; L->last_launch[2] = 0;
         return DTE_OK;
     }
-    if (sc.clear_first) DTE_CUDA(cudaMemsetAsync(sc.cursor, 0, sizeof(uint64_t), st));
+    if (sc.clear_first) DTE_CUDA(cudaMemsetAsync(sc.cursor, 0, 2 * sizeof(uint64_t), st));
     GatherParams g;
     g.rec = sc.rec;
     g.block_sum = sc.block_sum;

@@ -365,6 +365,7 @@ __device__ __forceinline__ void extract_tile(const ExtractParams& p, uint32_t in
         // ---- phase B: exact evaluation of the queue, 32 entries per round; the changed
         //      entries are compacted to the front of the queue as (index | value << 16) -----
         uint32_t n_changed = 0;
+        uint32_t n_odd = 0;     // this lane's elements whose reconstruction is NaN, or Inf from a finite theta
         // the loads of round r + 1 are issued before round r is evaluated (their latency is an
         // L2 hit, several hundred ns, and rounds are otherwise serial)
         uint32_t e_cur = 0;
@@ -391,6 +392,10 @@ __device__ __forceinline__ void extract_tile(const ExtractParams& p, uint32_t in
                 const uint32_t bt = bf16_rne_bits(tj), bp = bf16_rne_bits(prev);
                 changed = bt != bp;
                 entry = e_cur | (bt << 16);
+                // reconstructions that broke: NaN, or an overflow from a finite theta (every such
+                // element reaches this path: the screen's ordered compares fail on NaN and on an
+                // infinite bound; an infinite theta that stays infinite may pass it and is not counted)
+                n_odd += (prev != prev) | (isinf(prev) & (fabsf(tj) <= 3.402823466e38f));
             }
             // the ballot also orders this round's (and the next round's) queue reads before the
             // writes below, which land at or before slot q0 + 31
@@ -400,6 +405,11 @@ __device__ __forceinline__ void extract_tile(const ExtractParams& p, uint32_t in
             e_cur = e_nxt; tj = tn; mj = mn; vj = vn;
         }
         __syncwarp();
+        if (__any_sync(0xFFFFFFFFu, n_odd != 0)) {      // rare: one atomic per warp-tile that saw any
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) n_odd += __shfl_xor_sync(0xFFFFFFFFu, n_odd, d);
+            if (lane == 0) atomicAdd(p.cursor + 1, (unsigned long long)n_odd);
+        }
 
         // ---- phase C: one reservation per CTA, coalesced writes in tile order, the record -----
         if (lane == 0) s_count[warp] = n_changed;

@@ -109,7 +109,7 @@ struct GatherParams {
     uint64_t capacity;
     uint64_t* list_ptr;
     uint64_t* counters;
-    unsigned long long* cursor;      // staging cursor: left at zero for the next call
+    unsigned long long* cursor;      // staging cursor and non-finite count: left at zero for the next call
     // delivery to the receivers (dte_extract_delta_push); n_recv == 0: none
     uint32_t n_recv;
     const uint32_t* recv_first_list; // n_recv: first list of each receiver (then n_recv: one past its last)
@@ -126,7 +126,7 @@ struct ExtractParams {
     const float* const* theta;   // device table, n_tensors
     const float* const* m;
     const float* const* v;
-    unsigned long long* cursor;  // zeroed before launch: entries appended to the staging buffer
+    unsigned long long* cursor;  // [0] entries appended to the staging buffer, [1] non-finite elements seen; both rest at zero
     uint64_t* rec;               // n_tiles placement records (written in full)
     uint32_t* stage;             // staging buffer, stage_capacity words: tile-relative index | value << 16
     uint64_t stage_capacity;
@@ -240,7 +240,8 @@ __device__ __forceinline__ void gather_finish_totals(const GatherParams& p, uint
         p.counters[0] = total;
         p.counters[1] = p.scanned;
         p.counters[2] = total > p.capacity ? (uint64_t)DTE_DEV_OVERFLOW : 0ull;
-        p.counters[3] = 0;
+        p.counters[3] = __ldcg(p.cursor + 1);      // non-finite elements the extract counted (atomics: L2)
+        p.cursor[1] = 0ull;                         // ready for the next call
         p.list_ptr[p.n_lists] = total;
     }
     for (uint32_t k = tid; k < p.n_lists; k += n_threads)
@@ -299,7 +300,7 @@ struct dte_layout {
     dte::SegRec* d_segs = nullptr;
     uint64_t* d_rec = nullptr;             // n_tiles placement records
     uint64_t* d_block_sum = nullptr;       // one word per gather block
-    uint64_t* d_cursor = nullptr;          // staging cursor (rests at zero), a spare word, the ticket of the push's closing kernel
+    uint64_t* d_cursor = nullptr;          // staging cursor, non-finite count, ticket of the push's closing kernel: all rest at zero
     bool scratch_clean = false;            // the last call was enqueued completely, so they are at zero
     uint32_t* d_stage = nullptr;           // staging buffer, grown on demand to the caller's capacity
     uint64_t* d_rec_base = nullptr;        // n_tiles: destination base per placement record

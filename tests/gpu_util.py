@@ -19,7 +19,7 @@ def run_extract(plan, st, hp, capacity=None, layout=None, delta=None):
     return lay, d
 
 
-def oracle_extract(plan, st, hp, tensors=None):
+def oracle_extract(plan, st, hp, tensors=None, with_nonfinite=False):
     """Oracle on host copies.  With `tensors`, only those source tensors are evaluated
     (the other tensors' operations are dropped from the plan handed to the oracle)."""
     c = oracle.derive_constants(*hp.as_args())
@@ -34,7 +34,8 @@ def oracle_extract(plan, st, hp, tensors=None):
     def host(lst):
         return [lst[p].cpu().numpy() if p in need else zero for p in range(plan.n_tensors)]
 
-    return oracle.extract(shapes, plan.shard_numels, ops, host(st.theta), host(st.m), host(st.v), c)
+    return oracle.extract(shapes, plan.shard_numels, ops, host(st.theta), host(st.m), host(st.v), c,
+                          with_nonfinite=with_nonfinite)
 
 
 def assert_lists_equal(got, want, plan=None, lists=None):

@@ -100,11 +100,14 @@ def test_every_fp32_pattern_of_one_operand(which, hp):
         th, mm, vv = _operands(which, lo, CHUNK)
         mask, v16 = oracle.changed_mask(th, mm, vv, consts)
         idx = np.nonzero(mask)[0]
-        return lo, (idx + (lo % HALF)).astype(np.uint32), v16[idx]
+        prev = oracle.invert(th, mm, vv, consts)
+        odd = int((np.isnan(prev) | (np.isinf(prev) & np.isfinite(th))).sum())
+        return lo, (idx + (lo % HALF)).astype(np.uint32), v16[idx], odd
 
-    cursor = 0
+    cursor, odd_total = 0, 0
     with ThreadPoolExecutor(max_workers=os.cpu_count() or 4) as pool:
-        for lo, want_off, want_val in pool.map(job, range(0, N, CHUNK)):
+        for lo, want_off, want_val, odd in pool.map(job, range(0, N, CHUNK)):
+            odd_total += odd
             if lo == HALF:
                 assert cursor == int(lp[1]), "boundary between the two lists"
             n = want_off.size
@@ -115,3 +118,5 @@ def test_every_fp32_pattern_of_one_operand(which, hp):
             assert np.array_equal(val, want_val), f"values of chunk at {lo:#x}"
             cursor += n
     assert cursor == total
+    # reconstructions that are NaN (NaN operands, negative v, 0/0) or overflowed were all counted
+    assert int(d.counters[3].item()) == odd_total and odd_total >= (1 << 24)

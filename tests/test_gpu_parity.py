@@ -38,10 +38,12 @@ def _full_parity(wl, capacity=None):
     lay, d = run_extract(wl.plan, st, wl.hp, capacity)
     assert d.status_bits() == 0
     got = d.to_host()
-    want = oracle_extract(wl.plan, st, wl.hp)
+    *want, odd = oracle_extract(wl.plan, st, wl.hp, with_nonfinite=True)
+    want = tuple(want)
     assert_lists_equal(got, want, wl.plan)
     cnt = d.counters.cpu().numpy()
     assert cnt[0] == int(want[0][-1]) and cnt[1] == wl.plan.total_scanned_elements()
+    assert cnt[3] == odd, "count of non-finite elements"
     bufs = _apply_and_check(wl.plan, st, lay, d, got, want)
     return st, lay, d, got, bufs
 
@@ -90,7 +92,13 @@ def test_config5_edge_sweep_reduced_dims(point):
 
 def test_config5_nonfinite_robustness():
     wl = configs.config5(1e-4, 1, 0.1, 1e-2, dims=configs.SMALL_DENSE, nonfinite=True)
-    _full_parity(wl)
+    st, lay, d, got, bufs = _full_parity(wl)          # compares counters[3] with the oracle's count
+    assert int(d.counters[3].item()) >= 20               # the planted NaNs and infinities were seen
+    # and the count starts from zero on every call
+    run_extract(wl.plan, st, wl.hp, layout=lay, delta=d)
+    first = int(d.counters[3].item())
+    run_extract(wl.plan, st, wl.hp, layout=lay, delta=d)
+    assert int(d.counters[3].item()) == first
 
 
 def test_row_parallel_non_multiple_of_four_and_single_rows():
