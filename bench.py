@@ -624,6 +624,7 @@ def main():
     if bits:
         raise SystemExit(f"extract reported device status bits {bits} (capacity {delta.capacity}, total {delta.total()})")
     M = delta.total()
+    broken = int(delta.counters[3].item())      # reconstructions that came out NaN or overflowed
     lp_d = delta.list_ptr.cpu()
     init_vals = torch.empty(M, dtype=torch.int16, device=device)
     for k in range(plan.n_shards):
@@ -785,7 +786,8 @@ def main():
                          "kernel": "extract call (extract_kernel launches + scan + gather)",
                          "read_only_ceiling": ceiling,
                          "frac_of_read_only_ceiling": achieved / ceiling["GBps"] if ceiling else None},
-            "reconstruction_vs_truth": {"false_negatives": fn, "false_positives": fp, "variant": wl.variant},
+            "reconstruction_vs_truth": {"false_negatives": fn, "false_positives": fp, "variant": wl.variant,
+                                        "nan_or_overflowed_reconstructions": broken},
             "storage_path": codec, "push": push,
             "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": launches, "clocks": clocks,
             "launch": launch_info, **extra,
