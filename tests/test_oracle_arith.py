@@ -212,6 +212,27 @@ def test_bf16_rne_against_fp64_nearest_and_library_cast():
     assert (~finite_or_inf).sum() > 1000
 
 
+def test_bf16_rne_every_fp32_pattern_against_the_library_cast():
+    """All 2^32 inputs: the oracle's integer round-to-nearest-even equals torch's fp32 -> bf16 cast
+    on every pattern that is not a NaN, and gives 0x7FC0 on every NaN."""
+    import torch
+    chunk = 1 << 20          # small enough for the allocator to reuse its buffers
+    base = np.arange(chunk, dtype=np.uint32)
+    nans = 0
+    for lo in range(0, 1 << 32, chunk):
+        bits = base + np.uint32(lo)
+        got = oracle.bf16_rne(bits.view(np.float32))
+        lib = torch.from_numpy(bits.view(np.int32)).view(torch.float32).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        nan = (bits & np.uint32(0x7FFFFFFF)) > np.uint32(0x7F800000)
+        if nan.any():
+            assert np.all(got[nan] == 0x7FC0), hex(lo)
+            assert np.array_equal(got[~nan], lib[~nan]), hex(lo)
+            nans += int(nan.sum())
+        else:
+            assert np.array_equal(got, lib), hex(lo)
+    assert nans == 2 * ((1 << 23) - 1)
+
+
 def test_bf16_rne_named_cases():
     cases = {0x3F808000: 0x3F80, 0x3F818000: 0x3F82, 0x3F808001: 0x3F81, 0x3F807FFF: 0x3F80,
              0x7F7F8000: 0x7F80, 0x7F7F7FFF: 0x7F7F, 0xFF7F8000: 0xFF80, 0x00000000: 0x0000,
