@@ -322,6 +322,8 @@ __device__ __forceinline__ uint32_t phase_a(const WarpTile& cur, int lane, uint3
     return qn;
 }
 
+constexpr uint32_t kDescAhead = 4 * 148;   // CTAs resident at once: 4 per SM (registers and shared memory) on 148 SMs
+
 // One tile: `index` counts within the tiles of its kind.  GROUPS: the constants come from the
 // tile's parameter group instead of the kernel parameters.  EARLY: give the dependent-launch
 // signal at once instead of after the stream (see the kernels below).
@@ -338,6 +340,12 @@ __device__ __forceinline__ void extract_tile(const ExtractParams& p, uint32_t in
 
     WarpTile cur;
     uint32_t tile;
+    // A hint for the CTA that will take this one's place about one wave from now: its descriptor
+    // is the first link of its start-up chain (descriptor, source pointers, first chunk) and the
+    // only one that would otherwise come from DRAM.  Measured: 0.3 % of the step on the large
+    // workloads, 1 % on a single matrix.
+    if (!PACKED && threadIdx.x == 0 && index + kDescAhead < p.n_regular)
+        asm volatile("prefetch.global.L2 [%0];" ::"l"(p.tiles + index + kDescAhead));
     {
         const uint32_t tensor = decode<PACKED>(p, index, lane, warp, &s_geom[warp], cur, tile);
         if (GROUPS) {   // one 48-byte record per parameter group
