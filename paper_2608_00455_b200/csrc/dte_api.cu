@@ -64,6 +64,7 @@ dte_status sync_source_table(dte_layout* L, const float* const* theta, const flo
 //   kb    >= sqrt(bc2) * (1 + 2^-10)
 //   kc    >= 1 / eps                      (+inf when eps == 0)
 //   kappa >= (|1/decay - 1| + 2^-24) * (1 + 2^-7) * (1 + 2^-10)
+//   tiny  >= 2^-133 * kappa + 2^-148    (the absolute part of the decay bound, for subnormal ranges)
 float round_up(double x) {
     if (!(x == x)) return std::numeric_limits<float>::infinity();
     float f = (float)x;
@@ -78,6 +79,7 @@ Screen make_screen(const Consts& c) {
     s.kb = round_up(std::sqrt((double)c.bc2) * infl);
     s.kc = c.eps > 0.f ? round_up(1.0 / (double)c.eps) : std::numeric_limits<float>::infinity();
     s.kappa = round_up((std::fabs(1.0 / (double)c.decay - 1.0) + std::ldexp(1.0, -24)) * (1.0 + 1.0 / 128.0) * infl);
+    s.tiny = round_up(std::ldexp((double)s.kappa, -133) + std::ldexp(1.0, -148));
     return s;
 }
 

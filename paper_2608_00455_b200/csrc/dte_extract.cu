@@ -48,32 +48,42 @@ __device__ __forceinline__ uint32_t bf16_rne_bits(float x) {
 
 // ---- the screen --------------------------------------------------------------------
 //
-// Let a = |theta|, c = the BF16 value nearest to a, and lo < a < hi the two rounding
-// boundaries (tie points) around c, as fp32 numbers.  Any real x with lo < x < hi rounds (in
-// fp32, then in BF16) to c, because rounding is monotone.  The screen proves that the exact
-// quotient whose rounding is the reconstruction lies in [lo'', hi''] = [lo + 2 ulp, hi - 2 ulp]
-// (ulp = fp32 spacing at the boundary), hence the reconstruction has the BF16 pattern of
-// theta: unchanged, no exact evaluation needed.
-//
-// The bound mirrors Eq. 2 operation by operation and leans on the monotonicity of
-// round-to-nearest: if real x <= real y then RN(x) <= RN(y), overflow and underflow included.
-//     exact                      bound (all operands non-negative)
+// Most elements cannot have changed, and the screen proves it for them without the divisions and
+// the square root of Eq. 2.  It brackets the reconstruction between two fp32 numbers q and p and
+// casts both: if they have the same BF16 pattern, so has everything between them.  Every step
+// leans on one fact: round-to-nearest is monotone (real x <= y  =>  RN(x) <= RN(y), overflow and
+// underflow included), so a bound pushed through the SAME rounded operation stays a bound, with
+// no margin for rounding errors.
+//     exact                      bound (operands non-negative)
 //     mhat = RN(m / bc1)         A = RN(|m| * ka),        ka >= 1/bc1          => A >= |mhat|
 //     den  = RN(RN(sqrt(RN(v/bc2))) + eps)
 //                                W = min(|rsqrt(v)| * kb, kc),  kb >= sqrt(bc2)(1+2^-10),
 //                                    kc >= 1/eps                               => W >= 1/den
 //     u    = RN(mhat / den)      U = RN(A * W)                                 => U >= |u|
 //     s    = RN(lr * u)          S = RN(U * |lr|)                              => S >= |s|
-// so theta + s lies within S of theta, and num = RN(theta + s) stays in any fp32 interval
-// that contains [a - S, a + S].  For decay != 1, num/decay differs from theta by at most
-// S + a(1+2^-7)(|1/decay - 1| + 2^-24) <= B = fma(a, kappa, S) up to B's own rounding, which
-// is below one ulp and is absorbed by the second ulp of margin; the first ulp of margin
-// absorbs sub-ulp absolute errors in the subnormal range.  2^-10 in kb covers the 2^-22 error
-// of the hardware rsqrt and the rounding of RN(v/bc2), sqrt and the product.  rsqrt.ftz turns
-// subnormal v into +Inf, so W = kc there (den >= eps always); a negative subnormal v (whose
-// exact square root is NaN) becomes -0, then -Inf, and |B| = Inf.  NaN, Inf, negative v, zero
-// theta, an intermediate that overflows: all make B NaN / Inf or the room NaN (min.NaN and an
-// ordered compare), so those elements fall through to the exact path.
+// (2^-10 in kb covers the 2^-22 error of the hardware rsqrt and the roundings of v/bc2, of the
+// root and of the product; rsqrt.ftz turns a subnormal v into +Inf, so W = kc there, and
+// den >= eps always.)  The step s has the sign of lr * m, because den >= +0 or NaN.  Give S that
+// sign: theta + s lies between theta and theta + S, hence
+//     num = RN(theta + s)  lies between  theta  and  far = RN(theta + S)       (by value).
+// Without a division by decay the reconstruction is num: q = theta, p = far.
+// With it, recon = RN(num / decay) differs from num by at most
+//     |num| |1/decay - 1|  +  2^-24 |num| / decay  (rounding; 2^-150 if the quotient is subnormal).
+// If q and p (below) cast to the same BF16 pattern then theta and far, which lie between them,
+// are in one BF16 rounding cell, so |num| <= |theta| (1 + 2^-7) where BF16 is normal and
+// |num| <= |theta| + 2^-133 (a subnormal cell's width) where it is not.  With
+//     kappa >= (|1/decay - 1| + 2^-24)(1 + 2^-7)(1 + 2^-10),   tiny >= 2^-133 kappa + 2^-148,
+//     D = RN(|theta| kappa + tiny)   (one fma; its own rounding is inside the 2^-10 and the 2^-148)
+// recon lies within D of num, so between the reals theta - D and theta + S + D (signs as for S), and,
+// being an fp32 number, between their roundings
+//     q = RN(theta - D),   p = RN(far + D).
+// Equal values may still differ in pattern as +0 and -0; a reconstruction of -0 needs theta = -0
+// and a step of -0, and then q or p is -0 or negative too.  Elements whose reconstruction is
+// infinite or NaN must reach the exact path (it counts them): then p or q is infinite or NaN
+// (monotonicity again; NaN arises only from NaN or infinite operands, which make S, far or D
+// NaN or infinite), so a non-finite p or q never passes.  Everything else that is odd - negative
+// v (W = -Inf or NaN), v = 0 with eps = 0, overflowing intermediates - makes S infinite or NaN and
+// ends the same way.
 __device__ __forceinline__ float min_nan(float x, float y) {
     float r;
     asm("min.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(x), "f"(y));
@@ -84,56 +94,31 @@ __device__ __forceinline__ float rsqrt_ftz(float x) {
     asm("rsqrt.approx.ftz.f32 %0, %1;" : "=f"(r) : "f"(x));
     return r;
 }
+// Two BF16 casts (round to nearest even, subnormals kept, any NaN -> 0x7FFF) in one instruction.
+// Only equality of the two halves is used, and never when either is NaN or infinite; the values
+// that are emitted come from bf16_rne_bits.
+__device__ __forceinline__ uint32_t bf16x2_rn(float hi, float lo) {
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
 
 template <bool DIV_BC1, bool DIV_DECAY>
 __device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s, float lr) {
-    // boundaries from the raw pattern: the sign bit rides along (no carry reaches it below the NaN
-    // range) and is dropped by the |.| operand modifiers, which cost nothing
-    const uint32_t u = __float_as_uint(theta);
-    const float at = fabsf(theta);
-    // the step lr * u has the sign of lr * m (den >= +0 or NaN): sign bit of x set <=> it shrinks |theta|
-    const uint32_t x = u ^ __float_as_uint(m) ^ __float_as_uint(lr);
-    if (DIV_DECAY) {
-        // The step moves |theta| by at most S in a KNOWN direction; the division by decay then
-        // moves it by at most D = a(1+2^-7)(|1/decay - 1| + 2^-24) in either direction.  So the
-        // boundary the step moves towards must be further than S + D, the other one further than
-        // D only - a few ulps, which nearly always holds.  (Testing both sides against S + D sent
-        // about twice as many elements to the exact path.)  A step larger than the room on its
-        // side fails there, so it cannot flip the sign either.
-        const uint32_t hi = ((u + 0x8000u) & 0xFFFF0000u) | 0x7FFEu;   // boundary above |theta|, minus 2 ulp
-        const uint32_t lo = hi - 0xFFFCu;                               // boundary below, plus 2 ulp
-        const float room_up = fabsf(__uint_as_float(hi)) - at;          // exact differences; NaN for theta = 0,
-        const float room_dn = at - fabsf(__uint_as_float(lo));          // Inf, NaN; a tie has room_dn < 0
-        const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
-        const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);   // -Inf for v = -0 or a negative subnormal
-        const float sa = fabsf(__fmul_rn(__fmul_rn(am, w), fabsf(lr))); // |.|: a negative v must not pass
-        const float d_only = __fmul_rn(at, s.kappa);
-        const float s_and_d = __fmaf_rn(at, s.kappa, sa);
-        const bool down = (int32_t)x < 0;
-        // ordered, strict compares: NaN anywhere fails, and an infinite bound never passes
-        return (down ? d_only : s_and_d) < room_up && (down ? s_and_d : d_only) < room_dn;
-    }
-    float room;
-    {
-        // Without it the reconstruction is RN(theta + lr * u) and u has the sign of m (den >= +0 or
-        // NaN), so the direction is known: |theta| grows when theta and lr * m agree in sign and
-        // shrinks otherwise, and only the boundary on that side matters.  This halves the elements
-        // that reach the exact path (a step larger than the distance to the boundary BEHIND it
-        // cannot change the pattern).  A theta exactly on a tie point belongs to the cell above or
-        // below it depending on parity; each direction takes the cell that has the tie as its
-        // boundary on that side, so a tie never passes.
-        const bool down = (int32_t)x < 0;
-        const uint32_t cell = (u + (down ? 0x8000u : 0x7FFFu)) & 0xFFFF0000u;
-        const uint32_t bnd = down ? cell - 0x7FFEu : cell + 0x7FFEu;       // 2 ulp inside the boundary
-        const float d = fabsf(__uint_as_float(bnd)) - at;                  // exact; negative on the lower side
-        room = __uint_as_float(__float_as_uint(d) ^ (x & 0x80000000u));    // distance to that boundary (or NaN)
-    }
     const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
-    const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);   // -Inf for v = -0 or a negative subnormal
-    const float b = __fmul_rn(__fmul_rn(am, w), fabsf(lr));
-    // |b|: a negative v (w = -Inf or NaN) must not pass.  Strict: theta = +-Inf has room = +Inf on
-    // its lower side, and an infinite bound (the step may be -Inf, the sum NaN) must not pass it.
-    return fabsf(b) < room;
+    const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);      // -Inf for v = -0 or a negative subnormal
+    const float sb = __fmul_rn(__fmul_rn(am, w), fabsf(lr));           // S, or -Inf / NaN
+    const uint32_t dir = (__float_as_uint(m) ^ __float_as_uint(lr)) & 0x80000000u;   // sign of the step
+    const float far = __fadd_rn(theta, __uint_as_float((__float_as_uint(sb) & 0x7FFFFFFFu) | dir));
+    if (DIV_DECAY) {
+        const float d = __uint_as_float(__float_as_uint(__fmaf_rn(fabsf(theta), s.kappa, s.tiny)) | dir);
+        const uint32_t r = bf16x2_rn(__fadd_rn(far, d), __fsub_rn(theta, d));
+        // halves equal, and (one test for both then) neither infinite nor NaN
+        return r == __byte_perm(r, 0, 0x1032) && (r << 1) < 0xFF000000u;
+    }
+    const uint32_t r = bf16x2_rn(far, theta);
+    // far is at least as extreme as theta: finite far, finite both (ordered compare: NaN fails)
+    return r == __byte_perm(r, 0, 0x1032) && fabsf(far) < __int_as_float(0x7F800000);
 }
 
 __device__ __forceinline__ const float* ldg_ptr(const float* const* slot) {
@@ -354,7 +339,7 @@ __device__ __forceinline__ void extract_tile(const ExtractParams& p, uint32_t in
             c.bc1 = __uint_as_float(g0.x); c.bc2 = __uint_as_float(g0.y); c.decay = __uint_as_float(g0.z);
             c.lr = __uint_as_float(g0.w); c.eps = __uint_as_float(g1.x);
             sc.ka = __uint_as_float(g1.y); sc.kb = __uint_as_float(g1.z); sc.kc = __uint_as_float(g1.w);
-            sc.kappa = __uint_as_float(g2.x);
+            sc.kappa = __uint_as_float(g2.x); sc.tiny = __uint_as_float(g2.y);
         }
 
         const float lr = c.lr;

@@ -83,14 +83,14 @@ struct Consts {
 
 // Constants of the conservative "cannot have changed" screen (see dte_extract.cu).
 struct Screen {
-    float ka, kb, kc, kappa;
+    float ka, kb, kc, kappa, tiny;
 };
 
 // Per-parameter-group constants (exact path + screen), read with three 16-byte loads.
 struct __align__(16) GroupConsts {
     Consts c;
     Screen s;
-    float pad[3];
+    float pad[2];
 };
 static_assert(sizeof(GroupConsts) == 48, "GroupConsts is read as three uint4");
 

@@ -39,6 +39,27 @@ def _near_boundary_state(n, hp: Hyper, seed, spread_ulps=24, with_specials=True)
     return theta, m, v
 
 
+def _run_and_compare(plan, hp, theta, m, v, n):
+    """Lists bit-exact against the oracle, and the count of broken reconstructions too (every
+    element whose reconstruction is NaN or overflowed has to reach the exact path to be counted)."""
+    c = oracle.derive_constants(*hp.as_args())
+    with np.errstate(all="ignore"):
+        *want, odd = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), [theta], [m], [v], c,
+                                    with_nonfinite=True)
+    lay = dte.Layout.from_plan(plan, 0)
+    d = lay.new_delta(n)
+    t, mm, vv = (torch.from_numpy(a.copy()).cuda() for a in (theta, m, v))
+    dte.dte_extract_delta(lay, lay.source_tables([t], [mm], [vv]), *hp.as_args(), d)
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    lp, off, val = d.to_host()
+    assert np.array_equal(lp, want[0])
+    assert np.array_equal(off, want[1])
+    assert np.array_equal(val, want[2])
+    assert int(d.counters[3].item()) == int(odd)
+    return int(lp[-1]) / n, int(odd)
+
+
 @pytest.mark.parametrize("hp", [
     Hyper(step=500, lr=1e-6, wd=0.01),        # bc1 == 1, decay == 1
     Hyper(step=100, lr=1e-6, wd=0.01),        # bc1 != 1, decay == 1
@@ -52,19 +73,7 @@ def test_screen_threshold_cases_match_oracle(hp):
     n = rows * cols
     theta, m, v = _near_boundary_state(n, hp, seed=hp.step)
     plan = plans.single_matrix_plan(rows, cols, 2)
-    c = oracle.derive_constants(*hp.as_args())
-    want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), [theta], [m], [v], c)
-    lay = dte.Layout.from_plan(plan, 0)
-    d = lay.new_delta(n)
-    t, mm, vv = (torch.from_numpy(a).cuda() for a in (theta, m, v))
-    dte.dte_extract_delta(lay, lay.source_tables([t], [mm], [vv]), *hp.as_args(), d)
-    torch.cuda.synchronize()
-    assert d.status_bits() == 0
-    lp, off, val = d.to_host()
-    assert np.array_equal(lp, want[0])
-    assert np.array_equal(off, want[1])
-    assert np.array_equal(val, want[2])
-    frac = int(lp[-1]) / n
+    frac, _ = _run_and_compare(plan, hp, theta, m, v, n)
     assert 0.05 < frac < 0.95, frac            # the cases really straddle the decision
 
 
@@ -96,26 +105,18 @@ def test_random_bit_patterns_match_oracle(hp):
     m[:k] = (rng.standard_normal(k) * 10.0 ** rng.uniform(-12, 2, k)).astype(np.float32)
     v[:k] = np.abs(rng.standard_normal(k) * 10.0 ** rng.uniform(-20, 2, k)).astype(np.float32)
     plan = plans.single_matrix_plan(rows, cols, 2)
-    c = oracle.derive_constants(*hp.as_args())
-    with np.errstate(all="ignore"):
-        want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), [theta], [m], [v], c)
-    lay = dte.Layout.from_plan(plan, 0)
-    d = lay.new_delta(n)
-    t, mm, vv = (torch.from_numpy(a.copy()).cuda() for a in (theta, m, v))
-    dte.dte_extract_delta(lay, lay.source_tables([t], [mm], [vv]), *hp.as_args(), d)
-    torch.cuda.synchronize()
-    lp, off, val = d.to_host()
-    assert np.array_equal(lp, want[0]) and np.array_equal(off, want[1]) and np.array_equal(val, want[2])
-    assert 0.3 < int(lp[-1]) / n <= 1.0
+    frac, odd = _run_and_compare(plan, hp, theta, m, v, n)
+    assert odd > n // 8                               # NaN operands, negative second moments, overflows
+    assert 0.3 < frac <= 1.0
 
 
-def _wide_exponent_threshold_state(n, hp: Hyper, seed):
+def _wide_exponent_threshold_state(n, hp: Hyper, seed, upper_range=(0x0000, 0x7F80)):
     """Like the near-boundary state, but over EVERY binade of theta and of the second moment:
     theta a few ulps off a BF16 tie point with any exponent (subnormals included), v with any
     exponent, m solved (in double) so that the update is 1/8 .. 8 times the distance to the tie -
     where that needs an m, m-hat or u beyond fp32's range it overflows or underflows, on purpose."""
     rng = np.random.default_rng(seed)
-    upper = rng.integers(0x0000, 0x7F80, size=n, dtype=np.uint32)
+    upper = rng.integers(upper_range[0], upper_range[1], size=n, dtype=np.uint32)
     sign = rng.integers(0, 2, size=n, dtype=np.uint32) << 31
     delta = rng.integers(-40, 41, size=n).astype(np.int64)
     bits = np.clip((upper.astype(np.int64) << 16) + 0x8000 + delta, 0, 0x7F7FFFFF).astype(np.uint32) | sign
@@ -149,14 +150,79 @@ def test_threshold_cases_in_every_binade_match_oracle(hp):
     n = rows * cols
     theta, m, v = _wide_exponent_threshold_state(n, hp, seed=1000 + hp.step)
     plan = plans.single_matrix_plan(rows, cols, 2)
-    c = oracle.derive_constants(*hp.as_args())
+    frac, _ = _run_and_compare(plan, hp, theta, m, v, n)
+    assert 0.02 < frac < 0.98
+
+
+@pytest.mark.parametrize("hp", [
+    Hyper(step=500, lr=1e-6, wd=0.01),                 # theta beyond the last BF16 tie point casts to Inf, and so does its reconstruction
+    Hyper(step=20, lr=30.0, wd=0.0, eps=1e-3),         # theta + lr * u overflows
+    Hyper(step=20, lr=0.5, wd=1.0),                    # the division by decay = 0.5 overflows
+    Hyper(step=20, lr=30.0, wd=0.01),                  # both can
+    Hyper(step=20, lr=-4.0, wd=1.0),                   # decay = 5: a finite sum shrinks, one that overflowed stays infinite
+], ids=lambda h: f"t{h.step}-lr{h.lr:g}-wd{h.wd:g}-eps{h.eps:g}")
+def test_reconstructions_at_the_top_of_the_range_match_oracle(hp):
+    """theta in the last binades of fp32 (up to the largest finite value, past the last BF16 tie
+    point), steps from negligible to several times theta: reconstructions that stay finite, that
+    overflow in the sum, and that overflow in the division by decay.  The lists and the count of
+    overflowed reconstructions must both match."""
+    rows, cols = 2048, 2048
+    n = rows * cols
+    rng = np.random.default_rng(4242 + hp.step + int(hp.lr * 10) % 97)
+    upper = rng.integers(0x7E00, 0x7F80, size=n, dtype=np.uint32)
+    low = rng.integers(0, 1 << 16, size=n, dtype=np.uint32)
+    sign = rng.integers(0, 2, size=n, dtype=np.uint32) << 31
+    theta = ((upper << 16) | low | sign).view(np.float32).copy()
+    theta[: n // 16] = np.float32(3.4028234663852886e38) * rng.choice([-1.0, 1.0], size=n // 16).astype(np.float32)
+    v = (2.0 ** rng.uniform(-20, 20, size=n)).astype(np.float32)
+    c = oracle.derive_constants(*hp.as_args()).astype(np.float64)
     with np.errstate(all="ignore"):
-        want = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), [theta], [m], [v], c)
-    lay = dte.Layout.from_plan(plan, 0)
-    d = lay.new_delta(n)
-    t, mm, vv = (torch.from_numpy(a.copy()).cuda() for a in (theta, m, v))
-    dte.dte_extract_delta(lay, lay.source_tables([t], [mm], [vv]), *hp.as_args(), d)
-    torch.cuda.synchronize()
-    lp, off, val = d.to_host()
-    assert np.array_equal(lp, want[0]) and np.array_equal(off, want[1]) and np.array_equal(val, want[2])
-    assert 0.02 < int(lp[-1]) / n < 0.98
+        step = np.abs(theta).astype(np.float64) * 2.0 ** rng.uniform(-30, 4, size=n) * rng.choice([-1.0, 1.0], size=n)
+        m = (step / abs(c[3]) * (np.sqrt(v.astype(np.float64) / c[1]) + c[4]) * c[0]).astype(np.float32)
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    frac, odd = _run_and_compare(plan, hp, theta, m, v, n)
+    if hp.lr >= 0.5 or hp.lr < 0:
+        assert odd > n // 100, odd            # overflows really happen
+    assert 0.001 < frac <= 1.0
+
+
+@pytest.mark.parametrize("hp", [
+    Hyper(step=20, lr=0.1, wd=1.0),                    # decay = 0.9
+    Hyper(step=20, lr=0.25, wd=1.0),                   # 0.75
+    Hyper(step=20, lr=0.5, wd=1.0),                    # 0.5: the division moves theta by as much as theta
+    Hyper(step=20, lr=0.999, wd=1.0),                  # 0.001
+    Hyper(step=20, lr=-0.1, wd=1.0),                   # 1.1
+    Hyper(step=20, lr=-4.0, wd=1.0),                   # 5
+    Hyper(step=20, lr=1e-3, wd=0.2),                   # 0.9998
+    Hyper(step=20, lr=1e-5, wd=1.0),                   # 0.99999
+], ids=lambda h: f"lr{h.lr:g}-wd{h.wd:g}")
+@pytest.mark.parametrize("still", [False, True], ids=["step", "no-step"])
+def test_division_by_decay_where_bf16_is_subnormal_matches_oracle(hp, still):
+    """theta in the fp32-subnormal, BF16-subnormal and first normal binades, where a BF16 rounding
+    cell is as wide as the values in it and the rounding error of the division is absolute, not
+    relative: a division by a decay well away from 1 leaves many of these elements in their cell,
+    so the decision is taken at its threshold there (in the normal range such a decay changes
+    everything).  Once with steps of about the distance to the tie point, once with m = 0, which
+    leaves the division alone."""
+    rows, cols = 2048, 2048
+    n = rows * cols
+    seed = 77 + int(abs(hp.lr) * 1e5) % 1000
+    theta, m, v = _wide_exponent_threshold_state(n, hp, seed=seed, upper_range=(0x0000, 0x0100))
+    # half of the elements anywhere in the sixteen lowest BF16 cells instead of next to a tie point:
+    # there the distance to the tie is of the size of the division's shift
+    rng = np.random.default_rng(seed + 1)
+    k = n // 2
+    bits = (rng.integers(0x0000, 0x0010, size=k, dtype=np.uint32) << 16) | rng.integers(0, 1 << 16, size=k, dtype=np.uint32)
+    theta[:k] = (bits | (rng.integers(0, 2, size=k, dtype=np.uint32) << 31)).view(np.float32)
+    # ... with steps of up to a cell and a half, so that theta and theta + step can sit at opposite
+    # ends of one cell (a step of next to nothing relative to anything normal, but here the sum
+    # is up to three times theta, and the division's shift grows with it)
+    c = oracle.derive_constants(*hp.as_args()).astype(np.float64)
+    v[:k] = (2.0 ** rng.uniform(20, 60, size=k)).astype(np.float32)
+    step = rng.uniform(-1.5, 1.5, size=k) * 2.0 ** -133
+    m[:k] = (step / abs(c[3]) * (np.sqrt(v[:k].astype(np.float64) / c[1]) + c[4]) * c[0]).astype(np.float32)
+    if still:
+        m[:] = 0.0
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    frac, _ = _run_and_compare(plan, hp, theta, m, v, n)
+    assert 0.01 < frac < 1.0
