@@ -226,3 +226,31 @@ def test_division_by_decay_where_bf16_is_subnormal_matches_oracle(hp, still):
     plan = plans.single_matrix_plan(rows, cols, 2)
     frac, _ = _run_and_compare(plan, hp, theta, m, v, n)
     assert 0.01 < frac < 1.0
+
+
+@pytest.mark.parametrize("hp", [
+    Hyper(step=500, lr=1e-6, wd=0.01),
+    Hyper(step=3, lr=1e-3, wd=0.2),
+    Hyper(step=20, lr=1e-3, wd=1.0),                   # decay = 0.999: a shift of a quarter of a BF16 cell
+    Hyper(step=20, lr=-1e-3, wd=0.5),
+    Hyper(step=7, lr=1e-3, wd=0.0, eps=0.0),
+], ids=lambda h: f"t{h.step}-lr{h.lr:g}-wd{h.wd:g}-eps{h.eps:g}")
+def test_steps_of_every_relative_size_in_every_binade_match_oracle(hp):
+    """theta anywhere (every binade, every position in its BF16 cell), the step from 2^-30 of
+    theta to 16 times theta and of either sign: elements that cannot change, that sit at the
+    threshold, that cancel to zero or flip their sign."""
+    rows, cols = 2048, 4096
+    n = rows * cols
+    rng = np.random.default_rng(31337 + hp.step)
+    upper = rng.integers(0x0000, 0x7F80, size=n, dtype=np.uint32)
+    theta = ((upper << 16) | rng.integers(0, 1 << 16, size=n, dtype=np.uint32)
+             | (rng.integers(0, 2, size=n, dtype=np.uint32) << 31)).view(np.float32).copy()
+    v = (2.0 ** rng.uniform(-60, 60, size=n)).astype(np.float32)
+    c = oracle.derive_constants(*hp.as_args()).astype(np.float64)
+    with np.errstate(all="ignore"):
+        step = np.abs(theta).astype(np.float64) * 2.0 ** rng.uniform(-30, 4, size=n) * rng.choice([-1.0, 1.0], size=n)
+        step[: n // 32] = -theta[: n // 32].astype(np.float64)            # exact cancellation
+        m = (step / c[3] * (np.sqrt(v.astype(np.float64) / c[1]) + c[4]) * c[0]).astype(np.float32)
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    frac, _ = _run_and_compare(plan, hp, theta, m, v, n)
+    assert 0.2 < frac < 0.9
