@@ -254,3 +254,47 @@ def test_steps_of_every_relative_size_in_every_binade_match_oracle(hp):
     plan = plans.single_matrix_plan(rows, cols, 2)
     frac, _ = _run_and_compare(plan, hp, theta, m, v, n)
     assert 0.2 < frac < 0.9
+
+
+def _random_hyper(rng) -> Hyper:
+    """Hyper-parameters from all over the accepted range (lr * wd < 1, betas in [0, 1), eps >= 0)."""
+    lr = float(10.0 ** rng.uniform(-10, 1)) * (1.0 if rng.random() < 0.85 else -1.0)
+    wd = float(rng.choice([0.0, 10.0 ** rng.uniform(-4, 0.3)]))
+    if lr * wd >= 0.999:
+        wd = 0.5 / abs(lr)
+    eps = float(rng.choice([0.0, 1e-8, 10.0 ** rng.uniform(-30, -1)]))
+    beta1 = float(rng.choice([0.0, 0.9, rng.uniform(0.0, 0.9999)]))
+    beta2 = float(rng.choice([0.5, 0.999, rng.uniform(0.1, 0.99999)]))
+    step = int(rng.choice([1, 2, 10, 100, 500, 5000, int(rng.integers(1, 20000))]))
+    return Hyper(step=step, lr=lr, wd=wd, beta1=beta1, beta2=beta2, eps=eps)
+
+
+@pytest.mark.parametrize("seed", range(32))
+def test_random_hyperparameters_match_oracle(seed):
+    """The screen's constants are derived from the call's hyper-parameters on the host; here those
+    are random, and the state mixes the adversarial kinds above: threshold cases in every binade,
+    raw bit patterns, the lowest BF16 cells with steps of about a cell, and plausible weights."""
+    rng = np.random.default_rng(9000 + seed)
+    hp = _random_hyper(rng)
+    rows, cols = 1024, 2048
+    n = rows * cols
+    q = n // 4
+    theta, m, v = _wide_exponent_threshold_state(n, hp, seed=seed)
+    # raw bit patterns
+    for a in (theta, m, v):
+        a[q:2 * q] = rng.integers(0, 1 << 32, size=q, dtype=np.uint64).astype(np.uint32).view(np.float32)
+    v[q:q + q // 2] = np.abs(v[q:q + q // 2])
+    c = oracle.derive_constants(*hp.as_args()).astype(np.float64)
+    with np.errstate(all="ignore"):
+        # the sixteen lowest BF16 cells, steps of up to a cell and a half
+        bits = (rng.integers(0, 0x10, size=q, dtype=np.uint32) << 16) | rng.integers(0, 1 << 16, size=q, dtype=np.uint32)
+        theta[2 * q:3 * q] = (bits | (rng.integers(0, 2, size=q, dtype=np.uint32) << 31)).view(np.float32)
+        v[2 * q:3 * q] = (2.0 ** rng.uniform(20, 60, size=q)).astype(np.float32)
+        step = rng.uniform(-1.5, 1.5, size=q) * 2.0 ** -133
+        m[2 * q:3 * q] = (step / abs(c[3]) * (np.sqrt(v[2 * q:3 * q].astype(np.float64) / c[1]) + c[4]) * c[0]).astype(np.float32)
+        # plausible weights and moments
+        theta[3 * q:] = (rng.standard_normal(n - 3 * q) * 0.02).astype(np.float32)
+        m[3 * q:] = (rng.standard_normal(n - 3 * q) * 1e-4).astype(np.float32)
+        v[3 * q:] = np.abs(rng.standard_normal(n - 3 * q) * 1e-6).astype(np.float32)
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    _run_and_compare(plan, hp, theta, m, v, n)
