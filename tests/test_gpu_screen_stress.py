@@ -298,3 +298,49 @@ def test_random_hyperparameters_match_oracle(seed):
         v[3 * q:] = np.abs(rng.standard_normal(n - 3 * q) * 1e-6).astype(np.float32)
     plan = plans.single_matrix_plan(rows, cols, 2)
     _run_and_compare(plan, hp, theta, m, v, n)
+
+
+@pytest.mark.parametrize("seed", range(8))
+def test_random_learning_rates_and_weight_decays_per_group_match_oracle(seed):
+    """Four tensors in four parameter groups with a learning rate and a weight decay each: groups
+    whose decay rounds to 1 next to groups whose decay is far from it, in one call (the kernel then
+    takes every constant, the screen's included, from the tile's group)."""
+    rng = np.random.default_rng(12000 + seed)
+    base = _random_hyper(rng)
+    lrs, wds = [], []
+    for g in range(4):
+        h = _random_hyper(rng)
+        lrs.append(h.lr if g else 1e-6)          # group 0: lr * wd below 2^-25, decay == 1
+        wds.append(h.wd if g else 0.01)
+    rows, cols = 512, 2048
+    n = rows * cols
+    plan = plans.Plan()
+    for g in range(4):
+        t = plan.add_tensor(f"w{g}", (rows, cols))
+        for r in range(2):
+            k = plan.add_shard(f"w{g}.{r}", r, n // 2)
+            plan.add_op(t, k, (r * rows // 2, 0), (rows // 2, cols), 0, cols, (0, 0))
+    thetas, ms, vs = [], [], []
+    for g in range(4):
+        hp = Hyper(step=base.step, lr=lrs[g], wd=wds[g], beta1=base.beta1, beta2=base.beta2, eps=base.eps)
+        theta, m, v = _wide_exponent_threshold_state(n, hp, seed=100 * seed + g)
+        q = n // 2
+        theta[q:] = (rng.standard_normal(n - q) * 0.02).astype(np.float32)
+        m[q:] = (rng.standard_normal(n - q) * 1e-4).astype(np.float32)
+        v[q:] = np.abs(rng.standard_normal(n - q) * 1e-6).astype(np.float32)
+        thetas.append(theta); ms.append(m); vs.append(v)
+    consts = np.stack([oracle.derive_constants(base.step, lrs[g], base.beta1, base.beta2, base.eps, wds[g])
+                       for g in range(4)])
+    with np.errstate(all="ignore"):
+        *want, odd = oracle.extract(plan.tensor_shapes, plan.shard_numels, plan.ops_array(), thetas, ms, vs, consts,
+                                    with_nonfinite=True)
+    lay = dte.Layout.from_plan(plan, 0, tensor_groups=[0, 1, 2, 3])
+    d = lay.new_delta(4 * n)
+    dev = lambda lst: [torch.from_numpy(a.copy()).cuda() for a in lst]
+    tabs = lay.source_tables(dev(thetas), dev(ms), dev(vs))
+    dte.dte_extract_delta_groups(lay, tabs, base.step, base.beta1, base.beta2, base.eps, lrs, wds, d)
+    torch.cuda.synchronize()
+    assert d.status_bits() == 0
+    lp, off, val = d.to_host()
+    assert np.array_equal(lp, want[0]) and np.array_equal(off, want[1]) and np.array_equal(val, want[2])
+    assert int(d.counters[3].item()) == int(odd)
