@@ -237,7 +237,7 @@ extern "C" dte_status dte_extract_delta_groups(const dte_layout* layout, const f
         if (s != DTE_OK) return s;
         groups[gi].c = Consts{c5[0], c5[1], c5[2], c5[3], c5[4]};
         groups[gi].s = make_screen(groups[gi].c);
-        groups[gi].pad[0] = groups[gi].pad[1] = groups[gi].pad[2] = 0.f;
+        for (float& x : groups[gi].pad) x = 0.f;
     }
     dte_layout* L = const_cast<dte_layout*>(layout);
     DeviceGuard g(L->device);
