@@ -428,11 +428,11 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
         guard(upload(&L->d_tensor_group, grp));
     }
     if (st == DTE_OK) {
-        const size_t n_rec = n_ctas;
-        const size_t n_blocks = (n_rec + kRecsPerBlock - 1) / kRecsPerBlock;
-        cudaError_t e = cudaMalloc((void**)&L->d_rec, std::max<size_t>(1, n_rec) * sizeof(uint64_t));
+        const size_t n_records = n_ctas;
+        const size_t n_blocks = (n_records + kRecsPerBlock - 1) / kRecsPerBlock;
+        cudaError_t e = cudaMalloc((void**)&L->d_rec, std::max<size_t>(1, n_records) * sizeof(uint64_t));
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_block_sum, std::max<size_t>(1, n_blocks) * sizeof(uint64_t));
-        // cursor, extract ticket, push ticket, spare: all rest at zero
+        // staging cursor, count of non-finite elements, push ticket, spare: all rest at zero
         if (e == cudaSuccess) e = cudaMalloc((void**)&L->d_cursor, 4 * sizeof(uint64_t));
         if (e == cudaSuccess) e = cudaMemset(L->d_cursor, 0, 4 * sizeof(uint64_t));
         if (e == cudaSuccess) L->scratch_clean = true;
