@@ -388,9 +388,10 @@ extern "C" dte_status dte_layout_create(const dte_tensor_desc* tensors, size_t n
             }
     }
     {   // receivers: who owns which list, tile and operation (used by dte_extract_delta_push only)
-        uint32_t n_recv = 0;
-        for (size_t k = 0; k < n_shards; ++k) n_recv = std::max(n_recv, shards[k].receiver + 1);
-        if (n_shards && n_recv <= 65535) {
+        uint64_t max_recv = 0;       // 64 bits: a receiver id of 2^32 - 1 must not wrap to a count of zero
+        for (size_t k = 0; k < n_shards; ++k) max_recv = std::max<uint64_t>(max_recv, (uint64_t)shards[k].receiver + 1);
+        if (n_shards && max_recv <= 65535) {
+            const uint32_t n_recv = (uint32_t)max_recv;
             L->n_receivers = n_recv;
             // [0, n_recv): first list of each receiver; [n_recv, 2 n_recv): one past its last list
             // (both 0 for a receiver without shards: an empty slice)

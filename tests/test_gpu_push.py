@@ -183,6 +183,31 @@ def test_push_needs_consecutive_shards_per_receiver():
     assert e.value.status == 2
 
 
+def test_receiver_ids_beyond_the_push_tables_leave_the_layout_usable_without_push():
+    """`receiver` is informational for extract and apply; ids above 65534 (2^32 - 1 included, which
+    must not wrap to a receiver count of zero) only switch the push off."""
+    for rid in (65535, 0xFFFFFFFF):
+        p = plans.Plan()
+        a = p.add_tensor("a", (64, 64))
+        k0 = p.add_shard("r0.a", 0, 2048)
+        k1 = p.add_shard("far.a", rid, 2048)
+        p.add_op(a, k0, (0, 0), (32, 64), 0, 64, (0, 0))
+        p.add_op(a, k1, (32, 0), (32, 64), 0, 64, (0, 0))
+        lay = dte.Layout.from_plan(p, 0)
+        assert lay.num_receivers == 0
+        theta = torch.randn(64 * 64, device="cuda") * 0.02
+        m = torch.randn(64 * 64, device="cuda") * 1e-2
+        v = torch.rand(64 * 64, device="cuda") * 1e-6
+        d = lay.new_delta(64 * 64)
+        dte.dte_extract_delta(lay, lay.source_tables([theta], [m], [v]), 10, 1e-3, 0.9, 0.999, 1e-8, 0.0, d)
+        torch.cuda.synchronize()
+        assert d.status_bits() == 0 and d.total() > 0
+        with pytest.raises(dte.DteError) as e:
+            dte.dte_extract_delta_push(lay, lay.source_tables([theta], [m], [v]), 10, 1e-3, 0.9, 0.999, 1e-8, 0.0,
+                                       d, [], 1)
+        assert e.value.status == 2
+
+
 def test_push_into_a_second_gpus_memory_when_there_is_one():
     """The intended deployment: the landing buffers live on the receiver's GPU and the sender's
     gather kernel stores into them through peer access.  Needs two GPUs that can reach each other
