@@ -158,7 +158,7 @@ DTE_API size_t dte_layout_num_groups(const dte_layout* layout);
 /* Elements one extract call scans (sum of extents; replicated tensors count per copy). */
 DTE_API uint64_t dte_layout_num_elements(const dte_layout* layout);
 /* Bytes of device workspace dte_extract_delta_host needs (12 bytes per source element,
- * each tensor padded to 256 bytes). */
+ * each tensor padded to 256 bytes); UINT64_MAX if the sum does not fit 64 bits. */
 DTE_API uint64_t dte_layout_host_workspace_bytes(const dte_layout* layout);
 
 /* The call-uniform fp32 scalars of Eq. 2, derived in double and rounded once:

@@ -122,7 +122,10 @@ extern "C" uint64_t dte_layout_host_workspace_bytes(const dte_layout* L) {
     if (!L) return 0;
     uint64_t b = 0;
     for (size_t p = 0; p < L->tensor_numel.size(); ++p)
-        if (L->tensor_used[p]) b += 3 * ((L->tensor_numel[p] * 4 + 255) / 256 * 256);
+        if (L->tensor_used[p]) {
+            if (L->tensor_numel[p] > (uint64_t(1) << 56) || b > (uint64_t(1) << 62)) return UINT64_MAX;   // no such host
+            b += 3 * ((L->tensor_numel[p] * 4 + 255) / 256 * 256);
+        }
     return b;
 }
 
