@@ -641,8 +641,9 @@ extern "C" dte_status dte_extract_delta_static(const dte_layout* layout, const f
     s = sync_source_table(L, theta, m, v, st);
     if (s != DTE_OK) return s;
     // the array keeps whatever the previous call left - possibly a call on another layout, or one
-    // that was cut short - so the one word that must start at zero (the cursor) is cleared in the
-    // stream every time; every other part is written before it is read
+    // that was cut short - so the two words that must start at zero (the staging cursor and the
+    // count of non-finite elements) are cleared in the stream every time; every other part is
+    // written before it is read
     const Consts c{c5[0], c5[1], c5[2], c5[3], c5[4]};
     const Scratch sc{reinterpret_cast<uint64_t*>(base + kStaticCursorOff),
                      reinterpret_cast<uint64_t*>(base + kStaticRecOff),
