@@ -33,24 +33,34 @@ T_TABLE = np.array([0x3C23D70A, 0xBCA3D70A, 0x3F808000, 0x3F807FFF, 0x3F808001, 
                     0x7F7F8000, 0x00008000, 0x3F800000, 0xC77FE000, 0x3A83126F, 0xBF818000], np.uint32).view(np.float32)
 
 
-def _operands(which, lo, n):
+# A second pair of moment tables for the run with a decay far from 1 (0.9): there the division
+# moves every normal theta out of its BF16 cell, and the decision is at its threshold only in the
+# lowest BF16 cells (|theta| < 2^-126), where a cell is as wide as its values.  These moments give
+# steps of 0 and of about a quarter, one and three of those cells (2^-133) next to ordinary ones.
+M_TABLE_TINY = np.array([1.4e-30, -1.4e-30, 0.0, 5.6e-30, -1.7e-29, 3e-4, -3e-31], np.float32)          # period 7
+V_TABLE_TINY = np.array([1e18, 1e18, 1e-6, 1e18, 4e18, 1e18, 0.0, 1e18, 2.5e17, 1e18, 1e18], np.float32)  # period 11
+
+
+def _operands(which, lo, n, tiny=False):
     """(theta, m, v) of elements lo .. lo+n-1: operand `which` has bit pattern i, the others cycle."""
     i = np.arange(lo, lo + n, dtype=np.int64)
     exhaustive = i.astype(np.uint32).view(np.float32)
     th = exhaustive if which == "theta" else T_TABLE[i % 13]
-    mm = exhaustive if which == "m" else M_TABLE[i % 7]
-    vv = exhaustive if which == "v" else V_TABLE[i % 11]
+    mm = exhaustive if which == "m" else (M_TABLE_TINY if tiny else M_TABLE)[i % 7]
+    vv = exhaustive if which == "v" else (V_TABLE_TINY if tiny else V_TABLE)[i % 11]
     return th, mm, vv
 
 
 HP_PLAIN = (500, 1e-6, 0.9, 0.999, 1e-8, 0.01)     # bc1 = decay = 1: no constant division
 HP_DECAY = (3, 2e-4, 0.9, 0.999, 1e-8, 0.1)         # both divisions, direction-aware screen with decay
 HP_EPS0 = (40, 1e-3, 0.8, 0.99, 0.0, 0.0)           # eps = 0: m = v = 0 gives 0/0
+HP_DECAY09 = (20, 0.1, 0.9, 0.999, 1e-8, 1.0)       # decay = 0.9, with the tiny-step tables
 
 
 @pytest.mark.parametrize("which,hp", [("theta", HP_PLAIN), ("theta", HP_DECAY), ("theta", HP_EPS0),
-                                      ("m", HP_DECAY), ("v", HP_DECAY), ("v", HP_PLAIN)],
-                         ids=["theta-plain", "theta-decay", "theta-eps0", "m-decay", "v-decay", "v-plain"])
+                                      ("m", HP_DECAY), ("v", HP_DECAY), ("v", HP_PLAIN), ("theta", HP_DECAY09)],
+                         ids=["theta-plain", "theta-decay", "theta-eps0", "m-decay", "v-decay", "v-plain",
+                              "theta-decay0.9-tiny-steps"])
 def test_every_fp32_pattern_of_one_operand(which, hp):
     free, _ = torch.cuda.mem_get_info()
     if free < 110e9:
@@ -59,7 +69,9 @@ def test_every_fp32_pattern_of_one_operand(which, hp):
     theta = torch.empty(N, dtype=torch.float32, device=dev)
     m = torch.empty(N, dtype=torch.float32, device=dev)
     v = torch.empty(N, dtype=torch.float32, device=dev)
-    tt, mt, vt = (torch.from_numpy(x.copy()).to(dev) for x in (T_TABLE, M_TABLE, V_TABLE))
+    tiny = hp is HP_DECAY09
+    tt, mt, vt = (torch.from_numpy(x.copy()).to(dev)
+                  for x in (T_TABLE, M_TABLE_TINY if tiny else M_TABLE, V_TABLE_TINY if tiny else V_TABLE))
     for lo in range(0, N, 1 << 28):
         sl = slice(lo, lo + (1 << 28))
         i = torch.arange(lo, lo + (1 << 28), dtype=torch.int64, device=dev)
@@ -97,7 +109,7 @@ def test_every_fp32_pattern_of_one_operand(which, hp):
     consts = oracle.derive_constants(*hp)
 
     def job(lo):
-        th, mm, vv = _operands(which, lo, CHUNK)
+        th, mm, vv = _operands(which, lo, CHUNK, tiny)
         mask, v16 = oracle.changed_mask(th, mm, vv, consts)
         idx = np.nonzero(mask)[0]
         prev = oracle.invert(th, mm, vv, consts)
