@@ -281,6 +281,33 @@ def test_changed_set_against_unfused_arrays(lr, step, wd):
     assert 0 < mask.sum() < mask.size
 
 
+@pytest.mark.parametrize("lr,wd", [(0.1, 1.0), (0.5, 1.0), (1e-3, 0.2), (-0.1, 1.0)])
+def test_changed_set_against_unfused_arrays_where_bf16_is_subnormal(lr, wd):
+    """The lowest BF16 cells (|theta| < 2^-126: fp32 and BF16 subnormals) with steps of up to a
+    cell and a half and a division by a decay away from 1: every intermediate here is subnormal
+    or next to it, so a flushed operand or result anywhere would show."""
+    hp = Hyper(step=20, lr=lr, wd=wd)
+    rng = np.random.default_rng(7)
+    n = 200003
+    pat = (rng.integers(0, 0x40, size=n, dtype=np.uint32) << 16) | rng.integers(0, 1 << 16, size=n, dtype=np.uint32)
+    theta = (pat | (rng.integers(0, 2, size=n, dtype=np.uint32) << 31)).view(np.float32).copy()
+    v = (2.0 ** rng.uniform(20, 60, size=n)).astype(np.float32)
+    c = oracle.derive_constants(*hp.as_args())
+    c64 = c.astype(np.float64)
+    step = rng.uniform(-1.5, 1.5, size=n) * 2.0 ** -133
+    m = (step / abs(c64[3]) * (np.sqrt(v.astype(np.float64) / c64[1]) + c64[4]) * c64[0]).astype(np.float32)
+    m[::7] = 0.0
+    prev, bt, bp = _unfused_numpy(theta, m, v, c)
+    assert np.array_equal(bits(oracle.invert(theta, m, v, c)), bits(prev))
+    mask, val = oracle.changed_mask(theta, m, v, c)
+    assert np.array_equal(mask.astype(bool), bt != bp)
+    assert np.array_equal(val, bt)
+    assert 0.05 < mask.mean() < 0.999
+    # the range is what it claims to be: subnormal operands and results
+    tiny = np.float32(2.0 ** -126)
+    assert (np.abs(theta) < tiny).mean() > 0.9 and (np.abs(prev) < tiny).mean() > 0.5
+
+
 def test_changed_set_zero_sign_and_nan_rules():
     c = oracle.derive_constants(100, 1e-6, 0.9, 0.999, 1e-8, 0.0)
     # +0 / -0 are different stored patterns
