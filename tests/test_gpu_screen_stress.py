@@ -344,3 +344,34 @@ def test_random_learning_rates_and_weight_decays_per_group_match_oracle(seed):
     lp, off, val = d.to_host()
     assert np.array_equal(lp, want[0]) and np.array_equal(off, want[1]) and np.array_equal(val, want[2])
     assert int(d.counters[3].item()) == int(odd)
+
+
+@pytest.mark.parametrize("hp", [
+    Hyper(step=500, lr=1e-6, wd=0.01),
+    Hyper(step=100, lr=1e-3, wd=0.0),
+    Hyper(step=3, lr=1e-3, wd=0.2),
+    Hyper(step=20, lr=-1e-3, wd=0.5),
+], ids=lambda h: f"t{h.step}-lr{h.lr:g}-wd{h.wd:g}")
+def test_large_steps_that_land_on_a_tie_point_match_oracle(hp):
+    """Steps solved so that the reconstruction lands within two ulps of a BF16 tie point: from a
+    theta several times smaller (of either sign), and from a theta in a cell next to that tie, where
+    the decision hangs on the last bits of the sum."""
+    rows, cols = 2048, 2048
+    n = rows * cols
+    rng = np.random.default_rng(555 + hp.step)
+    upper = rng.integers(0x2000, 0x5F00, size=n, dtype=np.uint32)
+    delta = rng.integers(-2, 3, size=n).astype(np.int64)
+    land = (((upper.astype(np.int64) << 16) + 0x8000 + delta).astype(np.uint32)
+            | (rng.integers(0, 2, size=n, dtype=np.uint32) << 31)).view(np.float32)
+    theta = (land.astype(np.float64) * rng.uniform(-0.25, 0.25, size=n)).astype(np.float32)
+    # half of the elements: theta already in the cell next to the tie, so that both outcomes occur
+    near = rng.random(n) < 0.5
+    theta[near] = (land[near].astype(np.float64) * (1.0 + rng.uniform(-3e-3, 3e-3, size=int(near.sum())))).astype(np.float32)
+    v = (2.0 ** rng.uniform(-40, 40, size=n)).astype(np.float32)
+    c = oracle.derive_constants(*hp.as_args()).astype(np.float64)
+    with np.errstate(all="ignore"):
+        step = land.astype(np.float64) * c[2] - theta.astype(np.float64)      # (theta + step) / decay = land
+        m = (step / c[3] * (np.sqrt(v.astype(np.float64) / c[1]) + c[4]) * c[0]).astype(np.float32)
+    plan = plans.single_matrix_plan(rows, cols, 2)
+    frac, _ = _run_and_compare(plan, hp, theta, m, v, n)
+    assert 0.3 < frac < 0.999
