@@ -152,6 +152,34 @@ def test_packed_tiles_next_to_regular_ones(rows, block_rows):
         assert torch.equal(d2.offsets[:d.total()], d.offsets[:d.total()])
 
 
+@pytest.mark.parametrize("tiles,packed_tail", [(4032, 0), (4095, 0), (4096, 0), (4095, 1), (4096, 1), (4097, 0), (4160, 0)])
+def test_tile_counts_around_the_switch_between_one_gather_launch_and_three(tiles, packed_tail):
+    """Up to 4096 placement records (64 gather blocks) the gather is one launch in which every
+    block scans all records; beyond, three launches.  Counts just below, at and just above the
+    switch, with the last block full and partly filled, and with a packed tile as the last
+    record or the one that crosses the limit."""
+    p = plans.Plan()
+    first = tiles // 2
+    a = p.add_tensor("rows", (tiles, 9216))            # one regular tile per row
+    k0 = p.add_shard("r0", 0, first * 9216)
+    k1 = p.add_shard("r1", 1, (tiles - first) * 9216)
+    p.add_op(a, k0, (0, 0), (first, 9216), 0, 9216, (0, 0))
+    p.add_op(a, k1, (first, 0), (tiles - first, 9216), 0, 9216, (0, 0))
+    specs = [Spec()]
+    if packed_tail:
+        b = p.add_tensor("tail", (3, 500))             # a short run: one packed tile, the last record
+        k2 = p.add_shard("r1.tail", 1, 1500)
+        p.add_op(b, k2, (0, 0), (3, 500), 0, 500, (0, 0))
+        specs.append(Spec())
+    wl = configs.Workload("switch", p, Hyper(step=50, lr=1e-5, wd=0.01), specs, 77)
+    st, lay, d, got, bufs = _full_parity(wl)
+    info = lay.last_launch()
+    n_rec = tiles + packed_tail
+    assert info["tiles"] == n_rec
+    assert info["kernels"] == (1 if n_rec <= 4096 else 3) + 1 + packed_tail
+    assert int(got[0][-1]) > tiles                     # every tile contributes
+
+
 def test_all_changed_and_none_changed():
     plan = plans.qwen3_dense_plan(1, 4, False, configs.SMALL_DENSE)
     # beta = 0.5, t = 1, m = v = 0.5, eps = 0: u = 1 exactly; lr = 8 moves every element far
