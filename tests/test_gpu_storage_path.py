@@ -14,7 +14,20 @@ from synth.tensors import Hyper, Spec
 
 pytestmark = pytest.mark.gpu
 
+def _many_small_tensors(n_tensors=4200):
+    """More tensors and more lists than the apply kernels keep list boundaries for in shared memory
+    (4096): boundaries then come from global memory."""
+    p = plans.Plan()
+    for i in range(n_tensors):
+        t = p.add_tensor(f"w{i}", (4, 96))
+        for r in range(2):
+            k = p.add_shard(f"w{i}.{r}", r, 2 * 96)
+            p.add_op(t, k, (2 * r, 0), (2, 96), 0, 96, (0, 0))
+    return p
+
+
 PLANS = {
+    "many_small_tensors": _many_small_tensors,
     "dense_tp4": lambda: plans.qwen3_dense_plan(2, 4, True, configs.SMALL_DENSE),
     "moe_tp8_ep4": lambda: plans.qwen3_moe_plan(1, 8, 4, configs.SMALL_MOE),
     "random3": lambda: plans.random_plan(1003),
