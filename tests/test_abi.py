@@ -75,3 +75,48 @@ def test_chunk_bounds_cover_what_the_oracle_writes(fmt, chunk_entries):
         assert d.shape[0] - 1 <= L.dte_chunk_count_bound(lens.size, n, chunk_entries)
         assert stream.size <= L.dte_chunk_bytes_bound(lens.size, n, chunk_entries, fmt)
     assert L.dte_chunk_count_bound(3, 100, 0) == 0
+
+
+C_PROGRAM = r"""
+#include <stdio.h>
+#include <string.h>
+#include "dte.h"
+
+int main(void) {
+    float c[5];
+    unsigned int bits[5];
+    dte_status s = dte_derive_constants(100, 1e-6, 0.9, 0.999, 1e-8, 0.01, c);
+    if (s != DTE_OK) return 2;
+    memcpy(bits, c, sizeof bits);
+    printf("%08x %08x %08x %08x %08x\n", bits[0], bits[1], bits[2], bits[3], bits[4]);
+    s = dte_derive_constants(0, 1e-6, 0.9, 0.999, 1e-8, 0.01, c);          /* step 0: refused */
+    printf("%d %s\n", (int)s, dte_status_string(s));
+    return dte_layout_num_lists(NULL) == 0 ? 0 : 3;
+}
+"""
+
+
+def test_header_is_plain_c_and_the_library_links_from_a_c_program(tmp_path):
+    """The boundary is a C ABI: the header compiles as strict C99 (and as C++11), and a C program
+    built with gcc alone links against the library and calls its host-only entry points."""
+    import shutil
+    import subprocess
+    if not shutil.which("gcc"):
+        pytest.skip("no gcc")
+    inc = os.path.join(ROOT, "include")
+    hdr = os.path.join(inc, "dte.h")
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c", hdr], check=True)
+    subprocess.run(["g++", "-std=c++11", "-Wall", "-Wextra", "-pedantic", "-Werror", "-fsyntax-only", "-x", "c++", hdr], check=True)
+    lib = dte.library_path()
+    if not os.path.exists(lib):
+        dte.lib()
+    src = tmp_path / "use_dte.c"
+    src.write_text(C_PROGRAM)
+    exe = tmp_path / "use_dte"
+    libdir = os.path.dirname(lib)
+    subprocess.run(["gcc", "-std=c99", "-Wall", "-Werror", "-I", inc, str(src), "-o", str(exe),
+                    "-L", libdir, "-l:" + os.path.basename(lib), "-Wl,-rpath," + libdir], check=True)
+    out = subprocess.run([str(exe)], check=True, capture_output=True, text=True).stdout.split("\n")
+    want = oracle.derive_constants(100, 1e-6, 0.9, 0.999, 1e-8, 0.01).view(np.uint32)
+    assert out[0].split() == [f"{int(x):08x}" for x in want[:5]]
+    assert out[1] == "1 invalid argument"
