@@ -63,8 +63,9 @@ __device__ __forceinline__ uint32_t bf16_rne_bits(float x) {
 //     s    = RN(lr * u)          S = RN(U * |lr|)                              => S >= |s|
 // (2^-10 in kb covers the 2^-22 error of the hardware rsqrt and the roundings of v/bc2, of the
 // root and of the product; rsqrt.ftz turns a subnormal v into +Inf, so W = kc there, and
-// den >= eps always.)  The step s has the sign of lr * m, because den >= +0 or NaN.  Give S that
-// sign: theta + s lies between theta and theta + S, hence
+// den >= eps always.)  The step s has the sign of lr * m, because den >= +0 or NaN.  With that
+// sign on S (it comes by itself when m and lr enter the products signed: rounding is symmetric),
+// theta + s lies between theta and theta + S, hence
 //     num = RN(theta + s)  lies between  theta  and  far = RN(theta + S)       (by value).
 // Without a division by decay the reconstruction is num: q = theta, p = far.
 // With it, recon = RN(num / decay) differs from num by at most
@@ -105,13 +106,15 @@ __device__ __forceinline__ uint32_t bf16x2_rn(float hi, float lo) {
 
 template <bool DIV_BC1, bool DIV_DECAY>
 __device__ __forceinline__ bool surely_unchanged(float theta, float m, float v, const Screen& s, float lr) {
-    const float am = DIV_BC1 ? __fmul_rn(fabsf(m), s.ka) : fabsf(m);
+    // m and lr go in with their signs: rounding is symmetric, so the product is S with the sign of
+    // lr * m, the step's (W >= +0; a negative v makes it -Inf or NaN, and the product infinite or NaN)
+    const float ms = DIV_BC1 ? __fmul_rn(m, s.ka) : m;
     const float w = min_nan(__fmul_rn(rsqrt_ftz(v), s.kb), s.kc);      // -Inf for v = -0 or a negative subnormal
-    const float sb = __fmul_rn(__fmul_rn(am, w), fabsf(lr));           // S, or -Inf / NaN
-    const uint32_t dir = (__float_as_uint(m) ^ __float_as_uint(lr)) & 0x80000000u;   // sign of the step
-    const float far = __fadd_rn(theta, __uint_as_float((__float_as_uint(sb) & 0x7FFFFFFFu) | dir));
+    const float sb = __fmul_rn(__fmul_rn(ms, w), lr);
+    const float far = __fadd_rn(theta, sb);
     if (DIV_DECAY) {
-        const float d = __uint_as_float(__float_as_uint(__fmaf_rn(fabsf(theta), s.kappa, s.tiny)) | dir);
+        const float d = __uint_as_float(__float_as_uint(__fmaf_rn(fabsf(theta), s.kappa, s.tiny)) |
+                                        (__float_as_uint(sb) & 0x80000000u));      // D, signed like S
         const uint32_t r = bf16x2_rn(__fadd_rn(far, d), __fsub_rn(theta, d));
         // halves equal, and (one test for both then) neither infinite nor NaN
         return r == __byte_perm(r, 0, 0x1032) && (r << 1) < 0xFF000000u;
